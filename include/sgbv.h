@@ -1,0 +1,127 @@
+/*
+ * sgbv.h -- C ABI of the batched multi-draft greedy block verification step (SpecTr-GBV).
+ *
+ * One call verifies, for every batch row, K i.i.d. draft blocks of gamma tokens against the
+ * target model's distributions and returns the accepted block and one extra token
+ * (Algorithm 1 of the paper with Eqs. 2, 3 and 4).  The draft and target model forwards are
+ * not part of this library: their logits are inputs.
+ *
+ * Tensor layouts (row-major, last index contiguous; "device" = CUDA device memory of the
+ * current device, "host" = ordinary or pinned host memory):
+ *   target_logits [B, K, gamma+1, V]   row (b,k,i): target logits after the first i tokens of
+ *                                      draft k, i = 0..gamma (the paper's q(. | x_k^{i}))
+ *   draft_logits  [B, K, gamma,   V]   row (b,k,i): draft logits after the same prefix
+ *                                      (the paper's p(. | x_k^{i})), i = 0..gamma-1
+ *   draft_tokens  [B, K, gamma]        int32, token i of draft k, 0 <= token < V
+ *   uniforms      [B, K*gamma + 1]     float32 in [0,1): entry k*gamma + (i-1) is the uniform eta of
+ *                                      the Bernoulli trial on the length-i sub-block of draft k
+ *                                      (Algorithm 1, lines "sample eta ~ U(0,1)"); the last entry
+ *                                      draws the extra token by inverse CDF
+ *   out_accept_len [B]                 int32 tau in 0..gamma, or -1 if the row was flagged invalid
+ *   out_draft_idx  [B]                 int32 accepted draft f in 0..K-1, -1 when tau == 0
+ *   out_tokens     [B, gamma+1]        int32: the tau accepted tokens, then the extra token y at
+ *                                      index tau, then -1 padding
+ * Probabilities are softmax(logits / temperature) of each row (one temperature for both models).
+ *
+ * Ownership: every pointer is owned by the caller; the library neither frees nor keeps it past
+ * the call.  Device entry points only enqueue work on `stream` (a cudaStream_t passed as void*;
+ * NULL = the legacy default stream) and return without synchronising: outputs are valid once the
+ * stream has been synchronised.
+ *
+ * Errors: the return value is SGBV_OK or a negative SGBV_ERR_* code found on the host before
+ * anything is launched (nothing has been written then).  Conditions found on the device never
+ * trap: they set per-row bits in the status array (SGBV_STATUS_*), and a row flagged
+ * TOKEN_RANGE or NONFINITE_LOGIT gets tau = f = -1 and tokens = -1.  There is no CPU fallback.
+ */
+#ifndef SGBV_H_
+#define SGBV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SGBV_OK 0
+#define SGBV_ERR_NULL (-1)        /* a required pointer is NULL */
+#define SGBV_ERR_SHAPE (-2)       /* B,K,gamma,V < 1, K > 64, gamma > 64, V > 2^22, unknown dtype */
+#define SGBV_ERR_TEMPERATURE (-3) /* temperature <= 0 or not finite */
+#define SGBV_ERR_ALIGN (-4)       /* a pointer is not aligned to its element size */
+#define SGBV_ERR_WORKSPACE (-5)   /* caller workspace too small or misaligned (256 B) */
+#define SGBV_ERR_CUDA (-6)        /* a CUDA runtime call failed (allocation, copy, launch) */
+
+#define SGBV_STATUS_TOKEN_RANGE 1         /* a draft token of the row is outside [0,V) */
+#define SGBV_STATUS_NONFINITE_LOGIT 2     /* NaN/+inf logit, or a row with no finite logit, among the rows read */
+#define SGBV_STATUS_DEGENERATE_RESIDUAL 4 /* Eq. 4 had zero total mass; y was drawn from q of that row */
+
+#define SGBV_DTYPE_F32 0
+#define SGBV_DTYPE_BF16 1
+
+/* Bytes of device scratch one call of the given shape needs (for sgbv_verify_ex). */
+int sgbv_workspace_bytes(int B, int K, int gamma, int V, int dtype, size_t *out_bytes);
+
+/*
+ * The verify step on float32 logits (problem statement and Algorithm 1; Eqs. 2-4).
+ * All tensor pointers are device pointers.  Scratch comes from a per-device buffer that the
+ * library grows with cudaMalloc when a larger shape is first seen (so the first call of a
+ * shape is not stream-capturable; later ones allocate nothing).
+ */
+int sgbv_verify(const float *target_logits, const float *draft_logits, const int32_t *draft_tokens,
+                const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, void *stream);
+
+/* Same with bfloat16 logits (raw 16-bit patterns), widened to float32 inside the kernels. */
+int sgbv_verify_bf16(const uint16_t *target_logits, const uint16_t *draft_logits,
+                     const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma,
+                     int V, float temperature, int32_t *out_accept_len, int32_t *out_draft_idx,
+                     int32_t *out_tokens, void *stream);
+
+/*
+ * Extended form: caller-provided scratch and diagnostics (device pointers).
+ *   dtype           SGBV_DTYPE_F32 or SGBV_DTYPE_BF16 (element type of the two logit tensors)
+ *   workspace       >= sgbv_workspace_bytes(...) bytes, 256-byte aligned, or NULL to use the
+ *                   library's own per-device buffer
+ *   out_h           [B,K,gamma] float64 or NULL: acceptance weight of the length-i sub-block at
+ *                   index i-1 (Eq. 2 for i < gamma, Eq. 3 for i = gamma), clamped to [0,1]
+ *   out_resmass     [B,K,gamma] float64 or NULL: S_i = sum_x q(x^i,x)(1-min{p(x^i,x)/q(x^i,x),1})^K,
+ *                   i = 0..gamma-1 (the vocabulary sum of Eq. 2 = normaliser of Eq. 4)
+ *   out_status      [B] int32 or NULL: SGBV_STATUS_* bits
+ */
+int sgbv_verify_ex(const void *target_logits, const void *draft_logits, int dtype,
+                   const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma, int V,
+                   float temperature, int32_t *out_accept_len, int32_t *out_draft_idx,
+                   int32_t *out_tokens, void *workspace, size_t workspace_bytes, double *out_h,
+                   double *out_resmass, int32_t *out_status, void *stream);
+
+/*
+ * Host-buffer form: every tensor pointer is a HOST pointer (pinned memory makes the copies
+ * asynchronous).  Copies the inputs to device staging buffers owned by the library, runs the
+ * verify step on `stream`, copies the three outputs (and out_status if not NULL) back and
+ * synchronises the stream before returning.
+ */
+int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dtype,
+                     const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma,
+                     int V, float temperature, int32_t *out_accept_len, int32_t *out_draft_idx,
+                     int32_t *out_tokens, int32_t *out_status, void *stream);
+
+/* Number of kernel launches the last successful call on this thread enqueued. */
+int sgbv_last_launch_count(void);
+
+/*
+ * Measurement support (not part of the method): between sgbv_profile_begin(n) and
+ * sgbv_profile_end, each of the next n verify calls records a CUDA event pair on its stream
+ * around the kernel that moves the logits (the one a memory roofline is quoted for).
+ * sgbv_profile_end waits for those events, returns their summed elapsed time in milliseconds
+ * and the number of recorded calls, and releases the events.  Not thread-safe.
+ */
+int sgbv_profile_begin(int max_records);
+int sgbv_profile_end(double *out_total_ms, int *out_records);
+
+/* Human-readable name of a return code. Never NULL. */
+const char *sgbv_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGBV_H_ */

@@ -216,20 +216,22 @@ static void verify_row(const float *zq, const float *zp, const int32_t *tok, con
     double *av = (double *)malloc((size_t)K * (gamma + 1) * sizeof(double)); /* a_i = q(x_k^i) */
     double *bv = (double *)malloc((size_t)K * (gamma + 1) * sizeof(double)); /* b_i = p(x_k^i) */
 
-    for (size_t n = 0; n < (size_t)K * (gamma + 1) * V; ++n)
-        if (isnan(zq[n]) || zq[n] == INFINITY) status |= ORACLE_STATUS_NONFINITE;
-    for (size_t n = 0; n < (size_t)K * gamma * V; ++n)
-        if (isnan(zp[n]) || zp[n] == INFINITY) status |= ORACLE_STATUS_NONFINITE;
-    for (int r = 0; r < K * (gamma + 1); ++r) { /* a row of only -inf has no softmax */
-        int any = 0;
-        for (int x = 0; x < V; ++x) any |= isfinite(zq[(size_t)r * V + x]);
-        if (!any) status |= ORACLE_STATUS_NONFINITE;
-    }
-    for (int r = 0; r < K * gamma; ++r) {
-        int any = 0;
-        for (int x = 0; x < V; ++x) any |= isfinite(zp[(size_t)r * V + x]);
-        if (!any) status |= ORACLE_STATUS_NONFINITE;
-    }
+    /* rows the method reads up front: target rows i < gamma and every draft row.  A NaN or +inf
+     * logit, or a row without any finite logit, invalidates the batch row.  (The target row
+     * i = gamma of a draft is read only after a full accept and is checked there.) */
+    for (int k = 0; k < K; ++k)
+        for (int i = 0; i < gamma; ++i) {
+            const float *rq = zq + ((size_t)k * (gamma + 1) + i) * V;
+            const float *rp = zp + ((size_t)k * gamma + i) * V;
+            int anyq = 0, anyp = 0;
+            for (int x = 0; x < V; ++x) {
+                if (isnan(rq[x]) || rq[x] == INFINITY || isnan(rp[x]) || rp[x] == INFINITY)
+                    status |= ORACLE_STATUS_NONFINITE;
+                anyq |= isfinite(rq[x]);
+                anyp |= isfinite(rp[x]);
+            }
+            if (!anyq || !anyp) status |= ORACLE_STATUS_NONFINITE;
+        }
     for (int n = 0; n < K * gamma; ++n)
         if (tok[n] < 0 || tok[n] >= V) status |= ORACLE_STATUS_TOKEN_RANGE;
 
@@ -292,14 +294,29 @@ static void verify_row(const float *zq, const float *zp, const int32_t *tok, con
                 y = sgbv_oracle_sample(q, V, us, &margin_s);
             }
         } else {
-            y = sgbv_oracle_sample(q, V, us, &margin_s);
+            int any = 0, badrow = 0; /* bonus row: checked when it is actually read */
+            for (int x = 0; x < V; ++x) {
+                badrow |= isnan(zq_row[x]) || zq_row[x] == INFINITY;
+                any |= isfinite(zq_row[x]);
+            }
+            if (badrow || !any) {
+                status |= ORACLE_STATUS_NONFINITE;
+                y = -1;
+            } else {
+                y = sgbv_oracle_sample(q, V, us, &margin_s);
+            }
         }
 
+        for (int i = 0; i <= gamma; ++i) out_tokens[i] = -1;
+        if (status & ORACLE_STATUS_NONFINITE) {
+            tau = -1;
+            f = -1;
+        } else {
+            for (int i = 0; i < tau; ++i) out_tokens[i] = tok[f * gamma + i];
+            out_tokens[tau] = y;
+        }
         *out_tau = tau;
         *out_f = f;
-        for (int i = 0; i <= gamma; ++i) out_tokens[i] = -1;
-        for (int i = 0; i < tau; ++i) out_tokens[i] = tok[f * gamma + i];
-        out_tokens[tau] = y;
         if (out_margin_accept) *out_margin_accept = margin_a;
         if (out_margin_sample) *out_margin_sample = margin_s;
         if (out_h) memcpy(out_h, h, (size_t)K * gamma * sizeof(double));

@@ -1,0 +1,218 @@
+"""Thin ctypes binding of ``libsgbv.so`` (declared in ``include/sgbv.h``).
+
+Argument marshalling only: every step of the verify path runs in the CUDA kernels behind the C
+ABI.  torch supplies device memory and the current stream.  There is no fallback of any kind: a
+missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+STATUS_TOKEN_RANGE = 1
+STATUS_NONFINITE_LOGIT = 2
+STATUS_DEGENERATE_RESIDUAL = 4
+DTYPE_F32 = 0
+DTYPE_BF16 = 1
+
+EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_verify_ex",
+           "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_status_string", "sgbv_profile_begin",
+           "sgbv_profile_end")
+
+_lib = None
+
+
+class SgbvError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(status_string(code))
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> ctypes.CDLL:
+    """Load the in-tree CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2604_25925_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = ctypes.CDLL(path)
+        vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        lib.sgbv_workspace_bytes.restype = i32
+        lib.sgbv_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
+        dev_args = [vp, vp, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp]
+        lib.sgbv_verify.restype = i32
+        lib.sgbv_verify.argtypes = dev_args
+        lib.sgbv_verify_bf16.restype = i32
+        lib.sgbv_verify_bf16.argtypes = dev_args
+        lib.sgbv_verify_ex.restype = i32
+        lib.sgbv_verify_ex.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, sz,
+                                       vp, vp, vp, vp]
+        lib.sgbv_verify_host.restype = i32
+        lib.sgbv_verify_host.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+        lib.sgbv_last_launch_count.restype = i32
+        lib.sgbv_last_launch_count.argtypes = []
+        lib.sgbv_profile_begin.restype = i32
+        lib.sgbv_profile_begin.argtypes = [i32]
+        lib.sgbv_profile_end.restype = i32
+        lib.sgbv_profile_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
+        lib.sgbv_status_string.restype = ctypes.c_char_p
+        lib.sgbv_status_string.argtypes = [i32]
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().sgbv_status_string(int(code)).decode()
+
+
+def last_launch_count() -> int:
+    return int(load().sgbv_last_launch_count())
+
+
+def profile_begin(max_records: int) -> None:
+    rc = load().sgbv_profile_begin(int(max_records))
+    if rc != OK:
+        raise SgbvError(rc)
+
+
+def profile_end():
+    """-> (summed milliseconds of the dominant kernel, number of recorded calls)."""
+    ms, n = ctypes.c_double(0.0), ctypes.c_int(0)
+    rc = load().sgbv_profile_end(ctypes.byref(ms), ctypes.byref(n))
+    if rc != OK:
+        raise SgbvError(rc)
+    return ms.value, n.value
+
+
+def workspace_bytes(B: int, K: int, gamma: int, V: int, dtype: int = DTYPE_F32) -> int:
+    out = ctypes.c_size_t(0)
+    rc = load().sgbv_workspace_bytes(B, K, gamma, V, dtype, ctypes.byref(out))
+    if rc != OK:
+        raise SgbvError(rc)
+    return int(out.value)
+
+
+@dataclass
+class VerifyOutput:
+    accept_len: torch.Tensor            # [B] int32
+    draft_idx: torch.Tensor             # [B] int32
+    tokens: torch.Tensor                # [B, gamma+1] int32
+    h: Optional[torch.Tensor] = None        # [B,K,gamma] float64
+    resmass: Optional[torch.Tensor] = None  # [B,K,gamma] float64
+    status: Optional[torch.Tensor] = None   # [B] int32
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _shapes(target_logits, draft_logits, draft_tokens, uniforms):
+    B, K, g1, V = target_logits.shape
+    gamma = g1 - 1
+    if tuple(draft_logits.shape) != (B, K, gamma, V):
+        raise ValueError(f"draft_logits shape {tuple(draft_logits.shape)} != {(B, K, gamma, V)}")
+    if tuple(draft_tokens.shape) != (B, K, gamma) or draft_tokens.dtype != torch.int32:
+        raise ValueError("draft_tokens must be int32 [B,K,gamma]")
+    if tuple(uniforms.shape) != (B, K * gamma + 1) or uniforms.dtype != torch.float32:
+        raise ValueError("uniforms must be float32 [B,K*gamma+1]")
+    if draft_logits.dtype != target_logits.dtype:
+        raise TypeError("target and draft logits must have the same dtype")
+    for t in (target_logits, draft_logits, draft_tokens, uniforms):
+        if not t.is_contiguous():
+            raise ValueError("inputs must be contiguous")
+    return B, K, gamma, V
+
+
+def sgbv_verify(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                out: Optional[VerifyOutput] = None) -> VerifyOutput:
+    """Plain entry point (``sgbv_verify`` / ``sgbv_verify_bf16``) on CUDA tensors, current stream."""
+    B, K, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    for t in (target_logits, draft_logits, draft_tokens, uniforms):
+        if not t.is_cuda:
+            raise ValueError("sgbv_verify takes CUDA tensors (use sgbv_verify_host for host buffers)")
+    dev = target_logits.device
+    if out is None:
+        out = VerifyOutput(torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty((B, gamma + 1), dtype=torch.int32, device=dev))
+    fn = load().sgbv_verify if _dtype_code(target_logits) == DTYPE_F32 else load().sgbv_verify_bf16
+    with torch.cuda.device(dev):
+        rc = fn(target_logits.data_ptr(), draft_logits.data_ptr(), draft_tokens.data_ptr(),
+                uniforms.data_ptr(), B, K, gamma, V, float(temperature), out.accept_len.data_ptr(),
+                out.draft_idx.data_ptr(), out.tokens.data_ptr(), torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                   workspace: Optional[torch.Tensor] = None, diagnostics: bool = True,
+                   out: Optional[VerifyOutput] = None) -> VerifyOutput:
+    """Extended entry point: optional caller workspace (uint8 CUDA tensor) and diagnostics."""
+    B, K, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    if not target_logits.is_cuda:
+        raise ValueError("sgbv_verify_ex takes CUDA tensors")
+    if out is None:
+        out = VerifyOutput(torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty((B, gamma + 1), dtype=torch.int32, device=dev))
+    if diagnostics and out.h is None:
+        out.h = torch.empty((B, K, gamma), dtype=torch.float64, device=dev)
+        out.resmass = torch.empty((B, K, gamma), dtype=torch.float64, device=dev)
+        out.status = torch.empty(B, dtype=torch.int32, device=dev)
+    ws_ptr, ws_bytes = (workspace.data_ptr(), workspace.numel() * workspace.element_size()) \
+        if workspace is not None else (None, 0)
+    with torch.cuda.device(dev):
+        rc = load().sgbv_verify_ex(
+            target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+            draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, V, float(temperature),
+            out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(), ws_ptr, ws_bytes,
+            out.h.data_ptr() if out.h is not None else None,
+            out.resmass.data_ptr() if out.resmass is not None else None,
+            out.status.data_ptr() if out.status is not None else None,
+            torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_verify_host(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                     out: Optional[VerifyOutput] = None, device: int = 0) -> VerifyOutput:
+    """Host-buffer entry point: CPU tensors in (pinned for asynchronous copies), CPU tensors out.
+    Returns after the stream has been synchronised."""
+    B, K, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    for t in (target_logits, draft_logits, draft_tokens, uniforms):
+        if t.is_cuda:
+            raise ValueError("sgbv_verify_host takes host tensors")
+    if out is None:
+        out = VerifyOutput(torch.empty(B, dtype=torch.int32).pin_memory(),
+                           torch.empty(B, dtype=torch.int32).pin_memory(),
+                           torch.empty((B, gamma + 1), dtype=torch.int32).pin_memory(),
+                           status=torch.empty(B, dtype=torch.int32).pin_memory())
+    with torch.cuda.device(device):
+        rc = load().sgbv_verify_host(
+            target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+            draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, V, float(temperature),
+            out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(),
+            out.status.data_ptr() if out.status is not None else None,
+            torch.cuda.current_stream(device).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out

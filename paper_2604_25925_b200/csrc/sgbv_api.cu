@@ -1,0 +1,308 @@
+// C ABI of the verify step: argument checks, scratch carving, launch sequence, host-buffer form.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+
+#include <mutex>
+
+#include "sgbv_common.cuh"
+
+namespace sgbv {
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxDevices = 64;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+Shape make_shape(int B, int K, int gamma, int V, float temperature) {
+    Shape s;
+    s.B = B;
+    s.K = K;
+    s.gamma = gamma;
+    s.V = V;
+    s.ntiles = (V + kTile - 1) / kTile;
+    const long rows = (long)B * K * gamma;
+    long want = (4L * 148 + rows - 1) / rows;  // enough slices to fill the machine a few times over
+    if (want < 1) want = 1;
+    if (want > s.ntiles) want = s.ntiles;
+    s.tiles_per_slice = (int)((s.ntiles + want - 1) / want);
+    s.nsplit = (s.ntiles + s.tiles_per_slice - 1) / s.tiles_per_slice;
+    s.scale = (float)((double)kLog2e / (double)temperature);
+    s.inv_T = 1.0 / (double)temperature;
+    return s;
+}
+
+struct Carve {
+    size_t rows, chain_end, part, wpart, dpart, mpart, h, resmass, status, total;
+};
+
+Carve carve(const Shape &s) {
+    const size_t NR = (size_t)s.B * s.K * s.gamma;
+    Carve c;
+    size_t off = 0;
+    c.rows = off;      off += align_up(NR * sizeof(RowInfo));
+    c.chain_end = off; off += align_up((size_t)s.B * s.K * 2 * sizeof(double));
+    c.part = off;      off += align_up(NR * s.nsplit * 4 * sizeof(float));
+    c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.mpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.h = off;         off += align_up(NR * sizeof(double));
+    c.resmass = off;   off += align_up(NR * sizeof(double));
+    c.status = off;    off += align_up((size_t)s.B * sizeof(int32_t));
+    c.total = off;
+    return c;
+}
+
+int check_shape(int B, int K, int gamma, int V, int dtype) {
+    if (B < 1 || K < 1 || gamma < 1 || V < 1 || K > kMaxK || gamma > kMaxGamma || V > kMaxV) return SGBV_ERR_SHAPE;
+    if (dtype != SGBV_DTYPE_F32 && dtype != SGBV_DTYPE_BF16) return SGBV_ERR_SHAPE;
+    if ((double)B * K * gamma > 2.0e8) return SGBV_ERR_SHAPE;
+    return SGBV_OK;
+}
+
+// Per-device buffers owned by the library: scratch for sgbv_verify, staging for sgbv_verify_host.
+struct DeviceBuffers {
+    void *scratch = nullptr;
+    size_t scratch_bytes = 0;
+    void *stage = nullptr;
+    size_t stage_bytes = 0;
+};
+DeviceBuffers g_buf[kMaxDevices];
+std::mutex g_mu;
+
+int grow(void **ptr, size_t *have, size_t need) {
+    if (*have >= need) return SGBV_OK;
+    if (*ptr) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return SGBV_ERR_CUDA;
+        cudaFree(*ptr);
+        *ptr = nullptr;
+        *have = 0;
+    }
+    if (cudaMalloc(ptr, need) != cudaSuccess) {
+        cudaGetLastError();
+        *ptr = nullptr;
+        return SGBV_ERR_CUDA;
+    }
+    *have = need;
+    return SGBV_OK;
+}
+
+thread_local int t_last_launches = 0;
+
+// Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
+struct Profile {
+    cudaEvent_t *begin = nullptr;
+    cudaEvent_t *end = nullptr;
+    int capacity = 0;
+    int used = 0;
+};
+Profile g_prof;
+
+int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok, const float *u, int B, int K,
+                  int gamma, int V, float temperature, int32_t *out_tau, int32_t *out_f, int32_t *out_tokens,
+                  void *workspace, size_t workspace_bytes, double *out_h, double *out_resmass,
+                  int32_t *out_status, cudaStream_t stream) {
+    if (!zq || !zp || !tok || !u || !out_tau || !out_f || !out_tokens) return SGBV_ERR_NULL;
+    int rc = check_shape(B, K, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return SGBV_ERR_TEMPERATURE;
+    const size_t esz = dtype == SGBV_DTYPE_BF16 ? 2 : 4;
+    if (((uintptr_t)zq % esz) || ((uintptr_t)zp % esz) || ((uintptr_t)tok % 4) || ((uintptr_t)u % 4) ||
+        ((uintptr_t)out_tau % 4) || ((uintptr_t)out_f % 4) || ((uintptr_t)out_tokens % 4) ||
+        ((uintptr_t)out_h % 8) || ((uintptr_t)out_resmass % 8) || ((uintptr_t)out_status % 4))
+        return SGBV_ERR_ALIGN;
+
+    Launch L;
+    L.s = make_shape(B, K, gamma, V, temperature);
+    const Carve c = carve(L.s);
+    unsigned char *base = nullptr;
+    if (workspace) {
+        if (workspace_bytes < c.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
+        base = (unsigned char *)workspace;
+    } else {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total);
+        if (rc != SGBV_OK) return rc;
+        base = (unsigned char *)g_buf[dev].scratch;
+    }
+    L.ws.rows = (RowInfo *)(base + c.rows);
+    L.ws.chain_end = (double *)(base + c.chain_end);
+    L.ws.part = (float *)(base + c.part);
+    L.ws.wpart = (float *)(base + c.wpart);
+    L.ws.dpart = (float *)(base + c.dpart);
+    L.ws.mpart = (float *)(base + c.mpart);
+    L.ws.h = out_h ? out_h : (double *)(base + c.h);
+    L.ws.resmass = out_resmass ? out_resmass : (double *)(base + c.resmass);
+    L.ws.status = out_status ? out_status : (int32_t *)(base + c.status);
+    L.zq = zq;
+    L.zp = zp;
+    L.dtype = dtype;
+    L.tok = tok;
+    L.u = u;
+    L.out_tau = out_tau;
+    L.out_f = out_f;
+    L.out_tokens = out_tokens;
+    L.stream = stream;
+
+    if (g_prof.used < g_prof.capacity) {
+        L.ev_begin = g_prof.begin[g_prof.used];
+        L.ev_end = g_prof.end[g_prof.used];
+        ++g_prof.used;
+    }
+    if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+    int n1 = launch_twopass(L);
+    if (n1 < 0) return n1;
+    int n2 = launch_finish(L);
+    if (n2 < 0) return n2;
+    t_last_launches = n1 + n2;
+    return SGBV_OK;
+}
+
+}  // namespace
+}  // namespace sgbv
+
+using namespace sgbv;
+
+extern "C" {
+
+int sgbv_workspace_bytes(int B, int K, int gamma, int V, int dtype, size_t *out_bytes) {
+    if (!out_bytes) return SGBV_ERR_NULL;
+    int rc = check_shape(B, K, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    *out_bytes = carve(make_shape(B, K, gamma, V, 1.0f)).total;
+    return SGBV_OK;
+}
+
+int sgbv_verify(const float *target_logits, const float *draft_logits, const int32_t *draft_tokens,
+                const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, void *stream) {
+    return verify_device(target_logits, draft_logits, SGBV_DTYPE_F32, draft_tokens, uniforms, B, K, gamma, V,
+                         temperature, out_accept_len, out_draft_idx, out_tokens, nullptr, 0, nullptr, nullptr,
+                         nullptr, (cudaStream_t)stream);
+}
+
+int sgbv_verify_bf16(const uint16_t *target_logits, const uint16_t *draft_logits, const int32_t *draft_tokens,
+                     const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                     int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, void *stream) {
+    return verify_device(target_logits, draft_logits, SGBV_DTYPE_BF16, draft_tokens, uniforms, B, K, gamma, V,
+                         temperature, out_accept_len, out_draft_idx, out_tokens, nullptr, 0, nullptr, nullptr,
+                         nullptr, (cudaStream_t)stream);
+}
+
+int sgbv_verify_ex(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                   const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                   int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, void *workspace,
+                   size_t workspace_bytes, double *out_h, double *out_resmass, int32_t *out_status, void *stream) {
+    return verify_device(target_logits, draft_logits, dtype, draft_tokens, uniforms, B, K, gamma, V, temperature,
+                         out_accept_len, out_draft_idx, out_tokens, workspace, workspace_bytes, out_h,
+                         out_resmass, out_status, (cudaStream_t)stream);
+}
+
+int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                     const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                     int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, int32_t *out_status,
+                     void *stream_) {
+    if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !out_accept_len || !out_draft_idx ||
+        !out_tokens)
+        return SGBV_ERR_NULL;
+    int rc = check_shape(B, K, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return SGBV_ERR_TEMPERATURE;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const size_t esz = dtype == SGBV_DTYPE_BF16 ? 2 : 4;
+    const size_t n_zq = (size_t)B * K * (gamma + 1) * V * esz, n_zp = (size_t)B * K * gamma * V * esz;
+    const size_t n_tok = (size_t)B * K * gamma * 4, n_u = (size_t)B * (K * gamma + 1) * 4;
+    const size_t n_tau = (size_t)B * 4, n_tokens = (size_t)B * (gamma + 1) * 4;
+    size_t off = 0;
+    const size_t o_zq = off;     off += align_up(n_zq);
+    const size_t o_zp = off;     off += align_up(n_zp);
+    const size_t o_tok = off;    off += align_up(n_tok);
+    const size_t o_u = off;      off += align_up(n_u);
+    const size_t o_tau = off;    off += align_up(n_tau);
+    const size_t o_f = off;      off += align_up(n_tau);
+    const size_t o_tokens = off; off += align_up(n_tokens);
+    const size_t o_status = off; off += align_up(n_tau);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+    unsigned char *st = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].stage, &g_buf[dev].stage_bytes, off);
+        if (rc != SGBV_OK) return rc;
+        st = (unsigned char *)g_buf[dev].stage;
+    }
+    bool ok = true;
+    ok &= cudaMemcpyAsync(st + o_zq, target_logits, n_zq, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + o_zp, draft_logits, n_zp, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + o_tok, draft_tokens, n_tok, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(st + o_u, uniforms, n_u, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) return SGBV_ERR_CUDA;
+    rc = verify_device(st + o_zq, st + o_zp, dtype, (const int32_t *)(st + o_tok), (const float *)(st + o_u), B, K,
+                       gamma, V, temperature, (int32_t *)(st + o_tau), (int32_t *)(st + o_f),
+                       (int32_t *)(st + o_tokens), nullptr, 0, nullptr, nullptr, (int32_t *)(st + o_status), stream);
+    if (rc != SGBV_OK) return rc;
+    ok &= cudaMemcpyAsync(out_accept_len, st + o_tau, n_tau, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out_draft_idx, st + o_f, n_tau, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out_tokens, st + o_tokens, n_tokens, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (out_status)
+        ok &= cudaMemcpyAsync(out_status, st + o_status, n_tau, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaStreamSynchronize(stream) == cudaSuccess;
+    return ok ? SGBV_OK : SGBV_ERR_CUDA;
+}
+
+int sgbv_last_launch_count(void) { return t_last_launches; }
+
+int sgbv_profile_begin(int max_records) {
+    if (max_records < 1 || max_records > (1 << 20) || g_prof.capacity != 0) return SGBV_ERR_SHAPE;
+    g_prof.begin = (cudaEvent_t *)calloc((size_t)max_records, sizeof(cudaEvent_t));
+    g_prof.end = (cudaEvent_t *)calloc((size_t)max_records, sizeof(cudaEvent_t));
+    if (!g_prof.begin || !g_prof.end) return SGBV_ERR_CUDA;
+    for (int i = 0; i < max_records; ++i)
+        if (cudaEventCreate(&g_prof.begin[i]) != cudaSuccess || cudaEventCreate(&g_prof.end[i]) != cudaSuccess)
+            return SGBV_ERR_CUDA;
+    g_prof.used = 0;
+    g_prof.capacity = max_records;
+    return SGBV_OK;
+}
+
+int sgbv_profile_end(double *out_total_ms, int *out_records) {
+    if (!out_total_ms || !out_records) return SGBV_ERR_NULL;
+    if (g_prof.capacity == 0) return SGBV_ERR_SHAPE;
+    double total = 0.0;
+    bool ok = true;
+    for (int i = 0; i < g_prof.used; ++i) {
+        float ms = 0.0f;
+        ok &= cudaEventSynchronize(g_prof.end[i]) == cudaSuccess;
+        ok &= cudaEventElapsedTime(&ms, g_prof.begin[i], g_prof.end[i]) == cudaSuccess;
+        total += ms;
+    }
+    for (int i = 0; i < g_prof.capacity; ++i) {
+        cudaEventDestroy(g_prof.begin[i]);
+        cudaEventDestroy(g_prof.end[i]);
+    }
+    free(g_prof.begin);
+    free(g_prof.end);
+    *out_total_ms = total;
+    *out_records = g_prof.used;
+    g_prof = Profile();
+    return ok ? SGBV_OK : SGBV_ERR_CUDA;
+}
+
+const char *sgbv_status_string(int code) {
+    switch (code) {
+        case SGBV_OK: return "SGBV_OK";
+        case SGBV_ERR_NULL: return "SGBV_ERR_NULL: a required pointer is NULL";
+        case SGBV_ERR_SHAPE: return "SGBV_ERR_SHAPE: B,K,gamma,V out of range or unknown dtype";
+        case SGBV_ERR_TEMPERATURE: return "SGBV_ERR_TEMPERATURE: temperature must be finite and > 0";
+        case SGBV_ERR_ALIGN: return "SGBV_ERR_ALIGN: pointer not aligned to its element size";
+        case SGBV_ERR_WORKSPACE: return "SGBV_ERR_WORKSPACE: workspace too small or not 256-byte aligned";
+        case SGBV_ERR_CUDA: return "SGBV_ERR_CUDA: a CUDA runtime call failed";
+        default: return "SGBV: unknown code";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,133 @@
+// Shared device-side definitions of the verify path: workspace layout, per-row records and the
+// element arithmetic of the coupling sums (Eq. 2's vocabulary sum / Eq. 4's weights).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sgbv.h"
+
+namespace sgbv {
+
+constexpr int kTile = 1024;        // vocabulary elements per tile (granularity of the cached partial sums)
+constexpr int kMaxK = 64;
+constexpr int kMaxGamma = 64;
+constexpr int kMaxV = 1 << 22;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Per (b,k,i) row pair, i < gamma.  Written by the statistics pass, read by the reduction pass
+// and by the finishing kernel.
+struct RowInfo {
+    double log_a;   // log q(x_k^i): joint target probability of the i-token prefix
+    double log_b;   // log p(x_k^i)
+    double Zq;      // sum_x exp((zq_x - mq)/T)
+    double Zp;
+    float mq;       // row maxima of the raw logits
+    float mp;
+    float kappa;    // c * Zq / Zp with c = b/a: ratio c*p(x)/q(x) = kappa * ep/eq in row-max units
+    float c;        // c = exp(log_b - log_a), for the c < 1 branch of the numerator
+};
+
+struct Workspace {
+    RowInfo *rows;      // [B*K*gamma]
+    double *chain_end;  // [B*K][2]: log a_gamma, log b_gamma
+    float *part;        // [B*K*gamma][nsplit][4]: slice partials (mq, Zq, mp, Zp)   (two-pass path)
+    float *wpart;       // [B*K*gamma][ntiles]: sum over the tile of eq * max(1 - kappa ep/eq, 0)^K
+    float *dpart;       // [B*K*gamma][ntiles]: sum of max(kappa ep - eq, 0)               (c < 1)
+    float *mpart;       // [B*K*gamma][ntiles]: sum of eq (c - t)^2 Q(t)                    (c < 1)
+    double *h;          // [B][K][gamma]
+    double *resmass;    // [B][K][gamma]
+    int32_t *status;    // [B]
+};
+
+struct Shape {
+    int B, K, gamma, V;
+    int ntiles;   // ceil(V / kTile)
+    int nsplit;   // slices per row in the two-pass path
+    int tiles_per_slice;
+    float scale;  // log2(e) / T
+    double inv_T;
+};
+
+template <typename T>
+__device__ __forceinline__ float ld_logit(const T *p, size_t i);
+template <>
+__device__ __forceinline__ float ld_logit<float>(const float *p, size_t i) {
+    return __ldg(p + i);
+}
+template <>
+__device__ __forceinline__ float ld_logit<uint16_t>(const uint16_t *p, size_t i) {
+    return __uint_as_float(((uint32_t)__ldg(p + i)) << 16);
+}
+
+// exp((z - m)/T) as 2^((z-m)*scale).
+__device__ __forceinline__ float expo(float z, float m, float scale) { return exp2f((z - m) * scale); }
+
+// One vocabulary element of the coupling sums, in row-max units (eq = exp((zq-mq)/T) etc.).
+//   w  = eq * max(1 - kappa*ep/eq, 0)^K       -> sum/Zq = R_i, and w is Eq. 4's weight
+//   dp = max(kappa*ep - eq, 0)                 -> sum/Zq = sum_x max(c p - q, 0)
+//   m2 = eq * (c - t)^2 * Q(t), t = min(kappa*ep/eq, 1),
+//        Q(t) = sum_{m=0}^{K-2} (K-1-m) (1-c)^(K-2-m) (1-t)^m
+// For c < 1 the numerator of Eq. 2 over a_i equals  sum(m2)/Zq + K (1-c)^(K-1) sum(dp)/Zq,
+// a sum of non-negative terms (no cancellation); for c >= 1 it equals sum(w)/Zq.
+template <bool kNeedAux>
+__device__ __forceinline__ void element_terms(float eq, float ep, float kappa, float c, int K, float &w,
+                                              float &dp, float &m2) {
+    float diff = fmaf(-kappa, ep, eq);
+    float d = fmaxf(diff, 0.0f);
+    float r = (eq > 0.0f) ? __fdividef(d, eq) : 0.0f;  // r = 1 - t in [0,1]
+    float pw = d;
+    for (int j = 1; j < K; ++j) pw *= r;
+    w = pw;
+    if (kNeedAux) {
+        dp = fmaxf(-diff, 0.0f);
+        float v = 1.0f - c;
+        float acc = (K >= 2) ? 1.0f : 0.0f;
+        float vj = 1.0f;
+        for (int j = 1; j <= K - 2; ++j) {
+            vj *= v;
+            acc = fmaf(acc, r, (float)(j + 1) * vj);
+        }
+        float ct = c - 1.0f + r;  // c - t
+        m2 = eq * ct * ct * acc;
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Host-side launchers (one translation unit each).
+struct Launch {
+    const void *zq;
+    const void *zp;
+    int dtype;
+    const int32_t *tok;
+    const float *u;
+    Shape s;
+    Workspace ws;
+    int32_t *out_tau;
+    int32_t *out_f;
+    int32_t *out_tokens;
+    cudaStream_t stream;
+    cudaEvent_t ev_begin = nullptr;  // optional: recorded around the dominant kernel
+    cudaEvent_t ev_end = nullptr;
+};
+
+int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
+int launch_finish(const Launch &L);   // weights, scan, extra token
+
+}  // namespace sgbv

@@ -1,0 +1,221 @@
+// Generic two-sweep path: works for any V, any alignment, either dtype.
+//   sweep 1  (rowstats_kernel)  slice-wise (max, sum-exp) of every target and draft row i < gamma
+//   chain    (chain_kernel)     per draft: row normalisers, log a_i / log b_i, c_i, kappa_i
+//   sweep 2  (otreduce_kernel)  per-tile sums of the residual weights (and of the two
+//                               non-negative numerator terms when c_i < 1)
+// It reads each needed logit twice, so it is the fallback, not the fast path.
+#include "sgbv_common.cuh"
+
+namespace sgbv {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+rowstats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shape s, float *__restrict__ part,
+                int32_t *__restrict__ status) {
+    const int r = blockIdx.x / s.nsplit;  // row pair (b,k,i), i < gamma
+    const int sl = blockIdx.x % s.nsplit;
+    const int i = r % s.gamma;
+    const int bk = r / s.gamma;
+    const T *zq = zq_all + ((size_t)bk * (s.gamma + 1) + i) * s.V;
+    const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
+    const int x0 = sl * s.tiles_per_slice * kTile;
+    const int x1 = min(s.V, x0 + s.tiles_per_slice * kTile);
+
+    __shared__ float red[4][kThreads / 32];
+    __shared__ float bcast[2];
+
+    float mq = -INFINITY, mp = -INFINITY;
+    bool bad = false;
+    for (int x = x0 + threadIdx.x; x < x1; x += kThreads) {
+        float a = ld_logit(zq, x), b = ld_logit(zp, x);
+        bad |= (a != a) | (b != b) | (a == INFINITY) | (b == INFINITY);
+        mq = fmaxf(mq, a);
+        mp = fmaxf(mp, b);
+    }
+    mq = warp_max(mq);
+    mp = warp_max(mp);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) {
+        red[0][wid] = mq;
+        red[1][wid] = mp;
+    }
+    if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status + bk / s.K, SGBV_STATUS_NONFINITE_LOGIT);
+    if (threadIdx.x == 0) {
+        float a = red[0][0], b = red[1][0];
+        for (int w = 1; w < kThreads / 32; ++w) {
+            a = fmaxf(a, red[0][w]);
+            b = fmaxf(b, red[1][w]);
+        }
+        bcast[0] = a;
+        bcast[1] = b;
+    }
+    __syncthreads();
+    mq = bcast[0];
+    mp = bcast[1];
+    float sq = 0.0f, sp = 0.0f;
+    if (mq > -INFINITY || mp > -INFINITY) {
+        for (int x = x0 + threadIdx.x; x < x1; x += kThreads) {
+            if (mq > -INFINITY) sq += expo(ld_logit(zq, x), mq, s.scale);
+            if (mp > -INFINITY) sp += expo(ld_logit(zp, x), mp, s.scale);
+        }
+    }
+    sq = warp_sum(sq);
+    sp = warp_sum(sp);
+    if (lane == 0) {
+        red[2][wid] = sq;
+        red[3][wid] = sp;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float a = 0.0f, b = 0.0f;
+        for (int w = 0; w < kThreads / 32; ++w) {
+            a += red[2][w];
+            b += red[3][w];
+        }
+        float *o = part + ((size_t)r * s.nsplit + sl) * 4;
+        o[0] = mq;
+        o[1] = a;
+        o[2] = mp;
+        o[3] = b;
+    }
+}
+
+// One thread per draft chain (b,k): sequential over the gamma positions.
+template <typename T>
+__global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all,
+                             const int32_t *__restrict__ tok, Shape s, const float *__restrict__ part,
+                             RowInfo *__restrict__ rows, double *__restrict__ chain_end,
+                             int32_t *__restrict__ status) {
+    const int bk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (bk >= s.B * s.K) return;
+    double la = 0.0, lb = 0.0;
+    for (int i = 0; i < s.gamma; ++i) {
+        const int r = bk * s.gamma + i;
+        const float *p = part + (size_t)r * s.nsplit * 4;
+        float mq = -INFINITY, mp = -INFINITY;
+        for (int sl = 0; sl < s.nsplit; ++sl) {
+            mq = fmaxf(mq, p[sl * 4 + 0]);
+            mp = fmaxf(mp, p[sl * 4 + 2]);
+        }
+        double Zq = 0.0, Zp = 0.0;
+        for (int sl = 0; sl < s.nsplit; ++sl) {
+            if (p[sl * 4 + 0] > -INFINITY) Zq += (double)p[sl * 4 + 1] * exp2((double)(p[sl * 4 + 0] - mq) * (double)s.scale);
+            if (p[sl * 4 + 2] > -INFINITY) Zp += (double)p[sl * 4 + 3] * exp2((double)(p[sl * 4 + 2] - mp) * (double)s.scale);
+        }
+        if (!(mq > -INFINITY) || !(mp > -INFINITY)) atomicOr(status + bk / s.K, SGBV_STATUS_NONFINITE_LOGIT);
+        RowInfo ri;
+        ri.log_a = la;
+        ri.log_b = lb;
+        ri.Zq = Zq;
+        ri.Zp = Zp;
+        ri.mq = mq;
+        ri.mp = mp;
+        double c = exp(lb - la);
+        ri.c = (float)c;
+        ri.kappa = (float)(c * Zq / Zp);
+        rows[r] = ri;
+        int t = tok[r];
+        if (t < 0 || t >= s.V) {
+            atomicOr(status + bk / s.K, SGBV_STATUS_TOKEN_RANGE);
+            t = 0;
+        }
+        const float zqt = ld_logit(zq_all, ((size_t)bk * (s.gamma + 1) + i) * s.V + t);
+        const float zpt = ld_logit(zp_all, ((size_t)bk * s.gamma + i) * s.V + t);
+        la += ((double)zqt - (double)mq) * s.inv_T - log(Zq);
+        lb += ((double)zpt - (double)mp) * s.inv_T - log(Zp);
+    }
+    chain_end[2 * bk + 0] = la;
+    chain_end[2 * bk + 1] = lb;
+}
+
+template <typename T, bool kNeedAux>
+__device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int t0,
+                                             int t1, float *wpart, float *dpart, float *mpart,
+                                             float (*red)[kThreads / 32]) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int t = t0; t < t1; ++t) {
+        const int x0 = t * kTile, x1 = min(s.V, x0 + kTile);
+        float sw = 0.0f, sd = 0.0f, sm = 0.0f;
+        for (int x = x0 + threadIdx.x; x < x1; x += kThreads) {
+            float eq = expo(ld_logit(zq, x), ri.mq, s.scale);
+            float ep = expo(ld_logit(zp, x), ri.mp, s.scale);
+            float w, dp = 0.0f, m2 = 0.0f;
+            element_terms<kNeedAux>(eq, ep, ri.kappa, ri.c, s.K, w, dp, m2);
+            sw += w;
+            sd += dp;
+            sm += m2;
+        }
+        sw = warp_sum(sw);
+        if (kNeedAux) {
+            sd = warp_sum(sd);
+            sm = warp_sum(sm);
+        }
+        if (lane == 0) {
+            red[0][wid] = sw;
+            red[1][wid] = sd;
+            red[2][wid] = sm;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float a = 0.0f, b = 0.0f, c = 0.0f;
+            for (int w = 0; w < kThreads / 32; ++w) {
+                a += red[0][w];
+                b += red[1][w];
+                c += red[2][w];
+            }
+            wpart[t] = a;
+            dpart[t] = b;
+            mpart[t] = c;
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shape s,
+                const RowInfo *__restrict__ rows, float *__restrict__ wpart, float *__restrict__ dpart,
+                float *__restrict__ mpart) {
+    const int r = blockIdx.x / s.nsplit;
+    const int sl = blockIdx.x % s.nsplit;
+    const int i = r % s.gamma;
+    const int bk = r / s.gamma;
+    const T *zq = zq_all + ((size_t)bk * (s.gamma + 1) + i) * s.V;
+    const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
+    __shared__ float red[3][kThreads / 32];
+    const RowInfo ri = rows[r];
+    const int t0 = sl * s.tiles_per_slice, t1 = min(s.ntiles, t0 + s.tiles_per_slice);
+    float *wp = wpart + (size_t)r * s.ntiles, *dp = dpart + (size_t)r * s.ntiles, *mp = mpart + (size_t)r * s.ntiles;
+    if (ri.c < 1.0f)
+        reduce_tiles<T, true>(zq, zp, s, ri, t0, t1, wp, dp, mp, red);
+    else
+        reduce_tiles<T, false>(zq, zp, s, ri, t0, t1, wp, dp, mp, red);
+}
+
+template <typename T>
+int run(const Launch &L) {
+    const Shape &s = L.s;
+    const int NR = s.B * s.K * s.gamma;
+    const unsigned grid = (unsigned)NR * (unsigned)s.nsplit;
+    const T *zq = (const T *)L.zq, *zp = (const T *)L.zp;
+    rowstats_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.part, L.ws.status);
+    const int nbk = s.B * s.K;
+    chain_kernel<T><<<(nbk + 127) / 128, 128, 0, L.stream>>>(zq, zp, L.tok, s, L.ws.part, L.ws.rows,
+                                                            L.ws.chain_end, L.ws.status);
+    if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
+    otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, L.ws.wpart, L.ws.dpart, L.ws.mpart);
+    if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
+    return cudaGetLastError() == cudaSuccess ? 3 : SGBV_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_twopass(const Launch &L) {
+    return L.dtype == SGBV_DTYPE_BF16 ? run<uint16_t>(L) : run<float>(L);
+}
+
+}  // namespace sgbv

@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA path (through the C ABI) against the float64 oracle on the same seeded
+inputs.  Rules are those of ``oracle/compare.py``: decisions bit-exact except rows within 1e-6 of
+a threshold (counted), weights and residual masses within 1e-5 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle.compare import compare
+from paper_2604_25925_b200 import binding, workloads
+from treemodel import chi_square, gbv_single_draft, np_softmax
+
+pytestmark = pytest.mark.gpu
+
+
+def _to_np32(t):
+    return t.detach().to("cpu", torch.float32).numpy()
+
+
+def run_both(inp, rows=None, host_inp=None):
+    """GPU on the whole batch; oracle on the batch rows `rows` (all if None). Returns the report."""
+    cfg = inp.cfg
+    out = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                 cfg.temperature)
+    torch.cuda.synchronize()
+    sel = slice(None) if rows is None else torch.as_tensor(rows, device=inp.target_logits.device)
+    ref = oracle.verify(_to_np32(inp.target_logits[sel]), _to_np32(inp.draft_logits[sel]),
+                        inp.draft_tokens[sel].cpu().numpy(), inp.uniforms[sel].cpu().numpy(), cfg.temperature)
+    rep = compare(ref, out.accept_len[sel].cpu().numpy(), out.draft_idx[sel].cpu().numpy(),
+                  out.tokens[sel].cpu().numpy(), out.h[sel].cpu().numpy(), out.resmass[sel].cpu().numpy(),
+                  out.status[sel].cpu().numpy())
+    print(cfg.name, rep.summary())
+    for d in rep.detail:
+        print("   ", d)
+    return rep, out, ref
+
+
+def assert_parity(rep):
+    assert rep.decision_mismatches == 0, rep.detail
+    assert rep.status_mismatches == 0, rep.detail
+    assert rep.h_violations == 0, rep.detail
+    assert rep.S_violations == 0, rep.detail
+    assert rep.threshold_exceptions <= max(2, rep.rows // 100)
+
+
+def test_config1_parity_and_20000_trials():
+    cfg = workloads.CONFIGS["c1"]
+    inp = workloads.make_inputs(cfg).to("cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+    # 20,000 trials on fixed logits/tokens with fresh uniforms: exact parity row by row and the
+    # empirical law of (tau, f, y) against the exhaustively enumerated law
+    n = 20000
+    big = workloads.VerifyInputs(
+        workloads.with_batch(cfg, n),
+        inp.target_logits.expand(n, -1, -1, -1).contiguous(), inp.draft_logits.expand(n, -1, -1, -1).contiguous(),
+        inp.draft_tokens.expand(n, -1, -1).contiguous(),
+        workloads.make_uniforms(n, cfg.K, cfg.gamma, seed=cfg.seed + 1, device="cuda"))
+    rep, out, ref = run_both(big)
+    assert_parity(rep)
+    from test_oracle_montecarlo import _chi2_critical, _exact_law_fixed_drafts
+    law = _exact_law_fixed_drafts(_to_np32(inp.target_logits)[0], _to_np32(inp.draft_logits)[0],
+                                  inp.draft_tokens.cpu().numpy()[0], cfg.temperature, cfg.K)
+    tau = out.accept_len.cpu().numpy()
+    f = out.draft_idx.cpu().numpy()
+    tokens = out.tokens.cpu().numpy()
+    counts = {}
+    for t, ff, row in zip(tau, f, tokens):
+        key = (int(t), int(ff), int(row[t]))
+        counts[key] = counts.get(key, 0) + 1
+    stat, dof = chi_square(counts, law)
+    assert stat < _chi2_critical(dof), (stat, dof)
+    assert abs(rep.block_efficiency_got - rep.block_efficiency_ref) < 1e-3
+
+
+def test_config2_parity_full():
+    inp = workloads.make_inputs(workloads.CONFIGS["c2"], device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+
+
+def test_config3_bf16_parity_full():
+    inp = workloads.make_inputs(workloads.CONFIGS["c3"], device="cuda")
+    assert inp.target_logits.dtype == torch.bfloat16
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+
+
+def test_config4_parity_sampled_rows():
+    """Full-size launch (the configuration the benchmark times); the oracle recomputes a sample of
+    whole batch rows, which are independent units."""
+    inp = workloads.make_inputs(workloads.CONFIGS["c4"], device="cuda")
+    rep, out, _ = run_both(inp, rows=[0, 7, 21, 38, 50, 63])
+    assert_parity(rep)
+    # properties that hold at any size, on all rows
+    tau = out.accept_len.cpu().numpy()
+    f = out.draft_idx.cpu().numpy()
+    tokens = out.tokens.cpu().numpy()
+    tok = inp.draft_tokens.cpu().numpy()
+    cfg = inp.cfg
+    assert ((tau >= 0) & (tau <= cfg.gamma)).all()
+    assert ((f == -1) == (tau == 0)).all()
+    for b in range(cfg.B):
+        assert list(tokens[b, :tau[b]]) == list(tok[b, f[b], :tau[b]])
+        assert 0 <= tokens[b, tau[b]] < cfg.V and (tokens[b, tau[b] + 1:] == -1).all()
+    h = out.h.cpu().numpy()
+    assert ((h >= 0) & (h <= 1)).all()
+
+
+@pytest.mark.parametrize("K", [1, 2, 4, 8])
+def test_config5_sweep_parity_sampled_rows(K):
+    rows = list(range(0, 256, 16))
+    for cfg in [c for c in workloads.sweep_c5() if c.K == K]:
+        inp = workloads.make_inputs(cfg, device="cuda")
+        rep, out, ref = run_both(inp, rows=rows)
+        assert_parity(rep)
+        if K == 1:   # K = 1 must reproduce single-draft GBV
+            zq, zp = _to_np32(inp.target_logits), _to_np32(inp.draft_logits)
+            tok, u = inp.draft_tokens.cpu().numpy(), inp.uniforms.cpu().numpy()
+            for b in rows[:4]:
+                q_rows = [np_softmax(zq[b, 0, i], cfg.temperature) for i in range(cfg.gamma + 1)]
+                p_rows = [np_softmax(zp[b, 0, i], cfg.temperature) for i in range(cfg.gamma)]
+                alpha, tau, y = gbv_single_draft(q_rows, p_rows, tok[b, 0], u[b, :cfg.gamma], float(u[b, cfg.gamma]))
+                np.testing.assert_allclose(out.h[b, 0].cpu().numpy(), alpha, rtol=1e-5, atol=1e-9)
+                if min(abs(u[b, j] - alpha[j]) for j in range(cfg.gamma)) > 1e-6:
+                    assert int(out.accept_len[b]) == tau
+
+
+EDGE_SHAPES = [
+    # B, K, gamma, V
+    (3, 1, 1, 1), (2, 2, 3, 7), (5, 3, 2, 1000), (2, 2, 2, 1025), (2, 4, 3, 32001), (1, 1, 1, 5000),
+    (4, 8, 1, 333), (1, 64, 2, 50), (2, 2, 64, 40), (1, 5, 7, 4099),
+]
+
+
+@pytest.mark.parametrize("B,K,gamma,V", EDGE_SHAPES)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_edge_shapes(B, K, gamma, V, dtype):
+    cfg = workloads.VerifyConfig(f"edge_{B}_{K}_{gamma}_{V}_{dtype}", B=B, K=K, gamma=gamma, V=V, dtype=dtype,
+                                 temperature=0.9, alpha=0.8, boost=4.0, seed=4242 + V)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+
+
+def test_unaligned_views_and_repeated_calls_are_deterministic():
+    cfg = workloads.VerifyConfig("unaligned", B=3, K=2, gamma=3, V=4099, alpha=0.8, seed=99)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    # place the logits one element past a 16-byte boundary
+    def shifted(t):
+        buf = torch.empty(t.numel() + 1, dtype=t.dtype, device=t.device)
+        v = buf[1:].view(t.shape)
+        v.copy_(t)
+        return v
+    sh = workloads.VerifyInputs(cfg, shifted(inp.target_logits), shifted(inp.draft_logits), inp.draft_tokens,
+                                inp.uniforms)
+    assert sh.target_logits.data_ptr() % 16 != 0
+    rep, out1, _ = run_both(sh)
+    assert_parity(rep)
+    out2 = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                  cfg.temperature)
+    out3 = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                  cfg.temperature)
+    torch.cuda.synchronize()
+    for a, b in ((out2, out3), (out1, out2)):
+        assert torch.equal(a.accept_len, b.accept_len) and torch.equal(a.tokens, b.tokens)
+        assert torch.equal(a.h, b.h) and torch.equal(a.resmass, b.resmass)
+
+
+def test_degenerate_and_flagged_rows():
+    cfg = workloads.VerifyConfig("flags", B=6, K=2, gamma=2, V=300, alpha=0.8, seed=7)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    zq, zp = inp.target_logits.clone(), inp.draft_logits.clone()
+    tok, u = inp.draft_tokens.clone(), inp.uniforms.clone()
+    zp[1] = zq[1, :, :2]                 # row 1: p == q everywhere -> zero residual mass
+    u[1, :4] = 0.999
+    tok[2, 1, 0] = 300                   # row 2: token out of range
+    zq[3, 0, 1, 17] = float("nan")       # row 3: NaN logit
+    zp[4, 1, 0, 5] = float("inf")        # row 4: +inf logit
+    zq[5, :, :, 11] = float("-inf")      # row 5: -inf is allowed (probability 0)
+    zp[5, :, :, 12] = float("-inf")
+    mod = workloads.VerifyInputs(cfg, zq, zp, tok, u)
+    rep, out, ref = run_both(mod)
+    assert_parity(rep)
+    st = out.status.cpu().numpy()
+    assert st[1] & binding.STATUS_DEGENERATE_RESIDUAL
+    assert st[2] & binding.STATUS_TOKEN_RANGE and st[3] & binding.STATUS_NONFINITE_LOGIT
+    assert st[4] & binding.STATUS_NONFINITE_LOGIT and st[0] == 0 and (st[5] & 3) == 0
+    assert (out.tokens[2:5].cpu().numpy() == -1).all() and (out.accept_len[2:5].cpu().numpy() == -1).all()
+
+
+def test_plain_bf16_and_host_entry_points_agree_with_extended():
+    for name in ("c2",):
+        cfg = workloads.CONFIGS[name]
+        inp = workloads.make_inputs(cfg, device="cuda")
+        ex = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                    cfg.temperature)
+        plain = binding.sgbv_verify(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                    cfg.temperature)
+        ws = torch.empty(binding.workspace_bytes(cfg.B, cfg.K, cfg.gamma, cfg.V) + 256, dtype=torch.uint8,
+                         device="cuda")
+        off = (-ws.data_ptr()) % 256
+        ex2 = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                     cfg.temperature, workspace=ws[off:off + ws.numel() - 256])
+        host = binding.sgbv_verify_host(inp.target_logits.cpu().pin_memory(), inp.draft_logits.cpu().pin_memory(),
+                                        inp.draft_tokens.cpu().pin_memory(), inp.uniforms.cpu().pin_memory(),
+                                        cfg.temperature)
+        torch.cuda.synchronize()
+        for o in (plain, ex2):
+            assert torch.equal(o.accept_len, ex.accept_len) and torch.equal(o.tokens, ex.tokens)
+            assert torch.equal(o.draft_idx, ex.draft_idx)
+        assert torch.equal(host.accept_len, ex.accept_len.cpu()) and torch.equal(host.tokens, ex.tokens.cpu())
+        assert binding.last_launch_count() > 0
+    small = workloads.VerifyConfig("bf", B=2, K=2, gamma=2, V=2048, dtype="bf16", seed=5)
+    inp = workloads.make_inputs(small, device="cuda")
+    a = binding.sgbv_verify(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, 1.0)
+    b = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, 1.0)
+    torch.cuda.synchronize()
+    assert torch.equal(a.tokens, b.tokens)
