@@ -21,6 +21,7 @@ class ParityReport:
     rows: int = 0
     rows_compared: int = 0
     threshold_exceptions: int = 0     # rows excused by the |u - threshold| < margin rule
+    exceptions_matching: int = 0      # excused rows that agree anyway
     decision_mismatches: int = 0      # rows outside the exception rule that differ
     status_mismatches: int = 0
     h_max_rel: float = 0.0
@@ -57,6 +58,7 @@ def compare(ref, tau, f, tokens, h=None, S=None, status=None, margin: float = 1e
     rep.rows_compared = int(check.sum())
     same = (tau == ref.tau) & (f == ref.f) & (tokens == ref.tokens).all(axis=1)
     bad = check & ~same
+    rep.exceptions_matching = int((excused & same).sum())
     rep.decision_mismatches = int(bad.sum())
     for b in np.nonzero(bad)[0][:8]:
         rep.detail.append(("decision", int(b), int(ref.tau[b]), int(tau[b]), int(ref.f[b]), int(f[b]),
