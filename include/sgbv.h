@@ -105,6 +105,36 @@ int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dt
                      int V, float temperature, int32_t *out_accept_len, int32_t *out_draft_idx,
                      int32_t *out_tokens, int32_t *out_status, void *stream);
 
+/*
+ * Allocation-free form of sgbv_verify_ex (the paper has no counterpart: this entry point exists
+ * for deployment, not for the method).
+ *
+ * Who needs it: a serving process that hands all free device memory to its own pool or KV cache
+ * at start-up cannot count on a later cudaMalloc succeeding, and a latency-critical decode loop
+ * cannot afford the device-wide synchronisation a cudaMalloc or cudaFree implies.  This call
+ * never allocates or frees: not with cudaMalloc/cudaFree, not through any library routine.
+ *
+ * Where the scratch lives: in a fixed array of SGBV_STATIC_SCRATCH_BYTES that is part of the
+ * library's device image; every GPU that loads the library holds it until the process exits.
+ * A shape whose sgbv_workspace_bytes(...) exceeds that size is refused with SGBV_ERR_WORKSPACE
+ * and nothing is launched.
+ *
+ * First call on a device: resolves the array's device address (once per device, with that
+ * device current).  Make that first call before starting any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, and it keeps the previous call's contents;
+ * the call clears what has to start at zero itself.  Two calls that overlap on the GPU (different
+ * streams, or the same shape from two threads) race on it: serialise them.
+ *
+ * Arguments, results and error codes are those of sgbv_verify_ex without the workspace pair.
+ */
+#define SGBV_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int sgbv_verify_static(const void *target_logits, const void *draft_logits, int dtype,
+                       const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma, int V,
+                       float temperature, int32_t *out_accept_len, int32_t *out_draft_idx,
+                       int32_t *out_tokens, double *out_h, double *out_resmass, int32_t *out_status,
+                       void *stream);
+
 /* Number of kernel launches the last successful call on this thread enqueued. */
 int sgbv_last_launch_count(void);
 

@@ -24,7 +24,7 @@ DTYPE_BF16 = 1
 
 EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_verify_ex",
            "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_status_string", "sgbv_profile_begin",
-           "sgbv_profile_end")
+           "sgbv_profile_end", "sgbv_verify_static")
 
 _lib = None
 
@@ -59,6 +59,8 @@ def load() -> ctypes.CDLL:
         lib.sgbv_verify_ex.restype = i32
         lib.sgbv_verify_ex.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, sz,
                                        vp, vp, vp, vp]
+        lib.sgbv_verify_static.restype = i32
+        lib.sgbv_verify_static.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp]
         lib.sgbv_verify_host.restype = i32
         lib.sgbv_verify_host.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
         lib.sgbv_last_launch_count.restype = i32
@@ -184,6 +186,42 @@ def sgbv_verify_ex(target_logits, draft_logits, draft_tokens, uniforms, temperat
             target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
             draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, V, float(temperature),
             out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(), ws_ptr, ws_bytes,
+            out.h.data_ptr() if out.h is not None else None,
+            out.resmass.data_ptr() if out.resmass is not None else None,
+            out.status.data_ptr() if out.status is not None else None,
+            torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def sgbv_verify_static(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0,
+                       out: Optional[VerifyOutput] = None) -> VerifyOutput:
+    """Allocation-free entry point: scratch is the library's fixed device array, so the library
+    itself never allocates.  For callers that cannot allocate device memory after start-up (all
+    of it already belongs to their pool) or cannot take the device-wide stall of an allocation.
+    Pass a pre-built ``out`` (with h, resmass, status tensors) to keep this wrapper from
+    allocating too.  Shapes needing more than STATIC_SCRATCH_BYTES raise SGBV_ERR_WORKSPACE;
+    calls that overlap on the GPU race on the shared scratch."""
+    B, K, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    if not target_logits.is_cuda:
+        raise ValueError("sgbv_verify_static takes CUDA tensors")
+    if out is None:
+        out = VerifyOutput(torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty(B, dtype=torch.int32, device=dev),
+                           torch.empty((B, gamma + 1), dtype=torch.int32, device=dev),
+                           torch.empty((B, K, gamma), dtype=torch.float64, device=dev),
+                           torch.empty((B, K, gamma), dtype=torch.float64, device=dev),
+                           torch.empty(B, dtype=torch.int32, device=dev))
+    with torch.cuda.device(dev):
+        rc = load().sgbv_verify_static(
+            target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+            draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, V, float(temperature),
+            out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(),
             out.h.data_ptr() if out.h is not None else None,
             out.resmass.data_ptr() if out.resmass is not None else None,
             out.status.data_ptr() if out.status is not None else None,

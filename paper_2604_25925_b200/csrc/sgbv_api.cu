@@ -256,6 +256,45 @@ int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dt
 
 int sgbv_last_launch_count(void) { return t_last_launches; }
 
+// ---- allocation-free variant ---------------------------------------------------------------------
+// Scratch for sgbv_verify_static: a fixed array inside the library's device image.  Every device
+// that loads the library holds these bytes until the process exits.  In host code the name below
+// is only a handle for the symbol, not a device address: the kernels get the address that
+// cudaGetSymbolAddress returns for the current device.
+static __device__ __align__(256) unsigned char g_static_scratch[SGBV_STATIC_SCRATCH_BYTES];
+
+namespace {
+void *g_static_ptr[kMaxDevices];  // resolved once per device, under g_mu
+}
+
+int sgbv_verify_static(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                       const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                       int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens, double *out_h,
+                       double *out_resmass, int32_t *out_status, void *stream) {
+    int rc = check_shape(B, K, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    const size_t need = carve(make_shape(B, K, gamma, V, 1.0f)).total;
+    if (need > (size_t)SGBV_STATIC_SCRATCH_BYTES) return SGBV_ERR_WORKSPACE;  // shape exceeds the fixed scratch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_static_ptr[dev]) {  // first call on this device: look the symbol up with this device current
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+                cudaGetLastError();
+                return SGBV_ERR_CUDA;
+            }
+            g_static_ptr[dev] = p;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    return verify_device(target_logits, draft_logits, dtype, draft_tokens, uniforms, B, K, gamma, V, temperature,
+                         out_accept_len, out_draft_idx, out_tokens, scratch, (size_t)SGBV_STATIC_SCRATCH_BYTES, out_h,
+                         out_resmass, out_status, (cudaStream_t)stream);
+}
+
 int sgbv_profile_begin(int max_records) {
     if (max_records < 1 || max_records > (1 << 20) || g_prof.capacity != 0) return SGBV_ERR_SHAPE;
     g_prof.begin = (cudaEvent_t *)calloc((size_t)max_records, sizeof(cudaEvent_t));
