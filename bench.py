@@ -283,7 +283,7 @@ def main():
             "hbm_gbs_step": ab["step"] / (ms_step * 1e-3) / 1e9,
             "algorithmic_bytes_per_step": ab["step"],
             "block_efficiency": be,
-            "roofline": {"bound": "hbm", "kernel": "otreduce_kernel", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": binding.last_main_kernel(), "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                          "peak_source": f"of {which}", "kernel_ms": kern_avg_ms, "launches_timed": kern_n,
                          "algorithmic_bytes_per_launch": ab["sweep"], "traffic": None},

@@ -55,6 +55,8 @@ extern "C" {
 #define SGBV_STATUS_NONFINITE_LOGIT 2     /* NaN/+inf logit, or a row with no finite logit, among the rows read */
 #define SGBV_STATUS_DEGENERATE_RESIDUAL 4 /* Eq. 4 had zero total mass; y was drawn from q of that row */
 
+#define SGBV_STATUS_TIMEOUT 8             /* a bounded device-side wait expired; the row's outputs are -1 */
+
 #define SGBV_DTYPE_F32 0
 #define SGBV_DTYPE_BF16 1
 
@@ -138,6 +140,10 @@ int sgbv_verify_static(const void *target_logits, const void *draft_logits, int 
 /* Number of kernel launches the last successful call on this thread enqueued. */
 int sgbv_last_launch_count(void);
 
+/* Name of the kernel that streamed the logits in the last successful call on this thread
+ * (the one sgbv_profile_begin/_end time). Never NULL. */
+const char *sgbv_last_main_kernel(void);
+
 /*
  * Measurement support (not part of the method): between sgbv_profile_begin(n) and
  * sgbv_profile_end, each of the next n verify calls records a CUDA event pair on its stream
@@ -147,6 +153,16 @@ int sgbv_last_launch_count(void);
  */
 int sgbv_profile_begin(int max_records);
 int sgbv_profile_end(double *out_total_ms, int *out_records);
+
+/*
+ * Tuning knobs for experiments (process-wide, not thread-safe; 0 restores the automatic choice):
+ *   "path"         1 = always the generic two-sweep kernels, 2 = the fused single-read kernel or fail
+ *   "cluster"      CTAs per cluster of the fused kernel (1, 2, 4 or 8)
+ *   "stages"       depth of its shared-memory ring (2..8)
+ *   "max_clusters" cap on the number of resident clusters it launches
+ * Returns SGBV_ERR_SHAPE for an unknown name or a value out of range.
+ */
+int sgbv_set_option(const char *name, int value);
 
 /* Human-readable name of a return code. Never NULL. */
 const char *sgbv_status_string(int code);

@@ -19,12 +19,14 @@ OK = 0
 STATUS_TOKEN_RANGE = 1
 STATUS_NONFINITE_LOGIT = 2
 STATUS_DEGENERATE_RESIDUAL = 4
+STATUS_TIMEOUT = 8
 DTYPE_F32 = 0
 DTYPE_BF16 = 1
 
 EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_verify_ex",
-           "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_status_string", "sgbv_profile_begin",
-           "sgbv_profile_end", "sgbv_verify_static")
+           "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_last_main_kernel", "sgbv_status_string",
+           "sgbv_profile_begin",
+           "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option")
 
 _lib = None
 
@@ -65,10 +67,14 @@ def load() -> ctypes.CDLL:
         lib.sgbv_verify_host.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
         lib.sgbv_last_launch_count.restype = i32
         lib.sgbv_last_launch_count.argtypes = []
+        lib.sgbv_last_main_kernel.restype = ctypes.c_char_p
+        lib.sgbv_last_main_kernel.argtypes = []
         lib.sgbv_profile_begin.restype = i32
         lib.sgbv_profile_begin.argtypes = [i32]
         lib.sgbv_profile_end.restype = i32
         lib.sgbv_profile_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
+        lib.sgbv_set_option.restype = i32
+        lib.sgbv_set_option.argtypes = [ctypes.c_char_p, i32]
         lib.sgbv_status_string.restype = ctypes.c_char_p
         lib.sgbv_status_string.argtypes = [i32]
         _lib = lib
@@ -81,6 +87,17 @@ def status_string(code: int) -> str:
 
 def last_launch_count() -> int:
     return int(load().sgbv_last_launch_count())
+
+
+def set_option(name: str, value: int) -> None:
+    """Tuning knob for experiments (see include/sgbv.h); 0 restores the automatic choice."""
+    rc = load().sgbv_set_option(name.encode(), int(value))
+    if rc != OK:
+        raise SgbvError(rc)
+
+
+def last_main_kernel() -> str:
+    return load().sgbv_last_main_kernel().decode()
 
 
 def profile_begin(max_records: int) -> None:

@@ -2,6 +2,7 @@
 #include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include <mutex>
 
@@ -35,7 +36,7 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
 }
 
 struct Carve {
-    size_t rows, chain_end, part, wpart, dpart, mpart, h, resmass, status, total;
+    size_t rows, chain_end, part, wpart, dpart, mpart, h, resmass, status, error, total;
 };
 
 Carve carve(const Shape &s) {
@@ -51,6 +52,7 @@ Carve carve(const Shape &s) {
     c.h = off;         off += align_up(NR * sizeof(double));
     c.resmass = off;   off += align_up(NR * sizeof(double));
     c.status = off;    off += align_up((size_t)s.B * sizeof(int32_t));
+    c.error = off;     off += align_up(sizeof(int32_t));
     c.total = off;
     return c;
 }
@@ -90,6 +92,8 @@ int grow(void **ptr, size_t *have, size_t need) {
 }
 
 thread_local int t_last_launches = 0;
+thread_local const char *t_last_kernel = "none";
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -138,6 +142,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     L.ws.h = out_h ? out_h : (double *)(base + c.h);
     L.ws.resmass = out_resmass ? out_resmass : (double *)(base + c.resmass);
     L.ws.status = out_status ? out_status : (int32_t *)(base + c.status);
+    L.ws.error = (int32_t *)(base + c.error);
     L.zq = zq;
     L.zp = zp;
     L.dtype = dtype;
@@ -154,11 +159,15 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         ++g_prof.used;
     }
     if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
-    int n1 = launch_twopass(L);
+    if (cudaMemsetAsync(L.ws.error, 0, sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+    const bool fused = g_opt_path != 1 && fused_supported(L);
+    if (g_opt_path == 2 && !fused) return SGBV_ERR_SHAPE;
+    int n1 = fused ? launch_fused(L, L.ws.error) : launch_twopass(L);
     if (n1 < 0) return n1;
     int n2 = launch_finish(L);
     if (n2 < 0) return n2;
     t_last_launches = n1 + n2;
+    t_last_kernel = fused ? "fused_chain_kernel" : "otreduce_kernel";
     return SGBV_OK;
 }
 
@@ -255,6 +264,29 @@ int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dt
 }
 
 int sgbv_last_launch_count(void) { return t_last_launches; }
+
+const char *sgbv_last_main_kernel(void) { return t_last_kernel; }
+
+int sgbv_set_option(const char *name, int value) {
+    if (!name) return SGBV_ERR_NULL;
+    if (!strcmp(name, "path")) {
+        if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
+        g_opt_path = value;
+    } else if (!strcmp(name, "cluster")) {
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return SGBV_ERR_SHAPE;
+        g_opt_cluster = value;
+    } else if (!strcmp(name, "stages")) {
+        if (value != 0 && (value < 2 || value > 8)) return SGBV_ERR_SHAPE;
+        g_opt_stages = value;
+    } else if (!strcmp(name, "max_clusters")) {
+        if (value < 0) return SGBV_ERR_SHAPE;
+        g_opt_max_clusters = value;
+    } else {
+        return SGBV_ERR_SHAPE;
+    }
+    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters);
+    return SGBV_OK;
+}
 
 // ---- allocation-free variant ---------------------------------------------------------------------
 // Scratch for sgbv_verify_static: a fixed array inside the library's device image.  Every device

@@ -10,7 +10,7 @@
 
 namespace sgbv {
 
-constexpr int kTile = 1024;        // vocabulary elements per tile (granularity of the cached partial sums)
+constexpr int kTile = 256;         // vocabulary elements per tile (granularity of the cached partial sums)
 constexpr int kMaxK = 64;
 constexpr int kMaxGamma = 64;
 constexpr int kMaxV = 1 << 22;
@@ -39,6 +39,7 @@ struct Workspace {
     double *h;          // [B][K][gamma]
     double *resmass;    // [B][K][gamma]
     int32_t *status;    // [B]
+    int32_t *error;     // [1]: set when a bounded device-side wait expired
 };
 
 struct Shape {
@@ -129,5 +130,8 @@ struct Launch {
 
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
 int launch_finish(const Launch &L);   // weights, scan, extra token
+bool fused_supported(const Launch &L);
+int launch_fused(const Launch &L, int *error_flag);  // single-read cluster path for steps A1-A3
+void fused_set_options(int cluster, int stages, int max_clusters);
 
 }  // namespace sgbv

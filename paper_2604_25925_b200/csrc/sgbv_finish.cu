@@ -14,7 +14,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kMaxTiles = kMaxV / kTile;  // 4096
+constexpr int kEpt = kTile / kThreads;  // elements per thread inside one tile
+static_assert(kEpt >= 1 && kEpt * kThreads == kTile, "a tile is a whole number of elements per thread");
 
 __device__ __forceinline__ double gfun(double u, int K) {  // 1 - (1-u)^K
     if (u >= 1.0) return 1.0;
@@ -67,16 +68,16 @@ struct Pick {
     int last;   // largest index with positive weight, -1 if none
 };
 
-// Inverse CDF inside one tile: element x0 + 4*tid + j has weight wfun(x). base = cumulative
+// Inverse CDF inside one tile: element x0 + kEpt*tid + j has weight wfun(x). base = cumulative
 // weight before the tile. All threads must call.
 template <typename F>
 __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun, double *sh_warp, int *sh_pick) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    float w[4];
+    float w[kEpt];
     double local = 0.0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int x = x0 + 4 * tid + j;
+    for (int j = 0; j < kEpt; ++j) {
+        const int x = x0 + kEpt * tid + j;
         w[j] = (x < x1) ? wfun(x) : 0.0f;
         local += (double)w[j];
     }
@@ -96,9 +97,9 @@ __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun,
     for (int k = 0; k < wid; ++k) off += sh_warp[k];
     double cum = off + incl - local;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < kEpt; ++j) {
         cum += (double)w[j];
-        const int x = x0 + 4 * tid + j;
+        const int x = x0 + kEpt * tid + j;
         if (w[j] > 0.0f) {
             atomicMax(&sh_pick[1], x);
             if (cum > target) atomicMin(&sh_pick[0], x);
@@ -136,8 +137,6 @@ __device__ void locate_tile(const float *partials, int ntiles, double target, in
     sh_d[1] = target;
 }
 
-static_assert(kTile == 4 * kThreads, "pick_in_tile gives four consecutive elements to each thread");
-
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const int32_t *__restrict__ tok_all,
@@ -148,8 +147,8 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     double *h_s = reinterpret_cast<double *>(smem_raw);                       // [K*g]
     double *W_s = h_s + KG;                                                   // [K*g] sum of wpart
     unsigned long long *rej_s = reinterpret_cast<unsigned long long *>(W_s + KG);  // [K]
-    unsigned char *lcp_s = reinterpret_cast<unsigned char *>(rej_s + K);      // [K*K]
-    __shared__ float tile_s[kMaxTiles];
+    float *tile_s = reinterpret_cast<float *>(rej_s + K);                     // [ntiles]
+    unsigned char *lcp_s = reinterpret_cast<unsigned char *>(tile_s + s.ntiles);  // [K*K]
     __shared__ double sh_warp[kWarps];
     __shared__ float sh_redf[kWarps];
     __shared__ int sh_pick[2];
@@ -161,7 +160,8 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int32_t *tok = tok_all + (size_t)b * KG;
     const float *u = u_all + (size_t)b * (KG + 1);
     const int status_in = ws.status[b];
-    const bool invalid = (status_in & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT)) != 0;
+    const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
+    const bool invalid = lost || (status_in & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT)) != 0;
 
     // ---- 1. weights ---------------------------------------------------------------------------
     for (int n = wid; n < KG; n += kWarps) {
@@ -213,6 +213,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         if (tid == 0) {
             out_tau[b] = -1;
             out_f[b] = -1;
+            if (lost) ws.status[b] = status_in | SGBV_STATUS_TIMEOUT;
         }
         for (int j = tid; j <= g; j += kThreads) out_tokens[(size_t)b * (g + 1) + j] = -1;
         return;
@@ -345,7 +346,8 @@ template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
     const size_t KG = (size_t)s.K * s.gamma;
-    const size_t smem = 2 * KG * sizeof(double) + s.K * sizeof(unsigned long long) + (size_t)s.K * s.K;
+    const size_t smem = 2 * KG * sizeof(double) + s.K * sizeof(unsigned long long) + (size_t)s.ntiles * sizeof(float) +
+                        (size_t)s.K * s.K;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;

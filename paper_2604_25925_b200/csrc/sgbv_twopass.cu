@@ -132,15 +132,15 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
     chain_end[2 * bk + 1] = lb;
 }
 
+// One warp per 256-element tile: lanes stride the tile, one shuffle reduction per sum.
 template <typename T, bool kNeedAux>
 __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int t0,
-                                             int t1, float *wpart, float *dpart, float *mpart,
-                                             float (*red)[kThreads / 32]) {
+                                             int t1, float *wpart, float *dpart, float *mpart) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (int t = t0; t < t1; ++t) {
+    for (int t = t0 + wid; t < t1; t += kThreads / 32) {
         const int x0 = t * kTile, x1 = min(s.V, x0 + kTile);
         float sw = 0.0f, sd = 0.0f, sm = 0.0f;
-        for (int x = x0 + threadIdx.x; x < x1; x += kThreads) {
+        for (int x = x0 + lane; x < x1; x += 32) {
             float eq = expo(ld_logit(zq, x), ri.mq, s.scale);
             float ep = expo(ld_logit(zp, x), ri.mp, s.scale);
             float w, dp = 0.0f, m2 = 0.0f;
@@ -155,23 +155,10 @@ __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Sha
             sm = warp_sum(sm);
         }
         if (lane == 0) {
-            red[0][wid] = sw;
-            red[1][wid] = sd;
-            red[2][wid] = sm;
+            wpart[t] = sw;
+            dpart[t] = sd;
+            mpart[t] = sm;
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float a = 0.0f, b = 0.0f, c = 0.0f;
-            for (int w = 0; w < kThreads / 32; ++w) {
-                a += red[0][w];
-                b += red[1][w];
-                c += red[2][w];
-            }
-            wpart[t] = a;
-            dpart[t] = b;
-            mpart[t] = c;
-        }
-        __syncthreads();
     }
 }
 
@@ -186,14 +173,13 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
     const int bk = r / s.gamma;
     const T *zq = zq_all + ((size_t)bk * (s.gamma + 1) + i) * s.V;
     const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
-    __shared__ float red[3][kThreads / 32];
     const RowInfo ri = rows[r];
     const int t0 = sl * s.tiles_per_slice, t1 = min(s.ntiles, t0 + s.tiles_per_slice);
     float *wp = wpart + (size_t)r * s.ntiles, *dp = dpart + (size_t)r * s.ntiles, *mp = mpart + (size_t)r * s.ntiles;
     if (ri.c < 1.0f)
-        reduce_tiles<T, true>(zq, zp, s, ri, t0, t1, wp, dp, mp, red);
+        reduce_tiles<T, true>(zq, zp, s, ri, t0, t1, wp, dp, mp);
     else
-        reduce_tiles<T, false>(zq, zp, s, ri, t0, t1, wp, dp, mp, red);
+        reduce_tiles<T, false>(zq, zp, s, ri, t0, t1, wp, dp, mp);
 }
 
 template <typename T>

@@ -146,6 +146,27 @@ def test_edge_shapes(B, K, gamma, V, dtype):
     assert_parity(rep)
 
 
+@pytest.mark.parametrize("option", [("path", 1), ("cluster", 1), ("cluster", 2), ("cluster", 4), ("cluster", 8),
+                                    ("stages", 2), ("max_clusters", 3)])
+def test_every_kernel_path_and_launch_shape_matches(option):
+    """The generic two-sweep kernels and the fused kernel at every cluster size / ring depth /
+    persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
+    cfgs = [workloads.VerifyConfig("paths_a", B=5, K=3, gamma=3, V=20480, temperature=0.8, alpha=0.8, seed=21),
+            workloads.VerifyConfig("paths_b", B=3, K=2, gamma=2, V=33000, dtype="bf16", temperature=1.1, alpha=0.7,
+                                   seed=22),
+            workloads.VerifyConfig("paths_c", B=2, K=2, gamma=5, V=1000, alpha=0.9, seed=23)]
+    binding.set_option(*option)
+    try:
+        for cfg in cfgs:
+            if option == ("cluster", 1) and cfg.V > 20480:
+                continue   # a single CTA cannot hold more than five chunks of a row
+            inp = workloads.make_inputs(cfg, device="cuda")
+            rep, _, _ = run_both(inp)
+            assert_parity(rep)
+    finally:
+        binding.set_option(option[0], 0)
+
+
 def test_unaligned_views_and_repeated_calls_are_deterministic():
     cfg = workloads.VerifyConfig("unaligned", B=3, K=2, gamma=3, V=4099, alpha=0.8, seed=99)
     inp = workloads.make_inputs(cfg, device="cuda")
