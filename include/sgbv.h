@@ -157,8 +157,8 @@ int sgbv_profile_end(double *out_total_ms, int *out_records);
 /*
  * Tuning knobs for experiments (process-wide, not thread-safe; 0 restores the automatic choice):
  *   "path"         1 = always the generic two-sweep kernels, 2 = the fused single-read kernel or fail
- *   "cluster"      CTAs per cluster of the fused kernel (1, 2, 4 or 8)
- *   "stages"       depth of its shared-memory ring (2..8)
+ *   "cluster"      CTAs per cluster of the fused kernel (1, 2, 4, 8 or 16)
+ *   "stages"       depth of its shared-memory ring (2..12)
  *   "max_clusters" cap on the number of resident clusters it launches
  * Returns SGBV_ERR_SHAPE for an unknown name or a value out of range.
  */

@@ -36,7 +36,7 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
 }
 
 struct Carve {
-    size_t rows, chain_end, part, wpart, dpart, mpart, h, resmass, status, error, total;
+    size_t rows, part, wpart, dpart, mpart, h, resmass, status, error, total;
 };
 
 Carve carve(const Shape &s) {
@@ -44,7 +44,6 @@ Carve carve(const Shape &s) {
     Carve c;
     size_t off = 0;
     c.rows = off;      off += align_up(NR * sizeof(RowInfo));
-    c.chain_end = off; off += align_up((size_t)s.B * s.K * 2 * sizeof(double));
     c.part = off;      off += align_up(NR * s.nsplit * 4 * sizeof(float));
     c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
@@ -134,7 +133,6 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         base = (unsigned char *)g_buf[dev].scratch;
     }
     L.ws.rows = (RowInfo *)(base + c.rows);
-    L.ws.chain_end = (double *)(base + c.chain_end);
     L.ws.part = (float *)(base + c.part);
     L.ws.wpart = (float *)(base + c.wpart);
     L.ws.dpart = (float *)(base + c.dpart);
@@ -160,10 +158,15 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     }
     if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
     if (cudaMemsetAsync(L.ws.error, 0, sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
-    const bool fused = g_opt_path != 1 && fused_supported(L);
-    if (g_opt_path == 2 && !fused) return SGBV_ERR_SHAPE;
-    int n1 = fused ? launch_fused(L, L.ws.error) : launch_twopass(L);
+    bool fused = g_opt_path != 1 && fused_supported(L);
+    int n1 = fused ? launch_fused(L, L.ws.error) : 0;
     if (n1 < 0) return n1;
+    if (n1 == 0) {
+        if (g_opt_path == 2) return SGBV_ERR_SHAPE;
+        fused = false;
+        n1 = launch_twopass(L);
+        if (n1 < 0) return n1;
+    }
     int n2 = launch_finish(L);
     if (n2 < 0) return n2;
     t_last_launches = n1 + n2;
@@ -273,10 +276,11 @@ int sgbv_set_option(const char *name, int value) {
         if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
         g_opt_path = value;
     } else if (!strcmp(name, "cluster")) {
-        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8) return SGBV_ERR_SHAPE;
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16)
+            return SGBV_ERR_SHAPE;
         g_opt_cluster = value;
     } else if (!strcmp(name, "stages")) {
-        if (value != 0 && (value < 2 || value > 8)) return SGBV_ERR_SHAPE;
+        if (value != 0 && (value < 2 || value > 12)) return SGBV_ERR_SHAPE;
         g_opt_stages = value;
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;

@@ -19,19 +19,17 @@ constexpr float kLog2e = 1.4426950408889634f;
 // Per (b,k,i) row pair, i < gamma.  Written by the statistics pass, read by the reduction pass
 // and by the finishing kernel.
 struct RowInfo {
-    double log_a;   // log q(x_k^i): joint target probability of the i-token prefix
-    double log_b;   // log p(x_k^i)
     double Zq;      // sum_x exp((zq_x - mq)/T)
     double Zp;
     float mq;       // row maxima of the raw logits
     float mp;
     float kappa;    // c * Zq / Zp with c = b/a: ratio c*p(x)/q(x) = kappa * ep/eq in row-max units
-    float c;        // c = exp(log_b - log_a), for the c < 1 branch of the numerator
+    float c;        // c = p(x_k^i)/q(x_k^i), ratio of the joint prefix probabilities (c < 1 selects
+                    // the cancellation-free numerator)
 };
 
 struct Workspace {
     RowInfo *rows;      // [B*K*gamma]
-    double *chain_end;  // [B*K][2]: log a_gamma, log b_gamma
     float *part;        // [B*K*gamma][nsplit][4]: slice partials (mq, Zq, mp, Zp)   (two-pass path)
     float *wpart;       // [B*K*gamma][ntiles]: sum over the tile of eq * max(1 - kappa ep/eq, 0)^K
     float *dpart;       // [B*K*gamma][ntiles]: sum of max(kappa ep - eq, 0)               (c < 1)
@@ -131,7 +129,9 @@ struct Launch {
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
 int launch_finish(const Launch &L);   // weights, scan, extra token
 bool fused_supported(const Launch &L);
-int launch_fused(const Launch &L, int *error_flag);  // single-read cluster path for steps A1-A3
+// single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
+// anything (the caller then takes the two-sweep path), or < 0
+int launch_fused(const Launch &L, int *error_flag);
 void fused_set_options(int cluster, int stages, int max_clusters);
 
 }  // namespace sgbv

@@ -1,4 +1,6 @@
 // Finishing kernel: one CTA per batch row.
+//   0. log a_i = log q(x_k^i), log b_i = log p(x_k^i) of every draft by running sums of the token
+//      log-probabilities (row maxima and normalisers come from the streaming pass);
 //   1. combine the cached per-tile sums of every (k,i) row into S_i and the acceptance weights
 //      (Eq. 2 for proper sub-blocks, Eq. 3 for the whole block), in float64;
 //   2. the scan of Algorithm 1 over drafts and positions with the pre-drawn uniforms;
@@ -146,7 +148,9 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int K = s.K, g = s.gamma, KG = K * g;
     double *h_s = reinterpret_cast<double *>(smem_raw);                       // [K*g]
     double *W_s = h_s + KG;                                                   // [K*g] sum of wpart
-    unsigned long long *rej_s = reinterpret_cast<unsigned long long *>(W_s + KG);  // [K]
+    double *la_s = W_s + KG;                                                  // [K*(g+1)] log q(x_k^i)
+    double *lb_s = la_s + K * (g + 1);                                        // [K*(g+1)] log p(x_k^i)
+    unsigned long long *rej_s = reinterpret_cast<unsigned long long *>(lb_s + K * (g + 1));  // [K]
     float *tile_s = reinterpret_cast<float *>(rej_s + K);                     // [ntiles]
     unsigned char *lcp_s = reinterpret_cast<unsigned char *>(tile_s + s.ntiles);  // [K*K]
     __shared__ double sh_warp[kWarps];
@@ -162,6 +166,26 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int status_in = ws.status[b];
     const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
     const bool invalid = lost || (status_in & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT)) != 0;
+
+    // ---- 0. joint prefix probabilities (logs), one thread per draft -----------------------------
+    for (int k = tid; k < K; k += kThreads) {
+        double la = 0.0, lb = 0.0;
+        for (int i = 0; i < g; ++i) {
+            la_s[k * (g + 1) + i] = la;
+            lb_s[k * (g + 1) + i] = lb;
+            const size_t r = ((size_t)b * K + k) * g + i;
+            const RowInfo ri = ws.rows[r];
+            int t = tok[k * g + i];
+            if (t < 0 || t >= s.V) t = 0;  // the row is flagged and produces no output
+            const float zqt = ld_logit(zq_all, (((size_t)b * K + k) * (g + 1) + i) * s.V + t);
+            const float zpt = ld_logit(zp_all, r * s.V + t);
+            la += ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
+            lb += ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
+        }
+        la_s[k * (g + 1) + g] = la;
+        lb_s[k * (g + 1) + g] = lb;
+    }
+    __syncthreads();
 
     // ---- 1. weights ---------------------------------------------------------------------------
     for (int n = wid; n < KG; n += kWarps) {
@@ -184,18 +208,18 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         if (lane == 0) {
             const double R = sw / ri.Zq;
             W_s[n] = sw;
-            const double S = exp(ri.log_a) * R;
+            const double la = la_s[k * (g + 1) + i], lb = lb_s[k * (g + 1) + i];
+            const double S = exp(la) * R;
             ws.resmass[(size_t)b * KG + n] = invalid ? NAN : S;
             if (i >= 1) {
-                const double hv = weight_sub(ri.log_a, ri.log_b, R, sd / ri.Zq, sm / ri.Zq, K, aux);
+                const double hv = weight_sub(la, lb, R, sd / ri.Zq, sm / ri.Zq, K, aux);
                 h_s[k * g + i - 1] = hv;
                 ws.h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
             }
         }
     }
     for (int k = tid; k < K; k += kThreads) {
-        const double *ce = ws.chain_end + 2 * ((size_t)b * K + k);
-        const double hv = weight_full(ce[0], ce[1], K);
+        const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
         h_s[k * g + g - 1] = hv;
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
         rej_s[k] = 0ull;
@@ -346,8 +370,8 @@ template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
     const size_t KG = (size_t)s.K * s.gamma;
-    const size_t smem = 2 * KG * sizeof(double) + s.K * sizeof(unsigned long long) + (size_t)s.ntiles * sizeof(float) +
-                        (size_t)s.K * s.K;
+    const size_t smem = 2 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
+                        s.K * sizeof(unsigned long long) + (size_t)s.ntiles * sizeof(float) + (size_t)s.K * s.K;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;

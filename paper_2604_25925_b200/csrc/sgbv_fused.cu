@@ -2,17 +2,22 @@
 //
 // For every position i = 0..gamma-1 of the chain the cluster
 //   * streams the target row and the draft row from HBM exactly once: one elected thread issues
-//     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts) of 4096-element chunks
+//     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks
 //     into a shared-memory ring that runs ahead across rows and chains;
 //   * keeps the whole row pair resident in REGISTERS (each CTA of the cluster owns a contiguous
-//     slice of the vocabulary, each thread 8 elements of every chunk), so the second sweep of the
-//     coupling sum never re-reads memory;
-//   * reduces max and sum-exp per CTA (warp shuffles + shared memory), exchanges the CTA partials
-//     through distributed shared memory with one cluster barrier per row, derives the chain
-//     scalars (log a_i, log b_i, c_i, kappa_i) redundantly and identically in every CTA;
+//     slice of the vocabulary, each thread 8 elements of every chunk) as exponentials relative to
+//     the thread's own maximum, so the second sweep of the coupling sum never re-reads memory;
+//   * exchanges per-warp (max, sum-exp) partials by PUSHING them into every CTA's shared memory
+//     (distributed shared memory stores) followed by one cluster barrier per row; after the barrier
+//     every warp combines the partials locally and identically, so there is no second block-wide
+//     synchronisation and no remote load on the critical path;
 //   * runs the second sweep from registers and writes one partial sum per 256-element cell
 //     (a cell is what one warp owns in one chunk: 256 contiguous vocabulary entries).
-// The finishing kernel (weights, scan, extra token) consumes the cell sums.
+// The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread,
+// which computes c_{i+1} while the other warps are already in the second sweep of row i.
+// Two CTAs of 256 threads share an SM (different clusters), so one CTA's exchange latency is
+// covered by the other's arithmetic.  The finishing kernel (weights, scan, extra token) consumes
+// the cell sums.
 //
 // Every wait on an mbarrier is bounded; on expiry the CTA records an error flag and keeps
 // executing the protocol (all cluster barriers are still reached), so a lost copy cannot hang.
@@ -22,12 +27,14 @@ namespace sgbv {
 
 namespace {
 
-constexpr int kFThreads = 512;
+constexpr int kFThreads = 256;
 constexpr int kFWarps = kFThreads / 32;
 constexpr int kCell = kTile;               // 256 contiguous elements: one warp's share of a chunk
-constexpr int kChunk = kFWarps * kCell;    // 4096 elements per chunk per tensor
-constexpr int kLag = 1;                    // the producer refills the stage consumed kLag chunks ago
-constexpr int kSpinLimit = 1 << 22;
+constexpr int kChunk = kFWarps * kCell;    // 2048 elements per chunk per tensor
+constexpr int kMaxNch = 5;                 // chunks of a row slice one CTA can hold in registers
+constexpr int kMaxStages = 12;
+constexpr int kMaxCluster = 16;
+constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
 
 struct FusedParams {
@@ -59,20 +66,20 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait: returns false if the phase did not complete within the spin limit.
+// Bounded wait: returns false if the phase did not complete within about a second.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (int it = 0; it < kSpinLimit; ++it) {
-        if (mbar_test(bar, parity)) return true;
-        if (it > 128) __nanosleep(40);
-    }
-    return false;
+    if (mbar_test(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_test(bar, parity))
+        if (clock64() - t0 > kWaitLimitCycles) return false;
+    return true;
 }
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -85,32 +92,40 @@ __device__ __forceinline__ uint32_t cluster_ctarank() {
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
-__device__ __forceinline__ float4 ld_dsmem_f4(const void *local, uint32_t rank) {
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Store 16 bytes into the shared memory of CTA `rank` of this cluster, at the address that
+// `local` has in this CTA.
+__device__ __forceinline__ void st_dsmem_f4(void *local, uint32_t rank, float4 v) {
     uint32_t remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(remote)
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z),
+                 "f"(v.w)
                  : "memory");
-    return v;
 }
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float rcp(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 // ---- shared memory layout ------------------------------------------------------------------------
 struct Control {
-    uint64_t full[8];
-    uint64_t empty[8];
-    float4 slot[2];        // this CTA's (mq, Zq, mp, Zp), double-buffered by row parity
-    float red[4][kFWarps];
-    float bc[8];           // fq, kp, c, aux, eq-reference, ep-reference
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    // per-warp partials (mq, sum eq, mp, sum ep) of every CTA of the cluster, pushed by their
+    // owners; double-buffered by row parity
+    float4 slots[2][kMaxCluster * kFWarps];
+    double c[2];           // joint likelihood ratio c_i of the current chain, by row parity
     int32_t tok[kMaxGamma];
 };
 
@@ -139,31 +154,52 @@ __device__ __forceinline__ int cell_offset(int lane, int e) {
     return lane * 8 + e;
 }
 
-// Second sweep over the register-resident row: cell sums of the residual weight and, for c < 1, of
-// the two non-negative numerator terms.  eq/ep are in CTA-max units; fq rescales eq to row-max
-// units and kp = kappa * fp does the same for the draft side.
+// r^K for r in [0,1]; KT > 0 is a compile-time K.
+template <int KT>
+__device__ __forceinline__ float ipow(float r, int K) {
+    if (KT == 1) return 1.0f;  // callers multiply by the base themselves where K = 1 matters
+    if (KT > 1) {
+        float acc = (KT & 1) ? r : 1.0f, sq = r;
+#pragma unroll
+        for (int k = KT >> 1; k > 0; k >>= 1) {
+            sq *= sq;
+            if (k & 1) acc *= sq;
+        }
+        return acc;
+    }
+    float acc = 1.0f;
+    for (int t = 0; t < K; ++t) acc *= r;
+    return acc;
+}
+
+// Second sweep over the register-resident row.  eq/ep are exponentials relative to the THREAD's
+// maxima; kt = kappa * (fp_t / fq_t) makes  c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d convert the
+// thread's sums to row-max units.  Per cell:
+//   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
+//   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
+//   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
 template <int NCH, int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float fq, float kp,
-                                          float c, int K, int lane, int first_cell, int ncells_valid, int warp,
-                                          float *wpart, float *dpart, float *mpart) {
+__device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
+                                          float scale_w, float scale_d, float c, int K, int lane, int warp,
+                                          int ncells_valid, float *wpart, float *dpart, float *mpart) {
     const float v1 = 1.0f - c;
 #pragma unroll
     for (int j = 0; j < NCH; ++j) {
+        const int cell = j * kFWarps + warp;  // cell index inside this CTA's slice (warp-uniform)
+        if (cell >= ncells_valid) break;
         float sw = 0.0f, sd = 0.0f, sm = 0.0f;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const float q = fq * eq[j][e];
-            const float diff = fmaf(-kp, ep[j][e], q);
-            const float d = fmaxf(diff, 0.0f);
-            const float r = (d > 0.0f) ? __fdividef(d, q) : 0.0f;
-            float pw = d;
-            if (KT > 0) {
-#pragma unroll
-                for (int t = 1; t < KT; ++t) pw *= r;
-            } else {
-                for (int t = 1; t < K; ++t) pw *= r;
+            const float q = eq[j][e];
+            const float diff = fmaf(-kt, ep[j][e], q);      // q - c p, thread units
+            if (KT == 1 && !kAux) {
+                sw += fmaxf(diff, 0.0f);
+                continue;
             }
-            sw += pw;
+            // r = 1 - min{c p/q, 1}; q = 0 gives -inf or NaN before the clamp, 0 after it
+            const float r = fmaxf(diff * rcp(q), 0.0f);
+            if (KT == 1) sw += fmaxf(diff, 0.0f);
+            else sw = fmaf(q, ipow<KT>(r, K), sw);
             if (kAux) {
                 sd += fmaxf(-diff, 0.0f);
                 float acc = 0.0f;
@@ -185,43 +221,44 @@ __device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float
                         acc = fmaf(acc, r, (float)(t + 1) * vj);
                     }
                 }
-                const float ct = c - 1.0f + r;
+                const float ct = r - v1;  // c - t with t = 1 - r
                 sm = fmaf(q * ct * ct, acc, sm);
             }
         }
-        sw = warp_sum(sw);
+        sw = warp_sum(sw * scale_w);
         if (kAux) {
-            sd = warp_sum(sd);
-            sm = warp_sum(sm);
+            sd = warp_sum(sd * scale_d);
+            sm = warp_sum(sm * scale_w);
         }
-        const int cell = j * kFWarps + warp;  // cell index inside this CTA's slice
-        if (lane == 0 && cell < ncells_valid) {
-            wpart[first_cell + cell] = sw;
+        if (lane == 0) {
+            wpart[cell] = sw;
             if (kAux) {
-                dpart[first_cell + cell] = sd;
-                mpart[first_cell + cell] = sm;
+                dpart[cell] = sd;
+                mpart[cell] = sm;
             }
         }
     }
 }
 
 template <int NCH, bool kAux>
-__device__ __forceinline__ void sweep_two_dispatch(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float fq,
-                                                   float kp, float c, int K, int lane, int first_cell,
-                                                   int ncells_valid, int warp, float *wpart, float *dpart,
-                                                   float *mpart) {
+__device__ __forceinline__ void sweep_two_dispatch(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
+                                                   float scale_w, float scale_d, float c, int K, int lane, int warp,
+                                                   int ncells_valid, float *wpart, float *dpart, float *mpart) {
+#define SGBV_SWEEP(KT) \
+    sweep_two<NCH, KT, kAux>(eq, ep, kt, scale_w, scale_d, c, K, lane, warp, ncells_valid, wpart, dpart, mpart)
     switch (K) {
-        case 1: sweep_two<NCH, 1, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
-        case 2: sweep_two<NCH, 2, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
-        case 3: sweep_two<NCH, 3, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
-        case 4: sweep_two<NCH, 4, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
-        case 8: sweep_two<NCH, 8, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
-        default: sweep_two<NCH, 0, kAux>(eq, ep, fq, kp, c, K, lane, first_cell, ncells_valid, warp, wpart, dpart, mpart); break;
+        case 1: SGBV_SWEEP(1); break;
+        case 2: SGBV_SWEEP(2); break;
+        case 3: SGBV_SWEEP(3); break;
+        case 4: SGBV_SWEEP(4); break;
+        case 8: SGBV_SWEEP(8); break;
+        default: SGBV_SWEEP(0); break;
     }
+#undef SGBV_SWEEP
 }
 
 template <typename T, int NCH>
-__global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedParams p) {
+__global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -247,7 +284,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    cluster_sync_all();  // every CTA of the cluster is running before any remote shared-memory access
+    cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
+    cluster_wait();
 
     const int my_chains = (p.nchains - cid + G - 1) / G;
     const int loads_per_chain = s.gamma * NCH;
@@ -299,27 +337,26 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
             }
             ctl->tok[tid] = t;
         }
+        if (tid == 0) ctl->c[rowcount & 1] = 1.0;  // c_0 = 1 (empty prefix)
         __syncthreads();
-        double la = 0.0, lb = 0.0;  // log a_i, log b_i (meaningful in warp 0)
 
         for (int i = 0; i < s.gamma; ++i) {
             const size_t r = bk * s.gamma + i;
-            const T *zq_row = reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V;
-            const T *zp_row = reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V;
-            // token logits for the chain scalars: fetched now, used after the first sweep
+            const int par = rowcount & 1;
+            // token logits for the chain ratio: fetched now, used after the exchange
             float zq_tok = 0.0f, zp_tok = 0.0f;
-            if (warp == 0 && lane == 0) {
+            if (tid == 0) {
                 const int t = ctl->tok[i];
-                zq_tok = ld_logit(zq_row, t);
-                zp_tok = ld_logit(zp_row, t);
+                zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
+                zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
             }
 
-            // ---- first sweep, part 1: ring -> registers, running max -------------------------------
+            // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
             float eq[NCH][8], ep[NCH][8];
             float mq = -INFINITY, mp = -INFINITY;
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
-                if (tid == 0 && consumed >= kLag && p_issued < total_loads) {
+                if (tid == 0 && consumed >= 1 && p_issued < total_loads) {
                     // refill the stage of the previous chunk once every warp has released it
                     if (!mbar_wait(&ctl->empty[prev_st], prev_ph)) timed_out = true;
                     issue_next();
@@ -355,23 +392,10 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
                 }
                 ++consumed;
             }
-            mq = warp_max(mq);
-            mp = warp_max(mp);
-            if (lane == 0) {
-                ctl->red[0][warp] = mq;
-                ctl->red[1][warp] = mp;
-            }
-            __syncthreads();
-            mq = ctl->red[0][0];
-            mp = ctl->red[1][0];
-#pragma unroll
-            for (int w = 1; w < kFWarps; ++w) {
-                mq = fmaxf(mq, ctl->red[0][w]);
-                mp = fmaxf(mp, ctl->red[1][w]);
-            }
-            // reference points for the exponentials: the CTA maxima (0 if the slice is all -inf)
-            const float rq = (mq > -INFINITY) ? mq : 0.0f;
-            const float rp = (mp > -INFINITY) ? mp : 0.0f;
+            // reference points of the exponentials: the thread's own maxima (0 if it saw only -inf)
+            const bool has_q = mq > -INFINITY, has_p = mp > -INFINITY;
+            const float rq = has_q ? mq : 0.0f;
+            const float rp = has_p ? mp : 0.0f;
 
             // ---- first sweep, part 2: exponentials in place, sums ----------------------------------
             float sq = 0.0f, sp = 0.0f;
@@ -385,83 +409,93 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
                     sp += ep[j][e];
                 }
             }
-            sq = warp_sum(sq);
-            sp = warp_sum(sp);
-            if (lane == 0) {
-                ctl->red[2][warp] = sq;
-                ctl->red[3][warp] = sp;
-            }
-            __syncthreads();
-            if (tid == 0) {
-                float a = 0.0f, b = 0.0f;
-#pragma unroll
-                for (int w = 0; w < kFWarps; ++w) {
-                    a += ctl->red[2][w];
-                    b += ctl->red[3][w];
-                }
-                ctl->slot[rowcount & 1] = make_float4(mq, a, mp, b);
-            }
-            cluster_sync_all();
+            // warp partials in warp-max units, pushed to every CTA of the cluster
+            const float mqw = warp_max(mq), mpw = warp_max(mp);
+            const float rqw = (mqw > -INFINITY) ? mqw : 0.0f, rpw = (mpw > -INFINITY) ? mpw : 0.0f;
+            sq = warp_sum(has_q ? sq * ex2((rq - rqw) * s.scale) : 0.0f);
+            sp = warp_sum(has_p ? sp * ex2((rp - rpw) * s.scale) : 0.0f);
+            if (lane < C) st_dsmem_f4(&ctl->slots[par][rank * kFWarps + warp], (uint32_t)lane, make_float4(mqw, sq, mpw, sp));
+            cluster_arrive();
+            cluster_wait();
 
-            // ---- chain scalars (warp 0 of every CTA, identical arithmetic) ---------------------------
-            if (warp == 0) {
-                float4 v = make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-                if (lane < C) v = ld_dsmem_f4(&ctl->slot[rowcount & 1], (uint32_t)lane);
-                const float mq_row = warp_max(v.x), mp_row = warp_max(v.z);
-                double zq_part = 0.0, zp_part = 0.0;
-                if (lane < C) {
-                    if (v.x > -INFINITY) zq_part = (double)v.y * exp2((double)(v.x - mq_row) * (double)s.scale);
-                    if (v.z > -INFINITY) zp_part = (double)v.w * exp2((double)(v.z - mp_row) * (double)s.scale);
+            // ---- row statistics: every warp combines all partials, in the same order ------------------
+            float mq_row = -INFINITY, mp_row = -INFINITY;
+            const int nslots = C * kFWarps;
+            for (int e = lane; e < nslots; e += 32) {
+                const float4 v = ctl->slots[par][e];
+                mq_row = fmaxf(mq_row, v.x);
+                mp_row = fmaxf(mp_row, v.z);
+            }
+            mq_row = warp_max(mq_row);
+            mp_row = warp_max(mp_row);
+            const float rq_row = (mq_row > -INFINITY) ? mq_row : 0.0f, rp_row = (mp_row > -INFINITY) ? mp_row : 0.0f;
+            double Zq = 0.0, Zp = 0.0;
+            for (int e = lane; e < nslots; e += 32) {
+                const float4 v = ctl->slots[par][e];
+                if (v.x > -INFINITY) Zq += (double)(v.y * ex2((v.x - rq_row) * s.scale));
+                if (v.z > -INFINITY) Zp += (double)(v.w * ex2((v.z - rp_row) * s.scale));
+            }
+            Zq = warp_sum(Zq);
+            Zp = warp_sum(Zp);
+            const double cd = ctl->c[par];
+            const double kappa_d = cd * Zq / Zp;
+            const float c = (float)cd;
+
+            if (tid == 0) {
+                // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
+                // -inf only has Z = 0
+                const bool bad = !(Zq > 0.0) || !(Zp > 0.0) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
+                                 !(mq_row < INFINITY) || !(mp_row < INFINITY);
+                if (rank == 0) {
+                    if (bad) atomicOr(p.ws.status + brow, SGBV_STATUS_NONFINITE_LOGIT);
+                    RowInfo ri;
+                    ri.Zq = Zq;
+                    ri.Zp = Zp;
+                    ri.mq = mq_row;
+                    ri.mp = mp_row;
+                    ri.kappa = (float)kappa_d;
+                    ri.c = c;
+                    p.ws.rows[r] = ri;
                 }
-                const double Zq = warp_sum(zq_part), Zp = warp_sum(zp_part);
-                if (lane == 0) {
-                    const double c = exp(lb - la);
-                    const double kappa = c * Zq / Zp;
-                    // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
-                    // -inf only has Z = 0
-                    const bool bad = !(Zq > 0.0) || !(Zp > 0.0) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
-                                     !(mq_row < INFINITY) || !(mp_row < INFINITY);
-                    if (rank == 0) {
-                        if (bad) atomicOr(p.ws.status + brow, SGBV_STATUS_NONFINITE_LOGIT);
-                        RowInfo ri;
-                        ri.log_a = la;
-                        ri.log_b = lb;
-                        ri.Zq = Zq;
-                        ri.Zp = Zp;
-                        ri.mq = mq_row;
-                        ri.mp = mp_row;
-                        ri.kappa = (float)kappa;
-                        ri.c = (float)c;
-                        p.ws.rows[r] = ri;
-                    }
-                    const float fq = ex2((rq - mq_row) * s.scale);   // CTA units -> row units
-                    const float fp = ex2((rp - mp_row) * s.scale);
-                    ctl->bc[0] = fq;
-                    ctl->bc[1] = (float)kappa * fp;
-                    ctl->bc[2] = (float)c;
-                    la += ((double)zq_tok - (double)mq_row) * s.inv_T - log(Zq);
-                    lb += ((double)zp_tok - (double)mp_row) * s.inv_T - log(Zp);
-                    if (i == s.gamma - 1 && rank == 0) {
-                        p.ws.chain_end[2 * bk + 0] = la;
-                        p.ws.chain_end[2 * bk + 1] = lb;
-                    }
+                // c_{i+1} = c_i p_i(tok_i)/q_i(tok_i), for the next row of this chain
+                const double lp = ((double)zp_tok - (double)mp_row) * s.inv_T;
+                const double lq = ((double)zq_tok - (double)mq_row) * s.inv_T;
+                ctl->c[par ^ 1] = cd * exp(lp - lq) * (Zq / Zp);
+            }
+
+            // thread units -> row units
+            const float fq = has_q ? ex2((rq - rq_row) * s.scale) : 0.0f;
+            const float fp = has_p ? ex2((rp - rp_row) * s.scale) : 0.0f;
+            float kt = (float)kappa_d * fp / fq;
+            float scale_w = fq, scale_d = fq;
+            if (__any_sync(0xffffffffu, !(fq > 1e-30f))) {
+                // a thread whose share of the target row underflows (or nearly so, which would
+                // overflow kt): its q is 0 in row units, its weights vanish, and max(c p - q, 0) = c p
+                if (!(fq > 1e-30f)) {
+#pragma unroll
+                    for (int j = 0; j < NCH; ++j)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) eq[j][e] = 0.0f;
+                    kt = 1.0f;
+                    scale_w = 0.0f;
+                    scale_d = (float)kappa_d * fp;
                 }
             }
-            __syncthreads();
-            const float fq = ctl->bc[0], kp = ctl->bc[1], c = ctl->bc[2];
 
             // ---- second sweep from registers ---------------------------------------------------------
-            float *wp = p.ws.wpart + r * s.ntiles, *dp = p.ws.dpart + r * s.ntiles, *mpp = p.ws.mpart + r * s.ntiles;
+            float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
+                  *mpp = p.ws.mpart + r * s.ntiles + first_cell;
             if (c < 1.0f)
-                sweep_two_dispatch<NCH, true>(eq, ep, fq, kp, c, s.K, lane, first_cell, ncells_valid, warp, wp, dp, mpp);
+                sweep_two_dispatch<NCH, true>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, warp, ncells_valid, wp, dp, mpp);
             else
-                sweep_two_dispatch<NCH, false>(eq, ep, fq, kp, c, s.K, lane, first_cell, ncells_valid, warp, wp, dp, mpp);
+                sweep_two_dispatch<NCH, false>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, warp, ncells_valid, wp, dp, mpp);
             ++rowcount;
         }
-        __syncthreads();  // ctl->tok is rewritten for the next chain
+        __syncthreads();  // ctl->tok and ctl->c are rewritten for the next chain
     }
     if (timed_out) atomicExch(p.error_flag, 1);
-    cluster_sync_all();  // no CTA leaves while a neighbour may still read its slots
+    cluster_arrive();  // no CTA leaves while a neighbour may still write into its slots
+    cluster_wait();
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -474,6 +508,13 @@ int g_opt_cluster = 0;     // 0 = automatic
 int g_opt_stages = 0;
 int g_opt_max_clusters = 0;
 
+constexpr int kSmemPerSm = 228 * 1024;     // shared memory of one SM
+constexpr int kSmemReserved = 1024;        // per resident CTA, taken by the system
+constexpr int kCtaSlots = 2 * 148;         // resident CTAs of this kernel on the whole device
+
+int cells_of(int V) { return (V + kCell - 1) / kCell; }
+int slice_cells(int cells, int C) { return (cells + C - 1) / C; }
+
 template <typename T, int NCH>
 int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     auto kernel = fused_chain_kernel<T, NCH>;
@@ -481,7 +522,10 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGBV_ERR_CUDA;
     if (!attr_done[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemPerSm / 2 - kSmemReserved) != cudaSuccess)
+            return SGBV_ERR_CUDA;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
             return SGBV_ERR_CUDA;
         attr_done[dev] = true;
     }
@@ -512,14 +556,14 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     int clusters = plan.grid_clusters;
     if (clusters <= 0) {
         // persistent grid: as many clusters as can be co-resident (queried once per configuration)
-        static int cached[9][9];  // [cluster size][stages]
-        int &slot = cached[plan.cluster][plan.stages];
+        static int cached[64][kMaxCluster + 1][kMaxStages + 1];  // [device][cluster size][stages]
+        int &slot = cached[dev][plan.cluster][plan.stages];
         if (slot == 0) {
-            cfg.gridDim = dim3(plan.cluster * 148);
+            cfg.gridDim = dim3(plan.cluster * (kCtaSlots / plan.cluster));
             int nmax = 0;
             if (cudaOccupancyMaxActiveClusters(&nmax, kernel, &cfg) != cudaSuccess || nmax < 1) {
                 cudaGetLastError();
-                nmax = 148 / plan.cluster;
+                return 0;  // this cluster shape cannot be scheduled here: nothing launched
             }
             slot = nmax;
         }
@@ -530,7 +574,11 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, fp);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
-    return e == cudaSuccess ? 1 : SGBV_ERR_CUDA;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return SGBV_ERR_CUDA;
+    }
+    return 1;
 }
 
 template <typename T>
@@ -554,35 +602,35 @@ void fused_set_options(int cluster, int stages, int max_clusters) {
 }
 
 // Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and
-// a CTA's slice must fit its registers (at most 5 chunks of 4096 elements, clusters of at most 8).
+// a CTA's slice must fit its registers (at most 5 chunks of 2048 elements, clusters of at most 16).
 bool fused_supported(const Launch &L) {
     const size_t esz = L.dtype == SGBV_DTYPE_BF16 ? 2 : 4;
     if (((uintptr_t)L.zq % 16) || ((uintptr_t)L.zp % 16) || (((size_t)L.s.V * esz) % 16)) return false;
-    const int cells = (L.s.V + kCell - 1) / kCell;
-    return (cells + 7) / 8 * kCell <= 5 * kChunk;
+    return slice_cells(cells_of(L.s.V), kMaxCluster) * kCell <= kMaxNch * kChunk;
 }
 
 int launch_fused(const Launch &L, int *error_flag) {
     const Shape &s = L.s;
     const size_t esz = L.dtype == SGBV_DTYPE_BF16 ? 2 : 4;
-    const int cells = (s.V + kCell - 1) / kCell;
-    const int nchains = s.B * s.K;
+    const int cells = cells_of(s.V);
+    const long nchains = (long)s.B * s.K;
     Plan plan;
     int C = g_opt_cluster;
     if (C == 0) {
         C = 1;
-        while ((cells + C - 1) / C * kCell > 5 * kChunk) C *= 2;  // smallest cluster whose slices fit
-        while (C < 8 && (long)nchains * C < 148 && cells / (2 * C) >= 4) C *= 2;  // few chains: spread each wider
+        while (slice_cells(cells, C) * kCell > kMaxNch * kChunk) C *= 2;  // smallest cluster whose slices fit
+        // few chains: spread each over more CTAs while they all stay co-resident in one wave
+        while (C < kMaxCluster && nchains * 2 * C <= kCtaSlots && cells / (2 * C) >= 4) C *= 2;
     }
-    if (C < 1 || C > 8 || (cells + C - 1) / C * kCell > 5 * kChunk) return SGBV_ERR_SHAPE;
+    if (C < 1 || C > kMaxCluster || slice_cells(cells, C) * kCell > kMaxNch * kChunk) return SGBV_ERR_SHAPE;
     plan.cluster = C;
-    plan.slice_len = (cells + C - 1) / C * kCell;
+    plan.slice_len = slice_cells(cells, C) * kCell;
     plan.nch = (plan.slice_len + kChunk - 1) / kChunk;
     const size_t stage_bytes = 2 * kChunk * esz;
-    int S = g_opt_stages ? g_opt_stages : 8;
-    const size_t budget = 227 * 1024 - sizeof(Control) - 1024;
+    int S = g_opt_stages ? g_opt_stages : kMaxStages;
+    const size_t budget = kSmemPerSm / 2 - kSmemReserved - sizeof(Control);
     if ((size_t)S * stage_bytes > budget) S = (int)(budget / stage_bytes);
-    if (S > 8) S = 8;
+    if (S > kMaxStages) S = kMaxStages;
     if (S < 2) return SGBV_ERR_SHAPE;
     plan.stages = S;
     plan.smem = (size_t)S * stage_bytes + sizeof(Control);

@@ -1,6 +1,6 @@
 // Generic two-sweep path: works for any V, any alignment, either dtype.
 //   sweep 1  (rowstats_kernel)  slice-wise (max, sum-exp) of every target and draft row i < gamma
-//   chain    (chain_kernel)     per draft: row normalisers, log a_i / log b_i, c_i, kappa_i
+//   chain    (chain_kernel)     per draft: row normalisers, c_i = p(x^i)/q(x^i), kappa_i
 //   sweep 2  (otreduce_kernel)  per-tile sums of the residual weights (and of the two
 //                               non-negative numerator terms when c_i < 1)
 // It reads each needed logit twice, so it is the fallback, not the fast path.
@@ -88,8 +88,7 @@ rowstats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
 template <typename T>
 __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all,
                              const int32_t *__restrict__ tok, Shape s, const float *__restrict__ part,
-                             RowInfo *__restrict__ rows, double *__restrict__ chain_end,
-                             int32_t *__restrict__ status) {
+                             RowInfo *__restrict__ rows, int32_t *__restrict__ status) {
     const int bk = blockIdx.x * blockDim.x + threadIdx.x;
     if (bk >= s.B * s.K) return;
     double la = 0.0, lb = 0.0;
@@ -108,8 +107,6 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
         }
         if (!(mq > -INFINITY) || !(mp > -INFINITY)) atomicOr(status + bk / s.K, SGBV_STATUS_NONFINITE_LOGIT);
         RowInfo ri;
-        ri.log_a = la;
-        ri.log_b = lb;
         ri.Zq = Zq;
         ri.Zp = Zp;
         ri.mq = mq;
@@ -128,8 +125,6 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
         la += ((double)zqt - (double)mq) * s.inv_T - log(Zq);
         lb += ((double)zpt - (double)mp) * s.inv_T - log(Zp);
     }
-    chain_end[2 * bk + 0] = la;
-    chain_end[2 * bk + 1] = lb;
 }
 
 // One warp per 256-element tile: lanes stride the tile, one shuffle reduction per sum.
@@ -191,7 +186,7 @@ int run(const Launch &L) {
     rowstats_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.part, L.ws.status);
     const int nbk = s.B * s.K;
     chain_kernel<T><<<(nbk + 127) / 128, 128, 0, L.stream>>>(zq, zp, L.tok, s, L.ws.part, L.ws.rows,
-                                                            L.ws.chain_end, L.ws.status);
+                                                            L.ws.status);
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
     otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, L.ws.wpart, L.ws.dpart, L.ws.mpart);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);

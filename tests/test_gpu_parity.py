@@ -146,8 +146,15 @@ def test_edge_shapes(B, K, gamma, V, dtype):
     assert_parity(rep)
 
 
-@pytest.mark.parametrize("option", [("path", 1), ("cluster", 1), ("cluster", 2), ("cluster", 4), ("cluster", 8),
-                                    ("stages", 2), ("max_clusters", 3)])
+def _slice_fits(V, cluster):
+    """A CTA of the fused kernel holds at most five chunks of 2048 elements of a row in registers."""
+    cells = -(-V // 256)
+    return -(-cells // cluster) * 256 <= 5 * 2048
+
+
+@pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 4),
+                                    ("cluster", 8), ("cluster", 16), ("stages", 2), ("stages", 3),
+                                    ("max_clusters", 3)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / ring depth /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
@@ -158,8 +165,8 @@ def test_every_kernel_path_and_launch_shape_matches(option):
     binding.set_option(*option)
     try:
         for cfg in cfgs:
-            if option == ("cluster", 1) and cfg.V > 20480:
-                continue   # a single CTA cannot hold more than five chunks of a row
+            if option[0] == "cluster" and not _slice_fits(cfg.V, option[1]):
+                continue   # forced cluster size whose slices do not fit the registers
             inp = workloads.make_inputs(cfg, device="cuda")
             rep, _, _ = run_both(inp)
             assert_parity(rep)
