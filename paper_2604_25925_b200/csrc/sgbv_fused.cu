@@ -1,26 +1,26 @@
 // Fused single-read path (steps A1-A3): one thread-block cluster walks one draft chain (b,k).
 //
 // For every position i = 0..gamma-1 of the chain the cluster
-//   * streams the target row and the draft row from HBM exactly once: one elected thread issues
-//     bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks
-//     into a shared-memory ring that runs ahead across rows and chains;
-//   * keeps the whole row pair resident in REGISTERS (each CTA of the cluster owns a contiguous
-//     slice of the vocabulary, each thread 8 elements of every chunk) as exponentials relative to
-//     the thread's own maximum, so the second sweep of the coupling sum never re-reads memory;
-//   * exchanges per-warp (max, sum-exp) partials by PUSHING them into every CTA's shared memory
-//     (distributed shared memory stores) followed by one cluster barrier per row; after the barrier
-//     every warp combines the partials locally and identically, so there is no second block-wide
-//     synchronisation and no remote load on the critical path;
-//   * runs the second sweep from registers and writes one partial sum per 256-element cell
-//     (a cell is what one warp owns in one chunk: 256 contiguous vocabulary entries).
-// The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread,
-// which computes c_{i+1} while the other warps are already in the second sweep of row i.
-// Two CTAs of 256 threads share an SM (different clusters), so one CTA's exchange latency is
-// covered by the other's arithmetic.  The finishing kernel (weights, scan, extra token) consumes
-// the cell sums.
+//   * streams the target row and the draft row from HBM exactly once.  Every WARP owns the
+//     256-element cells  warp, warp+8, warp+16, ...  of its CTA's slice of the vocabulary and runs
+//     its own ring of bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts, one
+//     cell of both tensors per stage) that runs ahead across rows and chains: no warp ever waits
+//     for another warp's loads, and there is no producer thread;
+//   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
+//     exponentials relative to the thread's own maximum, so the second
+//     sweep of the coupling sum never re-reads memory;
+//   * exchanges per-warp (max, sum-exp) partials by PUSHING them into every CTA's shared
+//     memory with asynchronous distributed-shared-memory stores that complete on the receiver's
+//     mbarrier; a warp goes on as soon as all partials of the row have landed.  There is no
+//     block-wide or cluster-wide barrier inside the row loop;
+//   * runs the second sweep from registers and writes one partial sum per cell.
+// The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread per
+// CTA, which computes c_{i+1} after its warp has pushed its partials of row i+1, i.e. while the
+// exchange is in flight.  Two CTAs of 256 threads share an SM (different clusters).  The finishing
+// kernel (weights, scan, extra token) consumes the cell sums.
 //
-// Every wait on an mbarrier is bounded; on expiry the CTA records an error flag and keeps
-// executing the protocol (all cluster barriers are still reached), so a lost copy cannot hang.
+// Every wait on an mbarrier is bounded; on expiry the warp records an error flag and keeps
+// executing the protocol, so a lost copy cannot hang the kernel.
 #include "sgbv_common.cuh"
 
 namespace sgbv {
@@ -30,9 +30,9 @@ namespace {
 constexpr int kFThreads = 256;
 constexpr int kFWarps = kFThreads / 32;
 constexpr int kCell = kTile;               // 256 contiguous elements: one warp's share of a chunk
-constexpr int kChunk = kFWarps * kCell;    // 2048 elements per chunk per tensor
-constexpr int kMaxNch = 5;                 // chunks of a row slice one CTA can hold in registers
-constexpr int kMaxStages = 12;
+constexpr int kChunk = kFWarps * kCell;    // 2048 elements: one cell of every warp
+constexpr int kMaxNch = 5;                 // cells per warp: what one thread can hold in registers (5 x 8 pairs)
+constexpr int kMaxStages = 12;             // ring depth per warp
 constexpr int kMaxCluster = 16;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
@@ -58,9 +58,6 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
@@ -98,13 +95,15 @@ __device__ __forceinline__ void cluster_arrive() {
 __device__ __forceinline__ void cluster_wait() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// Store 16 bytes into the shared memory of CTA `rank` of this cluster, at the address that
-// `local` has in this CTA.
-__device__ __forceinline__ void st_dsmem_f4(void *local, uint32_t rank, float4 v) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local)), "r"(rank));
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z),
-                 "f"(v.w)
+// Asynchronous store of 16 bytes into the shared memory of CTA `rank` of this cluster, at the
+// address that `local` has in this CTA; its completion is counted (16 bytes) on the receiver's
+// mbarrier that sits where `local_bar` sits here.
+__device__ __forceinline__ void push_f4(void *local, uint64_t *local_bar, uint32_t rank, float4 v) {
+    uint32_t dst, bar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(smem_u32(local)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(local_bar)), "r"(rank));
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1,%2,%3,%4}, [%5];" ::"r"(dst),
+                 "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(bar)
                  : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
@@ -119,29 +118,29 @@ __device__ __forceinline__ float rcp(float x) {
 }
 
 // ---- shared memory layout ------------------------------------------------------------------------
+// [ring: kFWarps x stages x (cell of zq, cell of zp)] [Control]
 struct Control {
-    uint64_t full[kMaxStages];
-    uint64_t empty[kMaxStages];
-    // per-warp partials (mq, sum eq, mp, sum ep) of every CTA of the cluster, pushed by their
-    // owners; double-buffered by row parity
+    uint64_t full[kFWarps][kMaxStages];  // one per warp and ring stage: "both cells have landed"
+    uint64_t xbar[2];                    // by row parity: "all partials of the row and c_i are here"
+    // per-warp partials (maximum of zq, sum eq, maximum of zp, sum ep) of every
+    // CTA of the cluster, pushed by their owners; double-buffered by row parity
     float4 slots[2][kMaxCluster * kFWarps];
-    double c[2];           // joint likelihood ratio c_i of the current chain, by row parity
-    int32_t tok[kMaxGamma];
+    double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
 };
 
-// Reads this lane's 8 elements of one chunk of one tensor from the ring.
+// Reads this lane's 8 elements of one cell of one tensor from the ring.
 template <typename T>
-__device__ __forceinline__ void read_cell(const unsigned char *stage_base, int warp, int lane, float (&v)[8]);
+__device__ __forceinline__ void read_cell(const unsigned char *cell_base, int lane, float (&v)[8]);
 template <>
-__device__ __forceinline__ void read_cell<float>(const unsigned char *stage_base, int warp, int lane, float (&v)[8]) {
-    const float4 *p = reinterpret_cast<const float4 *>(stage_base) + warp * 64 + lane;
+__device__ __forceinline__ void read_cell<float>(const unsigned char *cell_base, int lane, float (&v)[8]) {
+    const float4 *p = reinterpret_cast<const float4 *>(cell_base) + lane;
     const float4 a = p[0], b = p[32];
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
     v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
 }
 template <>
-__device__ __forceinline__ void read_cell<uint16_t>(const unsigned char *stage_base, int warp, int lane, float (&v)[8]) {
-    const uint4 a = reinterpret_cast<const uint4 *>(stage_base)[warp * 32 + lane];
+__device__ __forceinline__ void read_cell<uint16_t>(const unsigned char *cell_base, int lane, float (&v)[8]) {
+    const uint4 a = reinterpret_cast<const uint4 *>(cell_base)[lane];
     v[0] = __uint_as_float(a.x << 16); v[1] = __uint_as_float(a.x & 0xffff0000u);
     v[2] = __uint_as_float(a.y << 16); v[3] = __uint_as_float(a.y & 0xffff0000u);
     v[4] = __uint_as_float(a.z << 16); v[5] = __uint_as_float(a.z & 0xffff0000u);
@@ -173,20 +172,21 @@ __device__ __forceinline__ float ipow(float r, int K) {
 }
 
 // Second sweep over the register-resident row.  eq/ep are exponentials relative to the THREAD's
-// maxima; kt = kappa * (fp_t / fq_t) makes  c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d convert the
-// thread's sums to row-max units.  Per cell:
+// maxima; kt = kappa * (fp_t / fq_t) makes  c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d
+// convert the thread's sums to row-max units.  nj = number of cells this warp holds; the
+// output pointers address this warp's first cell, its cells are kFWarps apart.  Per cell:
 //   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
 //   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
 //   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
 template <int NCH, int KT, bool kAux>
 __device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
-                                          float scale_w, float scale_d, float c, int K, int lane, int warp,
-                                          int ncells_valid, float *wpart, float *dpart, float *mpart) {
+                                          float scale_w, float scale_d, float c, int K, int lane, int nj,
+                                          float *wpart, float *dpart, float *mpart) {
     const float v1 = 1.0f - c;
 #pragma unroll
     for (int j = 0; j < NCH; ++j) {
-        const int cell = j * kFWarps + warp;  // cell index inside this CTA's slice (warp-uniform)
-        if (cell >= ncells_valid) break;
+        if (j >= nj) break;  // warp-uniform
+        const int cell = j * kFWarps;
         float sw = 0.0f, sd = 0.0f, sm = 0.0f;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
@@ -242,10 +242,9 @@ __device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float
 
 template <int NCH, bool kAux>
 __device__ __forceinline__ void sweep_two_dispatch(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
-                                                   float scale_w, float scale_d, float c, int K, int lane, int warp,
-                                                   int ncells_valid, float *wpart, float *dpart, float *mpart) {
-#define SGBV_SWEEP(KT) \
-    sweep_two<NCH, KT, kAux>(eq, ep, kt, scale_w, scale_d, c, K, lane, warp, ncells_valid, wpart, dpart, mpart)
+                                                   float scale_w, float scale_d, float c, int K, int lane, int nj,
+                                                   float *wpart, float *dpart, float *mpart) {
+#define SGBV_SWEEP(KT) sweep_two<NCH, KT, kAux>(eq, ep, kt, scale_w, scale_d, c, K, lane, nj, wpart, dpart, mpart)
     switch (K) {
         case 1: SGBV_SWEEP(1); break;
         case 2: SGBV_SWEEP(2); break;
@@ -267,20 +266,25 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
     const int cid = blockIdx.x / C;
     const int G = gridDim.x / C;
     const int S = p.stages;
-    constexpr int kStageBytes = 2 * kChunk * (int)sizeof(T);
-    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)S * kStageBytes);
+    constexpr int kCellBytes = kCell * (int)sizeof(T);
+    constexpr int kStageBytes = 2 * kCellBytes;  // one cell of zq, then the same cell of zp
+    unsigned char *ring = smem + (size_t)warp * S * kStageBytes;
+    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * S * kStageBytes);
+    uint64_t *full = ctl->full[warp];
 
-    // this CTA's slice of the vocabulary
+    // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 8, ...
     const int x_begin = rank * p.slice_len;
     const int cta_len = max(0, min(s.V, x_begin + p.slice_len) - x_begin);
     const int ncells_valid = (cta_len + kCell - 1) / kCell;
-    const int first_cell = x_begin / kCell;
+    const int nj = ncells_valid > warp ? (ncells_valid - warp + kFWarps - 1) / kFWarps : 0;
+    const int first_cell = x_begin / kCell + warp;
+    const int x_warp = x_begin + warp * kCell;  // first element of this warp's first cell
 
     if (tid == 0) {
-        for (int i = 0; i < S; ++i) {
-            mbar_init(&ctl->full[i], 1);
-            mbar_init(&ctl->empty[i], kFWarps);
-        }
+        for (int w = 0; w < kFWarps; ++w)
+            for (int i = 0; i < S; ++i) mbar_init(&ctl->full[w][i], 1);
+        mbar_init(&ctl->xbar[0], 1);
+        mbar_init(&ctl->xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -288,67 +292,74 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
     cluster_wait();
 
     const int my_chains = (p.nchains - cid + G - 1) / G;
-    const int loads_per_chain = s.gamma * NCH;
-    const int total_loads = my_chains * loads_per_chain;
+    const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
+    const int total_loads = nrows * nj;         // cell pairs this warp loads
+    const uint32_t xbytes = (uint32_t)(C * kFWarps * sizeof(float4));
     bool timed_out = false;
 
-    // Producer (thread 0): loads are issued in consumption order; (p_cl, p_i, p_j, p_st) describe the
-    // next one: chain number within this cluster's list, position, chunk, ring stage.
-    int p_cl = 0, p_i = 0, p_j = 0, p_st = 0, p_issued = 0;
+    // Producer side of this warp's ring (lane 0): loads are issued in consumption order;
+    // (p_bk, p_i, p_j, p_st) describe the next one: chain, position, cell, ring stage.
+    int p_j = 0, p_st = 0, p_issued = 0;
+    size_t p_bk = (size_t)cid;
+    int p_i = 0;
     auto issue_next = [&]() {
-        const size_t bk = (size_t)cid + (size_t)p_cl * G;
-        const T *zq = reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + p_i) * s.V + x_begin + p_j * kChunk;
-        const T *zp = reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + p_i) * s.V + x_begin + p_j * kChunk;
-        const int nvalid = max(0, min(kChunk, cta_len - p_j * kChunk));
-        const uint32_t bytes = (uint32_t)nvalid * (uint32_t)sizeof(T);
-        mbar_expect_tx(&ctl->full[p_st], 2 * bytes);
-        if (bytes) {
-            unsigned char *dst = smem + (size_t)p_st * kStageBytes;
-            bulk_load(dst, zq, bytes, &ctl->full[p_st]);
-            bulk_load(dst + kChunk * sizeof(T), zp, bytes, &ctl->full[p_st]);
-        }
+        const int x0 = x_warp + p_j * kChunk;  // first element of the cell
+        const T *zq = reinterpret_cast<const T *>(p.zq) + (p_bk * (s.gamma + 1) + p_i) * s.V + x0;
+        const T *zp = reinterpret_cast<const T *>(p.zp) + (p_bk * s.gamma + p_i) * s.V + x0;
+        const uint32_t bytes = (uint32_t)min(kCell, s.V - x0) * (uint32_t)sizeof(T);
+        unsigned char *dst = ring + (size_t)p_st * kStageBytes;
+        mbar_expect_tx(&full[p_st], 2 * bytes);
+        bulk_load(dst, zq, bytes, &full[p_st]);
+        bulk_load(dst + kCellBytes, zp, bytes, &full[p_st]);
         ++p_issued;
         if (++p_st == S) p_st = 0;
-        if (++p_j == NCH) {
+        if (++p_j == nj) {
             p_j = 0;
             if (++p_i == s.gamma) {
                 p_i = 0;
-                ++p_cl;
+                p_bk += G;
             }
         }
     };
-    if (tid == 0) {
+    if (lane == 0) {
         const int first = total_loads < S ? total_loads : S;
         for (int k = 0; k < first; ++k) issue_next();
     }
 
-    // consumption state (same in every thread): ring stage and phase parity of the next chunk, and of
-    // the chunk consumed one step earlier (the one whose stage the producer refills)
-    int st = 0, prev_st = 0, consumed = 0, rowcount = 0;
-    uint32_t ph = 0, prev_ph = 0;
+    // The chain thread of this CTA (thread 0) carries c_i and fetches the token logits one row
+    // ahead: tok_next is the token of the next row of the walk.
+    int tok_next = 0;
+    if (tid == 0 && nrows > 0) tok_next = p.tok[(size_t)cid * s.gamma];
+    double c_run = 1.0;                 // c of the row being processed (chain thread)
+    float zq_tok = 0.0f, zp_tok = 0.0f;  // token logits of the previous row, and its statistics
+    float prev_bq = 0.0f, prev_bp = 0.0f, prev_Zq = 1.0f, prev_Zp = 1.0f;
+
+    int st = 0;
+    uint32_t ph = 0;
+    int n = 0;  // row number in this cluster's walk
     for (int cl = 0; cl < my_chains; ++cl) {
         const size_t bk = (size_t)cid + (size_t)cl * G;
         const int brow = (int)(bk / s.K);
-        if (tid < s.gamma) {
-            int t = p.tok[bk * s.gamma + tid];
-            if (t < 0 || t >= s.V) {
-                if (rank == 0) atomicOr(p.ws.status + brow, SGBV_STATUS_TOKEN_RANGE);
-                t = 0;
-            }
-            ctl->tok[tid] = t;
-        }
-        if (tid == 0) ctl->c[rowcount & 1] = 1.0;  // c_0 = 1 (empty prefix)
-        __syncthreads();
-
-        for (int i = 0; i < s.gamma; ++i) {
+        for (int i = 0; i < s.gamma; ++i, ++n) {
             const size_t r = bk * s.gamma + i;
-            const int par = rowcount & 1;
-            // token logits for the chain ratio: fetched now, used after the exchange
-            float zq_tok = 0.0f, zp_tok = 0.0f;
+            const int par = n & 1;
+            const uint32_t xph = (uint32_t)(n >> 1) & 1u;
+
+            // ---- chain thread: c_i from the previous row, then the token logits of this row ----------
+            float zq_tok_new = 0.0f, zp_tok_new = 0.0f;
             if (tid == 0) {
-                const int t = ctl->tok[i];
-                zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
-                zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
+                int t = tok_next;
+                if (t < 0 || t >= s.V) {
+                    if (rank == 0) atomicOr(p.ws.status + brow, SGBV_STATUS_TOKEN_RANGE);
+                    t = 0;
+                }
+                zq_tok_new = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
+                zp_tok_new = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
+                if (n + 1 < nrows) {
+                    const size_t bk_n = (i + 1 < s.gamma) ? bk : bk + G;
+                    const int i_n = (i + 1 < s.gamma) ? i + 1 : 0;
+                    tok_next = p.tok[bk_n * s.gamma + i_n];
+                }
             }
 
             // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
@@ -356,117 +367,124 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             float mq = -INFINITY, mp = -INFINITY;
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
-                if (tid == 0 && consumed >= 1 && p_issued < total_loads) {
-                    // refill the stage of the previous chunk once every warp has released it
-                    if (!mbar_wait(&ctl->empty[prev_st], prev_ph)) timed_out = true;
-                    issue_next();
-                }
-                if (!mbar_wait(&ctl->full[st], ph)) timed_out = true;
-                const unsigned char *base = smem + (size_t)st * kStageBytes;
-                const int cell = j * kFWarps + warp;
-                if (cell < ncells_valid) {
-                    read_cell<T>(base, warp, lane, eq[j]);
-                    read_cell<T>(base + kChunk * sizeof(T), warp, lane, ep[j]);
-                    const int cell_x = x_begin + cell * kCell;
+                if (j < nj) {  // warp-uniform
+                    if (!mbar_wait(&full[st], ph)) timed_out = true;
+                    const unsigned char *base = ring + (size_t)st * kStageBytes;
+                    read_cell<T>(base, lane, eq[j]);
+                    read_cell<T>(base + kCellBytes, lane, ep[j]);
+                    const int cell_x = x_warp + j * kChunk;
                     if (cell_x + kCell > s.V) {  // the row ends inside this cell
 #pragma unroll
                         for (int e = 0; e < 8; ++e)
                             if (cell_x + cell_offset<T>(lane, e) >= s.V) eq[j][e] = ep[j][e] = -INFINITY;
                     }
-                } else {
+                    __syncwarp();
+                    if (lane == 0 && p_issued < total_loads) issue_next();  // refill the stage just read
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) eq[j][e] = ep[j][e] = -INFINITY;
+                    for (int e = 0; e < 8; ++e) {
+                        mq = fmaxf(mq, eq[j][e]);
+                        mp = fmaxf(mp, ep[j][e]);
+                    }
+                    if (++st == S) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->empty[st]);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    mq = fmaxf(mq, eq[j][e]);
-                    mp = fmaxf(mp, ep[j][e]);
-                }
-                prev_st = st;
-                prev_ph = ph;
-                if (++st == S) {
-                    st = 0;
-                    ph ^= 1u;
-                }
-                ++consumed;
             }
-            // reference points of the exponentials: the thread's own maxima (0 if it saw only -inf)
+            // reference points of this thread's exponentials: its own maxima (0 if it saw only -inf);
+            // the maximum itself maps to exactly 1, so point-mass rows stay exact
             const bool has_q = mq > -INFINITY, has_p = mp > -INFINITY;
-            const float rq = has_q ? mq : 0.0f;
-            const float rp = has_p ? mp : 0.0f;
+            const float bq = has_q ? mq : 0.0f;
+            const float bp = has_p ? mp : 0.0f;
 
             // ---- first sweep, part 2: exponentials in place, sums ----------------------------------
             float sq = 0.0f, sp = 0.0f;
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
+                if (j < nj) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    eq[j][e] = ex2((eq[j][e] - rq) * s.scale);
-                    ep[j][e] = ex2((ep[j][e] - rp) * s.scale);
-                    sq += eq[j][e];
-                    sp += ep[j][e];
+                    for (int e = 0; e < 8; ++e) {
+                        eq[j][e] = ex2((eq[j][e] - bq) * s.scale);
+                        ep[j][e] = ex2((ep[j][e] - bp) * s.scale);
+                        sq += eq[j][e];
+                        sp += ep[j][e];
+                    }
                 }
             }
-            // warp partials in warp-max units, pushed to every CTA of the cluster
-            const float mqw = warp_max(mq), mpw = warp_max(mp);
-            const float rqw = (mqw > -INFINITY) ? mqw : 0.0f, rpw = (mpw > -INFINITY) ? mpw : 0.0f;
-            sq = warp_sum(has_q ? sq * ex2((rq - rqw) * s.scale) : 0.0f);
-            sp = warp_sum(has_p ? sp * ex2((rp - rpw) * s.scale) : 0.0f);
-            if (lane < C) st_dsmem_f4(&ctl->slots[par][rank * kFWarps + warp], (uint32_t)lane, make_float4(mqw, sq, mpw, sp));
-            cluster_arrive();
-            cluster_wait();
+            // warp partials relative to the warp's maxima, pushed to every CTA
+            const float bqw = warp_max(has_q ? bq : -INFINITY), bpw = warp_max(has_p ? bp : -INFINITY);
+            const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
+            sq = warp_sum(has_q ? sq * ex2((bq - rqw) * s.scale) : 0.0f);
+            sp = warp_sum(has_p ? sp * ex2((bp - rpw) * s.scale) : 0.0f);
+            if (lane < C)
+                push_f4(&ctl->slots[par][rank * kFWarps + warp], &ctl->xbar[par], (uint32_t)lane,
+                        make_float4(bqw, sq, bpw, sp));
+
+            if (tid == 0) {
+                // c_i = c_{i-1} p_{i-1}(tok)/q_{i-1}(tok) from the previous row's statistics; c_0 = 1
+                if (i > 0) {
+                    const double lp = ((double)zp_tok - (double)prev_bp) * (double)s.scale;
+                    const double lq = ((double)zq_tok - (double)prev_bq) * (double)s.scale;
+                    c_run *= exp2(lp - lq) * ((double)prev_Zq / (double)prev_Zp);
+                } else {
+                    c_run = 1.0;
+                }
+                ctl->c[par] = c_run;
+                mbar_expect_tx(&ctl->xbar[par], xbytes);  // arms the exchange and publishes c_i
+                zq_tok = zq_tok_new;
+                zp_tok = zp_tok_new;
+            }
+            if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
 
             // ---- row statistics: every warp combines all partials, in the same order ------------------
-            float mq_row = -INFINITY, mp_row = -INFINITY;
+            float bq_row = -INFINITY, bp_row = -INFINITY;
             const int nslots = C * kFWarps;
             for (int e = lane; e < nslots; e += 32) {
                 const float4 v = ctl->slots[par][e];
-                mq_row = fmaxf(mq_row, v.x);
-                mp_row = fmaxf(mp_row, v.z);
+                bq_row = fmaxf(bq_row, v.x);
+                bp_row = fmaxf(bp_row, v.z);
             }
-            mq_row = warp_max(mq_row);
-            mp_row = warp_max(mp_row);
-            const float rq_row = (mq_row > -INFINITY) ? mq_row : 0.0f, rp_row = (mp_row > -INFINITY) ? mp_row : 0.0f;
-            double Zq = 0.0, Zp = 0.0;
+            bq_row = warp_max(bq_row);
+            bp_row = warp_max(bp_row);
+            const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
+            float Zq = 0.0f, Zp = 0.0f;
             for (int e = lane; e < nslots; e += 32) {
                 const float4 v = ctl->slots[par][e];
-                if (v.x > -INFINITY) Zq += (double)(v.y * ex2((v.x - rq_row) * s.scale));
-                if (v.z > -INFINITY) Zp += (double)(v.w * ex2((v.z - rp_row) * s.scale));
+                if (v.x > -INFINITY) Zq = fmaf(v.y, ex2((v.x - rq_row) * s.scale), Zq);
+                if (v.z > -INFINITY) Zp = fmaf(v.w, ex2((v.z - rp_row) * s.scale), Zp);
             }
             Zq = warp_sum(Zq);
             Zp = warp_sum(Zp);
             const double cd = ctl->c[par];
-            const double kappa_d = cd * Zq / Zp;
             const float c = (float)cd;
+            const float kappa = (float)(cd * (double)(Zq / Zp));
 
             if (tid == 0) {
-                // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
-                // -inf only has Z = 0
-                const bool bad = !(Zq > 0.0) || !(Zp > 0.0) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
-                                 !(mq_row < INFINITY) || !(mp_row < INFINITY);
+                prev_bq = rq_row;
+                prev_bp = rp_row;
+                prev_Zq = Zq;
+                prev_Zp = Zp;
                 if (rank == 0) {
+                    // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
+                    // -inf only has Z = 0
+                    const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
+                                     !(bq_row < INFINITY) || !(bp_row < INFINITY);
                     if (bad) atomicOr(p.ws.status + brow, SGBV_STATUS_NONFINITE_LOGIT);
                     RowInfo ri;
-                    ri.Zq = Zq;
-                    ri.Zp = Zp;
-                    ri.mq = mq_row;
-                    ri.mp = mp_row;
-                    ri.kappa = (float)kappa_d;
+                    ri.Zq = (double)Zq;
+                    ri.Zp = (double)Zp;
+                    ri.mq = bq_row;
+                    ri.mp = bp_row;
+                    ri.kappa = kappa;
                     ri.c = c;
                     p.ws.rows[r] = ri;
                 }
-                // c_{i+1} = c_i p_i(tok_i)/q_i(tok_i), for the next row of this chain
-                const double lp = ((double)zp_tok - (double)mp_row) * s.inv_T;
-                const double lq = ((double)zq_tok - (double)mq_row) * s.inv_T;
-                ctl->c[par ^ 1] = cd * exp(lp - lq) * (Zq / Zp);
             }
 
             // thread units -> row units
-            const float fq = has_q ? ex2((rq - rq_row) * s.scale) : 0.0f;
-            const float fp = has_p ? ex2((rp - rp_row) * s.scale) : 0.0f;
-            float kt = (float)kappa_d * fp / fq;
+            const float fq = has_q ? ex2((bq - rq_row) * s.scale) : 0.0f;
+            const float fp = has_p ? ex2((bp - rp_row) * s.scale) : 0.0f;
+            float kt = kappa * fp / fq;
             float scale_w = fq, scale_d = fq;
             if (__any_sync(0xffffffffu, !(fq > 1e-30f))) {
                 // a thread whose share of the target row underflows (or nearly so, which would
@@ -478,7 +496,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
                         for (int e = 0; e < 8; ++e) eq[j][e] = 0.0f;
                     kt = 1.0f;
                     scale_w = 0.0f;
-                    scale_d = (float)kappa_d * fp;
+                    scale_d = kappa * fp;
                 }
             }
 
@@ -486,14 +504,12 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
                   *mpp = p.ws.mpart + r * s.ntiles + first_cell;
             if (c < 1.0f)
-                sweep_two_dispatch<NCH, true>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, warp, ncells_valid, wp, dp, mpp);
+                sweep_two_dispatch<NCH, true>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
             else
-                sweep_two_dispatch<NCH, false>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, warp, ncells_valid, wp, dp, mpp);
-            ++rowcount;
+                sweep_two_dispatch<NCH, false>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
         }
-        __syncthreads();  // ctl->tok and ctl->c are rewritten for the next chain
     }
-    if (timed_out) atomicExch(p.error_flag, 1);
+    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(p.error_flag, 1);
     cluster_arrive();  // no CTA leaves while a neighbour may still write into its slots
     cluster_wait();
 }

@@ -71,11 +71,23 @@ def sweep_c5():
 
 
 def get_config(name: str) -> VerifyConfig:
+    """A named configuration (c1..c4, c5_K*_a*_T*), or a spec such as
+    ``B=8,K=8,gamma=8,V=151936,dtype=fp32,T=1.0,alpha=0.9`` (omitted fields keep their defaults)."""
     if name in CONFIGS:
         return CONFIGS[name]
     for c in sweep_c5():
         if c.name == name:
             return c
+    if "=" in name:
+        alias = {"T": "temperature", "g": "gamma"}
+        kinds = {"B": int, "K": int, "gamma": int, "V": int, "dtype": str, "temperature": float,
+                 "alpha": float, "sigma": float, "boost": float, "zipf_s": float, "seed": int}
+        fields = {"B": 8, "K": 4, "gamma": 4, "V": 32000}
+        for part in name.split(","):
+            k, v = part.split("=")
+            k = alias.get(k.strip(), k.strip())
+            fields[k] = kinds[k](v.strip())
+        return VerifyConfig(name.replace(" ", ""), **fields)
     raise KeyError(name)
 
 
