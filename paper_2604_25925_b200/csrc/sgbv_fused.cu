@@ -1,11 +1,12 @@
 // Fused single-read path (steps A1-A3): one thread-block cluster walks one draft chain (b,k).
 //
 // For every position i = 0..gamma-1 of the chain the cluster
-//   * streams the target row and the draft row from HBM exactly once.  Every WARP owns the
-//     256-element cells  warp, warp+8, warp+16, ...  of its CTA's slice of the vocabulary and runs
-//     its own ring of bulk asynchronous copies (cp.async.bulk + mbarrier transaction counts, one
-//     cell of both tensors per stage) that runs ahead across rows and chains: no warp ever waits
-//     for another warp's loads, and there is no producer thread;
+//   * streams the target row and the draft row from HBM exactly once: bulk asynchronous copies
+//     (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks of both tensors into a
+//     shared-memory ring that runs ahead across rows and chains.  A warp owns the 256-element
+//     cells  warp, warp+8, warp+16, ...  of its CTA's slice.  There is no producer thread: the
+//     warp that is LAST to finish reading a ring stage refills it, so no warp waits for another
+//     one to release a stage, and the copies stay large (few requests to the copy engine);
 //   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
 //     exponentials relative to the thread's own maximum, so the second
 //     sweep of the coupling sum never re-reads memory;
@@ -32,7 +33,7 @@ constexpr int kFWarps = kFThreads / 32;
 constexpr int kCell = kTile;               // 256 contiguous elements: one warp's share of a chunk
 constexpr int kChunk = kFWarps * kCell;    // 2048 elements: one cell of every warp
 constexpr int kMaxNch = 5;                 // cells per warp: what one thread can hold in registers (5 x 8 pairs)
-constexpr int kMaxStages = 12;             // ring depth per warp
+constexpr int kMaxStages = 12;             // ring depth
 constexpr int kMaxCluster = 16;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
@@ -118,9 +119,10 @@ __device__ __forceinline__ float rcp(float x) {
 }
 
 // ---- shared memory layout ------------------------------------------------------------------------
-// [ring: kFWarps x stages x (cell of zq, cell of zp)] [Control]
+// [ring: stages x (chunk of zq, chunk of zp)] [Control]
 struct Control {
-    uint64_t full[kFWarps][kMaxStages];  // one per warp and ring stage: "both cells have landed"
+    uint64_t full[kMaxStages];           // per ring stage: "both chunks have landed"
+    int readers_done[kMaxStages];        // per ring stage: warps that have finished reading it
     uint64_t xbar[2];                    // by row parity: "all partials of the row and c_i are here"
     // per-warp partials (maximum of zq, sum eq, maximum of zp, sum ep) of every
     // CTA of the cluster, pushed by their owners; double-buffered by row parity
@@ -267,22 +269,26 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
     const int G = gridDim.x / C;
     const int S = p.stages;
     constexpr int kCellBytes = kCell * (int)sizeof(T);
-    constexpr int kStageBytes = 2 * kCellBytes;  // one cell of zq, then the same cell of zp
-    unsigned char *ring = smem + (size_t)warp * S * kStageBytes;
-    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * S * kStageBytes);
-    uint64_t *full = ctl->full[warp];
+    constexpr int kChunkBytes = kChunk * (int)sizeof(T);
+    constexpr int kStageBytes = 2 * kChunkBytes;  // one chunk of zq, then the same chunk of zp
+    unsigned char *ring = smem;
+    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)S * kStageBytes);
+    uint64_t *full = ctl->full;
 
     // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 8, ...
     const int x_begin = rank * p.slice_len;
     const int cta_len = max(0, min(s.V, x_begin + p.slice_len) - x_begin);
     const int ncells_valid = (cta_len + kCell - 1) / kCell;
     const int nj = ncells_valid > warp ? (ncells_valid - warp + kFWarps - 1) / kFWarps : 0;
+    const int nchunks = (ncells_valid + kFWarps - 1) / kFWarps;  // chunks per row of this CTA
     const int first_cell = x_begin / kCell + warp;
     const int x_warp = x_begin + warp * kCell;  // first element of this warp's first cell
 
     if (tid == 0) {
-        for (int w = 0; w < kFWarps; ++w)
-            for (int i = 0; i < S; ++i) mbar_init(&ctl->full[w][i], 1);
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&ctl->full[i], 1);
+            ctl->readers_done[i] = 0;
+        }
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -293,27 +299,31 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
 
     const int my_chains = (p.nchains - cid + G - 1) / G;
     const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
-    const int total_loads = nrows * nj;         // cell pairs this warp loads
+    const int total_loads = nrows * nchunks;    // chunk pairs this CTA loads
     const uint32_t xbytes = (uint32_t)(C * kFWarps * sizeof(float4));
     bool timed_out = false;
 
-    // Producer side of this warp's ring (lane 0): loads are issued in consumption order;
-    // (p_bk, p_i, p_j, p_st) describe the next one: chain, position, cell, ring stage.
+    // Producer state, kept identically by lane 0 of every warp: loads are issued in consumption
+    // order; (p_bk, p_i, p_j, p_st) describe the next one: chain, position, chunk, ring stage.
+    // advance_producer(true) issues it, advance_producer(false) only steps the state (another
+    // warp issues that load).
     int p_j = 0, p_st = 0, p_issued = 0;
     size_t p_bk = (size_t)cid;
     int p_i = 0;
-    auto issue_next = [&]() {
-        const int x0 = x_warp + p_j * kChunk;  // first element of the cell
-        const T *zq = reinterpret_cast<const T *>(p.zq) + (p_bk * (s.gamma + 1) + p_i) * s.V + x0;
-        const T *zp = reinterpret_cast<const T *>(p.zp) + (p_bk * s.gamma + p_i) * s.V + x0;
-        const uint32_t bytes = (uint32_t)min(kCell, s.V - x0) * (uint32_t)sizeof(T);
-        unsigned char *dst = ring + (size_t)p_st * kStageBytes;
-        mbar_expect_tx(&full[p_st], 2 * bytes);
-        bulk_load(dst, zq, bytes, &full[p_st]);
-        bulk_load(dst + kCellBytes, zp, bytes, &full[p_st]);
+    auto advance_producer = [&](bool issue) {
+        if (issue) {
+            const int x0 = x_begin + p_j * kChunk;  // first element of the chunk
+            const T *zq = reinterpret_cast<const T *>(p.zq) + (p_bk * (s.gamma + 1) + p_i) * s.V + x0;
+            const T *zp = reinterpret_cast<const T *>(p.zp) + (p_bk * s.gamma + p_i) * s.V + x0;
+            const uint32_t bytes = (uint32_t)min(kChunk, cta_len - p_j * kChunk) * (uint32_t)sizeof(T);
+            unsigned char *dst = ring + (size_t)p_st * kStageBytes;
+            mbar_expect_tx(&full[p_st], 2 * bytes);
+            bulk_load(dst, zq, bytes, &full[p_st]);
+            bulk_load(dst + kChunkBytes, zp, bytes, &full[p_st]);
+        }
         ++p_issued;
         if (++p_st == S) p_st = 0;
-        if (++p_j == nj) {
+        if (++p_j == nchunks) {
             p_j = 0;
             if (++p_i == s.gamma) {
                 p_i = 0;
@@ -323,7 +333,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
     };
     if (lane == 0) {
         const int first = total_loads < S ? total_loads : S;
-        for (int k = 0; k < first; ++k) issue_next();
+        for (int k = 0; k < first; ++k) advance_producer(warp == 0);  // warp 0 issues the first S loads
     }
 
     // The chain thread of this CTA (thread 0) carries c_i and fetches the token logits one row
@@ -367,23 +377,34 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             float mq = -INFINITY, mp = -INFINITY;
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
-                if (j < nj) {  // warp-uniform
+                if (j < nchunks) {  // uniform over the CTA
+                    // every warp waits, also one without a cell in this chunk: it must not count
+                    // itself done with the stage's next use before this use has been refilled
                     if (!mbar_wait(&full[st], ph)) timed_out = true;
-                    const unsigned char *base = ring + (size_t)st * kStageBytes;
-                    read_cell<T>(base, lane, eq[j]);
-                    read_cell<T>(base + kCellBytes, lane, ep[j]);
-                    const int cell_x = x_warp + j * kChunk;
-                    if (cell_x + kCell > s.V) {  // the row ends inside this cell
+                    if (j < nj) {  // warp-uniform
+                        const unsigned char *base = ring + (size_t)st * kStageBytes + warp * kCellBytes;
+                        read_cell<T>(base, lane, eq[j]);
+                        read_cell<T>(base + kChunkBytes, lane, ep[j]);
+                        const int cell_x = x_warp + j * kChunk;
+                        if (cell_x + kCell > s.V) {  // the row ends inside this cell
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            if (cell_x + cell_offset<T>(lane, e) >= s.V) eq[j][e] = ep[j][e] = -INFINITY;
+                            for (int e = 0; e < 8; ++e)
+                                if (cell_x + cell_offset<T>(lane, e) >= s.V) eq[j][e] = ep[j][e] = -INFINITY;
+                        }
                     }
                     __syncwarp();
-                    if (lane == 0 && p_issued < total_loads) issue_next();  // refill the stage just read
+                    if (lane == 0) {
+                        // the last warp to finish with this stage refills it with the chunk S ahead
+                        const bool last = atomicAdd(&ctl->readers_done[st], 1) == kFWarps - 1;
+                        if (last) ctl->readers_done[st] = 0;
+                        if (p_issued < total_loads) advance_producer(last);
+                    }
+                    if (j < nj) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        mq = fmaxf(mq, eq[j][e]);
-                        mp = fmaxf(mp, ep[j][e]);
+                        for (int e = 0; e < 8; ++e) {
+                            mq = fmaxf(mq, eq[j][e]);
+                            mp = fmaxf(mp, ep[j][e]);
+                        }
                     }
                     if (++st == S) {
                         st = 0;
