@@ -132,21 +132,21 @@ struct Control {
 
 // Reads this lane's 8 elements of one cell of one tensor from the ring.
 template <typename T>
-__device__ __forceinline__ void read_cell(const unsigned char *cell_base, int lane, float (&v)[8]);
+__device__ __forceinline__ void read_cell(const unsigned char *cell_base, int lane, float2 (&v)[4]);
 template <>
-__device__ __forceinline__ void read_cell<float>(const unsigned char *cell_base, int lane, float (&v)[8]) {
+__device__ __forceinline__ void read_cell<float>(const unsigned char *cell_base, int lane, float2 (&v)[4]) {
     const float4 *p = reinterpret_cast<const float4 *>(cell_base) + lane;
     const float4 a = p[0], b = p[32];
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    v[0] = make_float2(a.x, a.y); v[1] = make_float2(a.z, a.w);
+    v[2] = make_float2(b.x, b.y); v[3] = make_float2(b.z, b.w);
 }
 template <>
-__device__ __forceinline__ void read_cell<uint16_t>(const unsigned char *cell_base, int lane, float (&v)[8]) {
+__device__ __forceinline__ void read_cell<uint16_t>(const unsigned char *cell_base, int lane, float2 (&v)[4]) {
     const uint4 a = reinterpret_cast<const uint4 *>(cell_base)[lane];
-    v[0] = __uint_as_float(a.x << 16); v[1] = __uint_as_float(a.x & 0xffff0000u);
-    v[2] = __uint_as_float(a.y << 16); v[3] = __uint_as_float(a.y & 0xffff0000u);
-    v[4] = __uint_as_float(a.z << 16); v[5] = __uint_as_float(a.z & 0xffff0000u);
-    v[6] = __uint_as_float(a.w << 16); v[7] = __uint_as_float(a.w & 0xffff0000u);
+    v[0] = make_float2(__uint_as_float(a.x << 16), __uint_as_float(a.x & 0xffff0000u));
+    v[1] = make_float2(__uint_as_float(a.y << 16), __uint_as_float(a.y & 0xffff0000u));
+    v[2] = make_float2(__uint_as_float(a.z << 16), __uint_as_float(a.z & 0xffff0000u));
+    v[3] = make_float2(__uint_as_float(a.w << 16), __uint_as_float(a.w & 0xffff0000u));
 }
 // Offset (in elements, within the 256-element cell) of this lane's e-th element.
 template <typename T>
@@ -155,95 +155,149 @@ __device__ __forceinline__ int cell_offset(int lane, int e) {
     return lane * 8 + e;
 }
 
-// r^K for r in [0,1]; KT > 0 is a compile-time K.
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ __forceinline__ float2 splat(float x) { return make_float2(x, x); }
+
+// r^K for both halves of r, r in [0,1]; KT > 1 is a compile-time K, KT = 0 takes K at run time.
 template <int KT>
-__device__ __forceinline__ float ipow(float r, int K) {
-    if (KT == 1) return 1.0f;  // callers multiply by the base themselves where K = 1 matters
+__device__ __forceinline__ float2 ipow2(float2 r, int K) {
     if (KT > 1) {
-        float acc = (KT & 1) ? r : 1.0f, sq = r;
+        float2 acc = r, sq = r;  // acc is only read once it has been assigned
+        bool have = (KT & 1) != 0;
 #pragma unroll
         for (int k = KT >> 1; k > 0; k >>= 1) {
-            sq *= sq;
-            if (k & 1) acc *= sq;
+            sq = __fmul2_rn(sq, sq);
+            if (k & 1) {
+                acc = have ? __fmul2_rn(acc, sq) : sq;
+                have = true;
+            }
         }
         return acc;
     }
-    float acc = 1.0f;
-    for (int t = 0; t < K; ++t) acc *= r;
+    float2 acc = r;
+    for (int t = 1; t < K; ++t) acc = __fmul2_rn(acc, r);
     return acc;
 }
 
-// Second sweep over the register-resident row.  eq/ep are exponentials relative to the THREAD's
-// maxima; kt = kappa * (fp_t / fq_t) makes  c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d
-// convert the thread's sums to row-max units.  nj = number of cells this warp holds; the
-// output pointers address this warp's first cell, its cells are kFWarps apart.  Per cell:
+// Sums N values over the 32 lanes of a warp at once ("transposed" butterfly: at every step a lane
+// hands half of its values to its partner and keeps the other half).  P = N rounded up to a power
+// of two (<= 16).  On return v[0] of lane l is the warp total of value number owner_index<P>(l).
+template <int P>
+__device__ __forceinline__ int owner_index(int lane) {
+    int idx = 0;
+    if (P >= 2) idx += (lane & 16) ? P / 2 : 0;
+    if (P >= 4) idx += (lane & 8) ? P / 4 : 0;
+    if (P >= 8) idx += (lane & 4) ? P / 8 : 0;
+    if (P >= 16) idx += (lane & 2) ? P / 16 : 0;
+    return idx;
+}
+template <int P>
+__device__ __forceinline__ void warp_sum_multi(float (&v)[P], int lane) {
+    int off = 16;
+#pragma unroll
+    for (int n = P; n > 1; n >>= 1, off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int k = 0; k < n / 2; ++k) {
+            const float keep = upper ? v[k + n / 2] : v[k];
+            const float send = upper ? v[k] : v[k + n / 2];
+            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
+}
+
+// Second sweep over the register-resident row, two vocabulary entries per instruction (f32x2).
+// eq/ep are exponentials relative to the THREAD's maxima; kt = kappa * (fp_t / fq_t) makes
+// c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d convert the thread's sums to row-max units.
+// nj = number of cells this warp holds; the output pointers address this warp's first cell, its
+// cells are kFWarps apart.  Per cell:
 //   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
 //   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
 //   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
 template <int NCH, int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
+__device__ __forceinline__ void sweep_two(const float2 (&eq)[NCH][4], const float2 (&ep)[NCH][4], float kt,
                                           float scale_w, float scale_d, float c, int K, int lane, int nj,
                                           float *wpart, float *dpart, float *mpart) {
+    constexpr int NV = kAux ? 3 * NCH : NCH;
+    constexpr int P = NV <= 1 ? 1 : NV <= 2 ? 2 : NV <= 4 ? 4 : NV <= 8 ? 8 : 16;
+    static_assert(NV <= 16, "at most 16 sums per thread");
+    float sums[P];
+#pragma unroll
+    for (int k = 0; k < P; ++k) sums[k] = 0.0f;
     const float v1 = 1.0f - c;
+    const float2 nkt = splat(-kt), nv1 = splat(-v1);
+    // Horner coefficients of Q: (t+1) (1-c)^t, t = 1..K-2 (uniform over the row)
+    float2 coef[KT > 2 ? KT - 2 : 1];
+    if (kAux && KT > 2) {
+        float vj = 1.0f;
+#pragma unroll
+        for (int t = 1; t <= KT - 2; ++t) {
+            vj *= v1;
+            coef[t - 1] = splat((float)(t + 1) * vj);
+        }
+    }
 #pragma unroll
     for (int j = 0; j < NCH; ++j) {
         if (j >= nj) break;  // warp-uniform
-        const int cell = j * kFWarps;
-        float sw = 0.0f, sd = 0.0f, sm = 0.0f;
+        float2 sw = splat(0.0f), sd = splat(0.0f), sm = splat(0.0f);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float q = eq[j][e];
-            const float diff = fmaf(-kt, ep[j][e], q);      // q - c p, thread units
-            if (KT == 1 && !kAux) {
-                sw += fmaxf(diff, 0.0f);
-                continue;
-            }
+        for (int e = 0; e < 4; ++e) {
+            const float2 q = eq[j][e];
+            const float2 diff = __ffma2_rn(nkt, ep[j][e], q);  // q - c p, thread units
+            const float2 pos = make_float2(fmaxf(diff.x, 0.0f), fmaxf(diff.y, 0.0f));
+            if (KT == 1) sw = __fadd2_rn(sw, pos);
+            if (KT == 1 && !kAux) continue;
             // r = 1 - min{c p/q, 1}; q = 0 gives -inf or NaN before the clamp, 0 after it
-            const float r = fmaxf(diff * rcp(q), 0.0f);
-            if (KT == 1) sw += fmaxf(diff, 0.0f);
-            else sw = fmaf(q, ipow<KT>(r, K), sw);
+            const float2 t = __fmul2_rn(diff, make_float2(rcp(q.x), rcp(q.y)));
+            const float2 r = make_float2(fmaxf(t.x, 0.0f), fmaxf(t.y, 0.0f));
+            if (KT != 1) sw = __ffma2_rn(q, ipow2<KT>(r, K), sw);
             if (kAux) {
-                sd += fmaxf(-diff, 0.0f);
-                float acc = 0.0f;
+                sd = __fadd2_rn(sd, make_float2(fmaxf(-diff.x, 0.0f), fmaxf(-diff.y, 0.0f)));
+                float2 acc = splat(0.0f);
                 if (KT > 0) {
                     if (KT >= 2) {
-                        acc = 1.0f;
-                        float vj = 1.0f;
+                        acc = splat(1.0f);
 #pragma unroll
-                        for (int t = 1; t <= KT - 2; ++t) {
-                            vj *= v1;
-                            acc = fmaf(acc, r, (float)(t + 1) * vj);
-                        }
+                        for (int u = 0; u < KT - 2; ++u) acc = __ffma2_rn(acc, r, coef[u]);
                     }
                 } else if (K >= 2) {
-                    acc = 1.0f;
+                    acc = splat(1.0f);
                     float vj = 1.0f;
-                    for (int t = 1; t <= K - 2; ++t) {
+                    for (int u = 1; u <= K - 2; ++u) {
                         vj *= v1;
-                        acc = fmaf(acc, r, (float)(t + 1) * vj);
+                        acc = __ffma2_rn(acc, r, splat((float)(u + 1) * vj));
                     }
                 }
-                const float ct = r - v1;  // c - t with t = 1 - r
-                sm = fmaf(q * ct * ct, acc, sm);
+                const float2 ct = __fadd2_rn(r, nv1);  // c - t with t = 1 - r
+                sm = __ffma2_rn(__fmul2_rn(q, __fmul2_rn(ct, ct)), acc, sm);
             }
         }
-        sw = warp_sum(sw * scale_w);
+        sums[j] = (sw.x + sw.y) * scale_w;
         if (kAux) {
-            sd = warp_sum(sd * scale_d);
-            sm = warp_sum(sm * scale_w);
+            sums[NCH + j] = (sd.x + sd.y) * scale_d;
+            sums[2 * NCH + j] = (sm.x + sm.y) * scale_w;
         }
-        if (lane == 0) {
-            wpart[cell] = sw;
-            if (kAux) {
-                dpart[cell] = sd;
-                mpart[cell] = sm;
-            }
+    }
+    warp_sum_multi<P>(sums, lane);
+    // the lane that owns value number idx (and has the low lane bits clear) stores it
+    const int idx = owner_index<P>(lane);
+    constexpr int kLowMask = P >= 16 ? 1 : P >= 8 ? 3 : P >= 4 ? 7 : P >= 2 ? 15 : 31;
+    if ((lane & kLowMask) == 0 && idx < NV) {
+        const int jj = kAux ? idx % NCH : idx, which = kAux ? idx / NCH : 0;
+        if (jj < nj) {
+            float *dst = which == 0 ? wpart : which == 1 ? dpart : mpart;
+            dst[jj * kFWarps] = sums[0];
         }
     }
 }
 
 template <int NCH, bool kAux>
-__device__ __forceinline__ void sweep_two_dispatch(const float (&eq)[NCH][8], const float (&ep)[NCH][8], float kt,
+__device__ __forceinline__ void sweep_two_dispatch(const float2 (&eq)[NCH][4], const float2 (&ep)[NCH][4], float kt,
                                                    float scale_w, float scale_d, float c, int K, int lane, int nj,
                                                    float *wpart, float *dpart, float *mpart) {
 #define SGBV_SWEEP(KT) sweep_two<NCH, KT, kAux>(eq, ep, kt, scale_w, scale_d, c, K, lane, nj, wpart, dpart, mpart)
@@ -373,7 +427,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             }
 
             // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
-            float eq[NCH][8], ep[NCH][8];
+            float2 eq[NCH][4], ep[NCH][4];  // two neighbouring vocabulary entries per register pair
             float mq = -INFINITY, mp = -INFINITY;
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
@@ -388,8 +442,10 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
                         const int cell_x = x_warp + j * kChunk;
                         if (cell_x + kCell > s.V) {  // the row ends inside this cell
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                if (cell_x + cell_offset<T>(lane, e) >= s.V) eq[j][e] = ep[j][e] = -INFINITY;
+                            for (int e = 0; e < 4; ++e) {
+                                if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[j][e].x = ep[j][e].x = -INFINITY;
+                                if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[j][e].y = ep[j][e].y = -INFINITY;
+                            }
                         }
                     }
                     __syncwarp();
@@ -401,9 +457,9 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
                     }
                     if (j < nj) {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            mq = fmaxf(mq, eq[j][e]);
-                            mp = fmaxf(mp, ep[j][e]);
+                        for (int e = 0; e < 4; ++e) {
+                            mq = max3(mq, eq[j][e].x, eq[j][e].y);
+                            mp = max3(mp, ep[j][e].x, ep[j][e].y);
                         }
                     }
                     if (++st == S) {
@@ -419,19 +475,23 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             const float bp = has_p ? mp : 0.0f;
 
             // ---- first sweep, part 2: exponentials in place, sums ----------------------------------
-            float sq = 0.0f, sp = 0.0f;
+            float2 sq2 = splat(0.0f), sp2 = splat(0.0f);
+            const float2 nbq = splat(-bq), nbp = splat(-bp), sc2 = splat(s.scale);
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 if (j < nj) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        eq[j][e] = ex2((eq[j][e] - bq) * s.scale);
-                        ep[j][e] = ex2((ep[j][e] - bp) * s.scale);
-                        sq += eq[j][e];
-                        sp += ep[j][e];
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 aq = __fmul2_rn(__fadd2_rn(eq[j][e], nbq), sc2);
+                        const float2 ap = __fmul2_rn(__fadd2_rn(ep[j][e], nbp), sc2);
+                        eq[j][e] = make_float2(ex2(aq.x), ex2(aq.y));
+                        ep[j][e] = make_float2(ex2(ap.x), ex2(ap.y));
+                        sq2 = __fadd2_rn(sq2, eq[j][e]);
+                        sp2 = __fadd2_rn(sp2, ep[j][e]);
                     }
                 }
             }
+            float sq = sq2.x + sq2.y, sp = sp2.x + sp2.y;
             // warp partials relative to the warp's maxima, pushed to every CTA
             const float bqw = warp_max(has_q ? bq : -INFINITY), bpw = warp_max(has_p ? bp : -INFINITY);
             const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
@@ -514,7 +574,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
 #pragma unroll
                     for (int j = 0; j < NCH; ++j)
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) eq[j][e] = 0.0f;
+                        for (int e = 0; e < 4; ++e) eq[j][e] = splat(0.0f);
                     kt = 1.0f;
                     scale_w = 0.0f;
                     scale_d = kappa * fp;
