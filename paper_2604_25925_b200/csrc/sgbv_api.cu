@@ -92,7 +92,7 @@ int grow(void **ptr, size_t *have, size_t need) {
 
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
-int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0;
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_occupancy = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -285,10 +285,13 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;
         g_opt_max_clusters = value;
+    } else if (!strcmp(name, "occupancy")) {
+        if (value != 0 && (value < 2 || value > 4)) return SGBV_ERR_SHAPE;
+        g_opt_occupancy = value;
     } else {
         return SGBV_ERR_SHAPE;
     }
-    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters);
+    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_occupancy);
     return SGBV_OK;
 }
 

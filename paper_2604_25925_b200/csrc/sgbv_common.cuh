@@ -132,6 +132,6 @@ bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0
 int launch_fused(const Launch &L, int *error_flag);
-void fused_set_options(int cluster, int stages, int max_clusters);
+void fused_set_options(int cluster, int stages, int max_clusters, int occupancy);
 
 }  // namespace sgbv

@@ -10,10 +10,11 @@
 //   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
 //     exponentials relative to the thread's own maximum, so the second
 //     sweep of the coupling sum never re-reads memory;
-//   * exchanges per-warp (max, sum-exp) partials by PUSHING them into every CTA's shared
-//     memory with asynchronous distributed-shared-memory stores that complete on the receiver's
-//     mbarrier; a warp goes on as soon as all partials of the row have landed.  There is no
-//     block-wide or cluster-wide barrier inside the row loop;
+//   * exchanges (max, sum-exp) partials in two levels: the warps of a CTA leave theirs in shared
+//     memory and the last one to arrive combines them and PUSHES one partial per CTA into every
+//     CTA's shared memory with asynchronous distributed-shared-memory stores that complete on the
+//     receiver's mbarrier; a warp goes on as soon as all CTA partials of the row have landed.
+//     There is no block-wide or cluster-wide barrier inside the row loop;
 //   * runs the second sweep from registers and writes one partial sum per cell.
 // The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread per
 // CTA, which computes c_{i+1} after its warp has pushed its partials of row i+1, i.e. while the
@@ -124,9 +125,11 @@ struct Control {
     uint64_t full[kMaxStages];           // per ring stage: "both chunks have landed"
     int readers_done[kMaxStages];        // per ring stage: warps that have finished reading it
     uint64_t xbar[2];                    // by row parity: "all partials of the row and c_i are here"
-    // per-warp partials (maximum of zq, sum eq, maximum of zp, sum ep) of every
-    // CTA of the cluster, pushed by their owners; double-buffered by row parity
-    float4 slots[2][kMaxCluster * kFWarps];
+    // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
+    // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
+    float4 wslots[2][kFWarps];
+    int warps_in[2];                     // warps of this CTA whose partial of the row is in wslots
+    float4 slots[2][kMaxCluster];
     double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
 };
 
@@ -312,8 +315,10 @@ __device__ __forceinline__ void sweep_two_dispatch(const float2 (&eq)[NCH][4], c
 #undef SGBV_SWEEP
 }
 
-template <typename T, int NCH>
-__global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedParams p) {
+// OCC = CTAs of this kernel that share an SM (2, 3 or 4): more co-resident CTAs hide more of each
+// other's exchange and pipeline latency, but leave each thread fewer registers, hence fewer cells.
+template <typename T, int NCH, int OCC>
+__global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const FusedParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -345,6 +350,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
         }
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
+        ctl->warps_in[0] = ctl->warps_in[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -354,7 +360,7 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
     const int my_chains = (p.nchains - cid + G - 1) / G;
     const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
     const int total_loads = nrows * nchunks;    // chunk pairs this CTA loads
-    const uint32_t xbytes = (uint32_t)(C * kFWarps * sizeof(float4));
+    const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
     bool timed_out = false;
 
     // Producer state, kept identically by lane 0 of every warp: loads are issued in consumption
@@ -497,9 +503,25 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
             sq = warp_sum(has_q ? sq * ex2((bq - rqw) * s.scale) : 0.0f);
             sp = warp_sum(has_p ? sp * ex2((bp - rpw) * s.scale) : 0.0f);
-            if (lane < C)
-                push_f4(&ctl->slots[par][rank * kFWarps + warp], &ctl->xbar[par], (uint32_t)lane,
-                        make_float4(bqw, sq, bpw, sp));
+            // two-level exchange: the warp partials meet in this CTA's shared memory; the warp that
+            // arrives last combines them (fixed order) and pushes ONE partial per CTA to every CTA
+            bool last_warp = false;
+            if (lane == 0) {
+                ctl->wslots[par][warp] = make_float4(bqw, sq, bpw, sp);
+                __threadfence_block();
+                last_warp = atomicAdd(&ctl->warps_in[par], 1) == kFWarps - 1;
+            }
+            if (__shfl_sync(0xffffffffu, last_warp, 0)) {
+                __threadfence_block();
+                if (lane == 0) ctl->warps_in[par] = 0;
+                const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+                const float mqc = warp_max(v.x), mpc = warp_max(v.z);
+                const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
+                const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
+                const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
+                if (lane < C)
+                    push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
+            }
 
             if (tid == 0) {
                 // c_i = c_{i-1} p_{i-1}(tok)/q_{i-1}(tok) from the previous row's statistics; c_0 = 1
@@ -517,25 +539,12 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
             }
             if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
 
-            // ---- row statistics: every warp combines all partials, in the same order ------------------
-            float bq_row = -INFINITY, bp_row = -INFINITY;
-            const int nslots = C * kFWarps;
-            for (int e = lane; e < nslots; e += 32) {
-                const float4 v = ctl->slots[par][e];
-                bq_row = fmaxf(bq_row, v.x);
-                bp_row = fmaxf(bp_row, v.z);
-            }
-            bq_row = warp_max(bq_row);
-            bp_row = warp_max(bp_row);
+            // ---- row statistics: every warp combines the CTA partials, in the same order -------------
+            const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+            const float bq_row = warp_max(cv.x), bp_row = warp_max(cv.z);
             const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
-            float Zq = 0.0f, Zp = 0.0f;
-            for (int e = lane; e < nslots; e += 32) {
-                const float4 v = ctl->slots[par][e];
-                if (v.x > -INFINITY) Zq = fmaf(v.y, ex2((v.x - rq_row) * s.scale), Zq);
-                if (v.z > -INFINITY) Zp = fmaf(v.w, ex2((v.z - rp_row) * s.scale), Zp);
-            }
-            Zq = warp_sum(Zq);
-            Zp = warp_sum(Zp);
+            const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
+            const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
             const double cd = ctl->c[par];
             const float c = (float)cd;
             const float kappa = (float)(cd * (double)(Zq / Zp));
@@ -597,30 +606,33 @@ __global__ void __launch_bounds__(kFThreads, 2) fused_chain_kernel(const FusedPa
 
 // ---- host side ----------------------------------------------------------------------------------------
 struct Plan {
-    int cluster, slice_len, nch, stages, grid_clusters;
+    int cluster, slice_len, nch, occ, stages, grid_clusters;
     size_t smem;
 };
 
 int g_opt_cluster = 0;     // 0 = automatic
 int g_opt_stages = 0;
 int g_opt_max_clusters = 0;
+int g_opt_occupancy = 0;
 
 constexpr int kSmemPerSm = 228 * 1024;     // shared memory of one SM
 constexpr int kSmemReserved = 1024;        // per resident CTA, taken by the system
-constexpr int kCtaSlots = 2 * 148;         // resident CTAs of this kernel on the whole device
+constexpr int kSms = 148;
+// cells per warp that fit the registers when OCC CTAs share an SM
+int max_nch(int occ) { return occ <= 2 ? kMaxNch : occ == 3 ? 2 : 1; }
 
 int cells_of(int V) { return (V + kCell - 1) / kCell; }
 int slice_cells(int cells, int C) { return (cells + C - 1) / C; }
 
-template <typename T, int NCH>
+template <typename T, int NCH, int OCC>
 int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
-    auto kernel = fused_chain_kernel<T, NCH>;
+    auto kernel = fused_chain_kernel<T, NCH, OCC>;
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGBV_ERR_CUDA;
     if (!attr_done[dev]) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemPerSm / 2 - kSmemReserved) != cudaSuccess)
+                                 kSmemPerSm / OCC - kSmemReserved) != cudaSuccess)
             return SGBV_ERR_CUDA;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
             return SGBV_ERR_CUDA;
@@ -656,7 +668,7 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
         static int cached[64][kMaxCluster + 1][kMaxStages + 1];  // [device][cluster size][stages]
         int &slot = cached[dev][plan.cluster][plan.stages];
         if (slot == 0) {
-            cfg.gridDim = dim3(plan.cluster * (kCtaSlots / plan.cluster));
+            cfg.gridDim = dim3(plan.cluster * (OCC * kSms / plan.cluster));
             int nmax = 0;
             if (cudaOccupancyMaxActiveClusters(&nmax, kernel, &cfg) != cudaSuccess || nmax < 1) {
                 cudaGetLastError();
@@ -680,22 +692,26 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
 
 template <typename T>
 int launch_t(const Launch &L, const Plan &plan, int *error_flag) {
-    switch (plan.nch) {
-        case 1: return launch_nch<T, 1>(L, plan, error_flag);
-        case 2: return launch_nch<T, 2>(L, plan, error_flag);
-        case 3: return launch_nch<T, 3>(L, plan, error_flag);
-        case 4: return launch_nch<T, 4>(L, plan, error_flag);
-        case 5: return launch_nch<T, 5>(L, plan, error_flag);
+    switch (plan.occ * 10 + plan.nch) {
+        case 21: return launch_nch<T, 1, 2>(L, plan, error_flag);
+        case 22: return launch_nch<T, 2, 2>(L, plan, error_flag);
+        case 23: return launch_nch<T, 3, 2>(L, plan, error_flag);
+        case 24: return launch_nch<T, 4, 2>(L, plan, error_flag);
+        case 25: return launch_nch<T, 5, 2>(L, plan, error_flag);
+        case 31: return launch_nch<T, 1, 3>(L, plan, error_flag);
+        case 32: return launch_nch<T, 2, 3>(L, plan, error_flag);
+        case 41: return launch_nch<T, 1, 4>(L, plan, error_flag);
         default: return SGBV_ERR_SHAPE;
     }
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int stages, int max_clusters) {
+void fused_set_options(int cluster, int stages, int max_clusters, int occupancy) {
     g_opt_cluster = cluster;
     g_opt_stages = stages;
     g_opt_max_clusters = max_clusters;
+    g_opt_occupancy = occupancy;
 }
 
 // Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and
@@ -712,20 +728,24 @@ int launch_fused(const Launch &L, int *error_flag) {
     const int cells = cells_of(s.V);
     const long nchains = (long)s.B * s.K;
     Plan plan;
+    const int occ = g_opt_occupancy ? g_opt_occupancy : 2;
+    const int cap = max_nch(occ) * kChunk;  // elements of a row one CTA can hold
+    const long cta_slots = (long)occ * kSms;
     int C = g_opt_cluster;
     if (C == 0) {
         C = 1;
-        while (slice_cells(cells, C) * kCell > kMaxNch * kChunk) C *= 2;  // smallest cluster whose slices fit
+        while (C < kMaxCluster && slice_cells(cells, C) * kCell > cap) C *= 2;  // smallest cluster whose slices fit
         // few chains: spread each over more CTAs while they all stay co-resident in one wave
-        while (C < kMaxCluster && nchains * 2 * C <= kCtaSlots && cells / (2 * C) >= 4) C *= 2;
+        while (C < kMaxCluster && nchains * 2 * C <= cta_slots && cells / (2 * C) >= 4) C *= 2;
     }
-    if (C < 1 || C > kMaxCluster || slice_cells(cells, C) * kCell > kMaxNch * kChunk) return SGBV_ERR_SHAPE;
+    if (C < 1 || C > kMaxCluster || slice_cells(cells, C) * kCell > cap) return g_opt_occupancy ? SGBV_ERR_SHAPE : 0;
     plan.cluster = C;
+    plan.occ = occ;
     plan.slice_len = slice_cells(cells, C) * kCell;
     plan.nch = (plan.slice_len + kChunk - 1) / kChunk;
     const size_t stage_bytes = 2 * kChunk * esz;
     int S = g_opt_stages ? g_opt_stages : kMaxStages;
-    const size_t budget = kSmemPerSm / 2 - kSmemReserved - sizeof(Control);
+    const size_t budget = kSmemPerSm / occ - kSmemReserved - sizeof(Control);
     if ((size_t)S * stage_bytes > budget) S = (int)(budget / stage_bytes);
     if (S > kMaxStages) S = kMaxStages;
     if (S < 2) return SGBV_ERR_SHAPE;
