@@ -4,9 +4,10 @@
 //   * streams the target row and the draft row from HBM exactly once: bulk asynchronous copies
 //     (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks of both tensors into a
 //     shared-memory ring that runs ahead across rows and chains.  A warp owns the 256-element
-//     cells  warp, warp+8, warp+16, ...  of its CTA's slice.  There is no producer thread: the
-//     warp that is LAST to finish reading a ring stage refills it, so no warp waits for another
-//     one to release a stage, and the copies stay large (few requests to the copy engine);
+//     cells  warp, warp+8, warp+16, ...  of its CTA's slice.  There is no producer thread and no
+//     "stage free" barrier: the warp that arrives last in the row's exchange (below) knows that
+//     every warp of its CTA has moved the row into registers, and refills the row's ring stages
+//     then, one lane per chunk, so the copies stay large (few requests to the copy engine);
 //   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
 //     exponentials relative to the thread's own maximum, so the second
 //     sweep of the coupling sum never re-reads memory;
@@ -123,7 +124,6 @@ __device__ __forceinline__ float rcp(float x) {
 // [ring: stages x (chunk of zq, chunk of zp)] [Control]
 struct Control {
     uint64_t full[kMaxStages];           // per ring stage: "both chunks have landed"
-    int readers_done[kMaxStages];        // per ring stage: warps that have finished reading it
     uint64_t xbar[2];                    // by row parity: "all partials of the row and c_i are here"
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
     // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
@@ -344,10 +344,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     const int x_warp = x_begin + warp * kCell;  // first element of this warp's first cell
 
     if (tid == 0) {
-        for (int i = 0; i < S; ++i) {
-            mbar_init(&ctl->full[i], 1);
-            ctl->readers_done[i] = 0;
-        }
+        for (int i = 0; i < S; ++i) mbar_init(&ctl->full[i], 1);
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
         ctl->warps_in[0] = ctl->warps_in[1] = 0;
@@ -363,38 +360,24 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
     bool timed_out = false;
 
-    // Producer state, kept identically by lane 0 of every warp: loads are issued in consumption
-    // order; (p_bk, p_i, p_j, p_st) describe the next one: chain, position, chunk, ring stage.
-    // advance_producer(true) issues it, advance_producer(false) only steps the state (another
-    // warp issues that load).
-    int p_j = 0, p_st = 0, p_issued = 0;
-    size_t p_bk = (size_t)cid;
-    int p_i = 0;
-    auto advance_producer = [&](bool issue) {
-        if (issue) {
-            const int x0 = x_begin + p_j * kChunk;  // first element of the chunk
-            const T *zq = reinterpret_cast<const T *>(p.zq) + (p_bk * (s.gamma + 1) + p_i) * s.V + x0;
-            const T *zp = reinterpret_cast<const T *>(p.zp) + (p_bk * s.gamma + p_i) * s.V + x0;
-            const uint32_t bytes = (uint32_t)min(kChunk, cta_len - p_j * kChunk) * (uint32_t)sizeof(T);
-            unsigned char *dst = ring + (size_t)p_st * kStageBytes;
-            mbar_expect_tx(&full[p_st], 2 * bytes);
-            bulk_load(dst, zq, bytes, &full[p_st]);
-            bulk_load(dst + kChunkBytes, zp, bytes, &full[p_st]);
-        }
-        ++p_issued;
-        if (++p_st == S) p_st = 0;
-        if (++p_j == nchunks) {
-            p_j = 0;
-            if (++p_i == s.gamma) {
-                p_i = 0;
-                p_bk += G;
-            }
-        }
+    // Loads are numbered in consumption order: chunk m of this CTA's walk is chunk m % nchunks of
+    // row m / nchunks and lands in ring stage m % S.  issue_chunk is stateless, so any lane can issue
+    // any chunk: lanes of one warp issue the chunks of a whole row side by side.
+    auto issue_chunk = [&](int m) {
+        const int row = m / nchunks, jc = m - row * nchunks;
+        const int chain = row / s.gamma, pos = row - chain * s.gamma;
+        const size_t bkc = (size_t)cid + (size_t)chain * G;
+        const int x0 = x_begin + jc * kChunk;  // first element of the chunk
+        const T *zq = reinterpret_cast<const T *>(p.zq) + (bkc * (s.gamma + 1) + pos) * s.V + x0;
+        const T *zp = reinterpret_cast<const T *>(p.zp) + (bkc * s.gamma + pos) * s.V + x0;
+        const uint32_t bytes = (uint32_t)min(kChunk, cta_len - jc * kChunk) * (uint32_t)sizeof(T);
+        const int stage = m % S;
+        unsigned char *dst = ring + (size_t)stage * kStageBytes;
+        mbar_expect_tx(&full[stage], 2 * bytes);
+        bulk_load(dst, zq, bytes, &full[stage]);
+        bulk_load(dst + kChunkBytes, zp, bytes, &full[stage]);
     };
-    if (lane == 0) {
-        const int first = total_loads < S ? total_loads : S;
-        for (int k = 0; k < first; ++k) advance_producer(warp == 0);  // warp 0 issues the first S loads
-    }
+    if (warp == 0 && lane < S && lane < total_loads) issue_chunk(lane);  // fill the ring
 
     // The chain thread of this CTA (thread 0) carries c_i and fetches the token logits one row
     // ahead: tok_next is the token of the next row of the walk.
@@ -435,12 +418,37 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
             float2 eq[NCH][4], ep[NCH][4];  // two neighbouring vocabulary entries per register pair
             float mq = -INFINITY, mp = -INFINITY;
+            {
+                // all stages of the row are tested at once (one shared-memory round trip when the data
+                // is there, which is the normal case); only a stage that is late is waited for
+                bool ready = true;
+                int stj = st;
+                uint32_t phj = ph;
+#pragma unroll
+                for (int j = 0; j < NCH; ++j) {
+                    if (j < nchunks) {
+                        ready &= mbar_test(&full[stj], phj);
+                        if (++stj == S) {
+                            stj = 0;
+                            phj ^= 1u;
+                        }
+                    }
+                }
+                if (!ready) {
+                    stj = st;
+                    phj = ph;
+                    for (int j = 0; j < nchunks; ++j) {
+                        if (!mbar_wait(&full[stj], phj)) timed_out = true;
+                        if (++stj == S) {
+                            stj = 0;
+                            phj ^= 1u;
+                        }
+                    }
+                }
+            }
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 if (j < nchunks) {  // uniform over the CTA
-                    // every warp waits, also one without a cell in this chunk: it must not count
-                    // itself done with the stage's next use before this use has been refilled
-                    if (!mbar_wait(&full[st], ph)) timed_out = true;
                     if (j < nj) {  // warp-uniform
                         const unsigned char *base = ring + (size_t)st * kStageBytes + warp * kCellBytes;
                         read_cell<T>(base, lane, eq[j]);
@@ -453,15 +461,6 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                                 if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[j][e].y = ep[j][e].y = -INFINITY;
                             }
                         }
-                    }
-                    __syncwarp();
-                    if (lane == 0) {
-                        // the last warp to finish with this stage refills it with the chunk S ahead
-                        const bool last = atomicAdd(&ctl->readers_done[st], 1) == kFWarps - 1;
-                        if (last) ctl->readers_done[st] = 0;
-                        if (p_issued < total_loads) advance_producer(last);
-                    }
-                    if (j < nj) {
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             mq = max3(mq, eq[j][e].x, eq[j][e].y);
@@ -514,6 +513,12 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             if (__shfl_sync(0xffffffffu, last_warp, 0)) {
                 __threadfence_block();
                 if (lane == 0) ctl->warps_in[par] = 0;
+                // every warp of this CTA has turned this row's ring stages into registers: refill
+                // them with the chunks S ahead (one lane per chunk)
+                if (lane < nchunks) {
+                    const int m = n * nchunks + lane + S;
+                    if (m < total_loads) issue_chunk(m);
+                }
                 const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
                 const float mqc = warp_max(v.x), mpc = warp_max(v.z);
                 const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
