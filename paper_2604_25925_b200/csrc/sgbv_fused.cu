@@ -18,8 +18,8 @@
 //     There is no block-wide or cluster-wide barrier inside the row loop;
 //   * runs the second sweep from registers and writes one partial sum per cell.
 // The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread per
-// CTA, which computes c_{i+1} after its warp has pushed its partials of row i+1, i.e. while the
-// exchange is in flight.  Two CTAs of 256 threads share an SM (different clusters).  The finishing
+// CTA, which computes c_{i+1} right after the statistics of row i and arms the next row's exchange
+// with it, a whole row before it is needed.  Two CTAs of 256 threads share an SM (different clusters).  The finishing
 // kernel (weights, scan, extra token) consumes the cell sums.
 //
 // Every wait on an mbarrier is bounded; on expiry the warp records an error flag and keeps
@@ -158,6 +158,36 @@ __device__ __forceinline__ int cell_offset(int lane, int e) {
     return lane * 8 + e;
 }
 
+// Maximum over the warp in one instruction (NaN inputs are passed over, as fmaxf does).
+__device__ __forceinline__ float warp_max_redux(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// 2^x in double precision: x = n + f with |f| <= 1/2, e^(f ln 2) by its Taylor series to degree 13
+// (remainder below 1e-17), scaled by 2^n.  A short dependent chain, unlike the library routine's.
+__device__ __forceinline__ double exp2_short(double x) {
+    if (x != x) return x;
+    if (x < -1100.0) return 0.0;
+    if (x > 1100.0) return INFINITY;
+    const double n = rint(x);
+    const double t = (x - n) * 0.6931471805599453094;
+    double pl = 1.0 / 6227020800.0;
+    pl = fma(pl, t, 1.0 / 479001600.0);
+    pl = fma(pl, t, 1.0 / 39916800.0);
+    pl = fma(pl, t, 1.0 / 3628800.0);
+    pl = fma(pl, t, 1.0 / 362880.0);
+    pl = fma(pl, t, 1.0 / 40320.0);
+    pl = fma(pl, t, 1.0 / 5040.0);
+    pl = fma(pl, t, 1.0 / 720.0);
+    pl = fma(pl, t, 1.0 / 120.0);
+    pl = fma(pl, t, 1.0 / 24.0);
+    pl = fma(pl, t, 1.0 / 6.0);
+    pl = fma(pl, t, 0.5);
+    pl = fma(pl, t, 1.0);
+    pl = fma(pl, t, 1.0);
+    return scalbn(pl, (int)n);
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -383,9 +413,10 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     // ahead: tok_next is the token of the next row of the walk.
     int tok_next = 0;
     if (tid == 0 && nrows > 0) tok_next = p.tok[(size_t)cid * s.gamma];
-    double c_run = 1.0;                 // c of the row being processed (chain thread)
-    float zq_tok = 0.0f, zp_tok = 0.0f;  // token logits of the previous row, and its statistics
-    float prev_bq = 0.0f, prev_bp = 0.0f, prev_Zq = 1.0f, prev_Zp = 1.0f;
+    if (tid == 0 && nrows > 0) {  // the first row of the walk starts a chain: c_0 = 1
+        ctl->c[0] = 1.0;
+        mbar_expect_tx(&ctl->xbar[0], xbytes);
+    }
 
     int st = 0;
     uint32_t ph = 0;
@@ -398,16 +429,16 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             const int par = n & 1;
             const uint32_t xph = (uint32_t)(n >> 1) & 1u;
 
-            // ---- chain thread: c_i from the previous row, then the token logits of this row ----------
-            float zq_tok_new = 0.0f, zp_tok_new = 0.0f;
+            // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
+            float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
             if (tid == 0) {
                 int t = tok_next;
                 if (t < 0 || t >= s.V) {
                     if (rank == 0) atomicOr(p.ws.status + brow, SGBV_STATUS_TOKEN_RANGE);
                     t = 0;
                 }
-                zq_tok_new = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
-                zp_tok_new = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
+                zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
+                zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
                 if (n + 1 < nrows) {
                     const size_t bk_n = (i + 1 < s.gamma) ? bk : bk + G;
                     const int i_n = (i + 1 < s.gamma) ? i + 1 : 0;
@@ -498,7 +529,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             }
             float sq = sq2.x + sq2.y, sp = sp2.x + sp2.y;
             // warp partials relative to the warp's maxima, pushed to every CTA
-            const float bqw = warp_max(has_q ? bq : -INFINITY), bpw = warp_max(has_p ? bp : -INFINITY);
+            const float bqw = warp_max_redux(has_q ? bq : -INFINITY), bpw = warp_max_redux(has_p ? bp : -INFINITY);
             const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
             sq = warp_sum(has_q ? sq * ex2((bq - rqw) * s.scale) : 0.0f);
             sp = warp_sum(has_p ? sp * ex2((bp - rpw) * s.scale) : 0.0f);
@@ -513,40 +544,26 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             if (__shfl_sync(0xffffffffu, last_warp, 0)) {
                 __threadfence_block();
                 if (lane == 0) ctl->warps_in[par] = 0;
+                const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+                const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
+                const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
+                const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
+                const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
+                if (lane < C)
+                    push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
                 // every warp of this CTA has turned this row's ring stages into registers: refill
                 // them with the chunks S ahead (one lane per chunk)
                 if (lane < nchunks) {
                     const int m = n * nchunks + lane + S;
                     if (m < total_loads) issue_chunk(m);
                 }
-                const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-                const float mqc = warp_max(v.x), mpc = warp_max(v.z);
-                const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
-                const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
-                const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
-                if (lane < C)
-                    push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
             }
 
-            if (tid == 0) {
-                // c_i = c_{i-1} p_{i-1}(tok)/q_{i-1}(tok) from the previous row's statistics; c_0 = 1
-                if (i > 0) {
-                    const double lp = ((double)zp_tok - (double)prev_bp) * (double)s.scale;
-                    const double lq = ((double)zq_tok - (double)prev_bq) * (double)s.scale;
-                    c_run *= exp2(lp - lq) * ((double)prev_Zq / (double)prev_Zp);
-                } else {
-                    c_run = 1.0;
-                }
-                ctl->c[par] = c_run;
-                mbar_expect_tx(&ctl->xbar[par], xbytes);  // arms the exchange and publishes c_i
-                zq_tok = zq_tok_new;
-                zp_tok = zp_tok_new;
-            }
             if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
 
             // ---- row statistics: every warp combines the CTA partials, in the same order -------------
             const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-            const float bq_row = warp_max(cv.x), bp_row = warp_max(cv.z);
+            const float bq_row = warp_max_redux(cv.x), bp_row = warp_max_redux(cv.z);
             const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
             const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
             const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
@@ -555,10 +572,18 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             const float kappa = (float)(cd * (double)(Zq / Zp));
 
             if (tid == 0) {
-                prev_bq = rq_row;
-                prev_bp = rp_row;
-                prev_Zq = Zq;
-                prev_Zp = Zp;
+                // c of the next row of the walk: c_{i+1} = c_i p_i(tok_i)/q_i(tok_i), or 1 at the start
+                // of the next chain; publishing it arms the next row's exchange
+                if (n + 1 < nrows) {
+                    double c_next = 1.0;
+                    if (i + 1 < s.gamma) {
+                        const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
+                        const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
+                        c_next = cd * exp2_short(lp - lq) * (double)(Zq / Zp);
+                    }
+                    ctl->c[par ^ 1] = c_next;
+                    mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
+                }
                 if (rank == 0) {
                     // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
                     // -inf only has Z = 0
