@@ -5,9 +5,9 @@
 //     (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks of both tensors into a
 //     shared-memory ring that runs ahead across rows and chains.  A warp owns the 256-element
 //     cells  warp, warp+8, warp+16, ...  of its CTA's slice.  There is no producer thread and no
-//     "stage free" barrier: the warp that arrives last in the row's exchange (below) knows that
-//     every warp of its CTA has moved the row into registers, and refills the row's ring stages
-//     then, one lane per chunk, so the copies stay large (few requests to the copy engine);
+//     "stage free" barrier: once the row's exchange (below) is complete, every warp of the CTA has
+//     moved the row into registers, so its ring stages are refilled right then, by a different warp
+//     for each chunk; the copies stay large (few requests to the copy engine);
 //   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
 //     exponentials relative to the thread's own maximum, so the second
 //     sweep of the coupling sum never re-reads memory;
@@ -186,7 +186,10 @@ __device__ __forceinline__ double exp2_short(double x) {
     pl = fma(pl, t, 0.5);
     pl = fma(pl, t, 1.0);
     pl = fma(pl, t, 1.0);
-    return scalbn(pl, (int)n);
+    // 2^n built from its bit pattern where it is a normal number, else the library's scaling
+    const int ni = (int)n;
+    if (ni > -1000 && ni < 1000) return pl * __longlong_as_double((long long)(ni + 1023) << 52);
+    return scalbn(pl, ni);
 }
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
@@ -409,11 +412,12 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     };
     if (warp == 0 && lane < S && lane < total_loads) issue_chunk(lane);  // fill the ring
 
-    // The chain thread of this CTA (thread 0) carries c_i and fetches the token logits one row
+    // The chain thread of this CTA carries c_i and fetches the token logits one row
     // ahead: tok_next is the token of the next row of the walk.
+    const bool chain_thread = tid == kFThreads - 32;  // lane 0 of the last warp; thread 0 writes the row records
     int tok_next = 0;
-    if (tid == 0 && nrows > 0) tok_next = p.tok[(size_t)cid * s.gamma];
-    if (tid == 0 && nrows > 0) {  // the first row of the walk starts a chain: c_0 = 1
+    if (chain_thread && nrows > 0) tok_next = p.tok[(size_t)cid * s.gamma];
+    if (chain_thread && nrows > 0) {  // the first row of the walk starts a chain: c_0 = 1
         ctl->c[0] = 1.0;
         mbar_expect_tx(&ctl->xbar[0], xbytes);
     }
@@ -431,7 +435,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
 
             // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
             float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
-            if (tid == 0) {
+            if (chain_thread) {
                 int t = tok_next;
                 if (t < 0 || t >= s.V) {
                     if (rank == 0) atomicOr(p.ws.status + brow, SGBV_STATUS_TOKEN_RANGE);
@@ -551,15 +555,20 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                 const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
                 if (lane < C)
                     push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
-                // every warp of this CTA has turned this row's ring stages into registers: refill
-                // them with the chunks S ahead (one lane per chunk)
-                if (lane < nchunks) {
-                    const int m = n * nchunks + lane + S;
-                    if (m < total_loads) issue_chunk(m);
-                }
             }
 
             if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
+
+            // The exchange is complete, so every warp of this CTA has turned this row's ring stages into
+            // registers: refill them with the chunks S ahead.  Warps 1, 2, ... take one chunk each (the
+            // chain thread's warp 0 has enough to do), so the copy requests are issued side by side.
+            {
+                const int jc = (warp + kFWarps - 1) % kFWarps;  // warp 1 -> chunk 0, ..., warp 0 -> chunk 7
+                if (lane == 0 && jc < nchunks) {
+                    const int m = n * nchunks + jc + S;
+                    if (m < total_loads) issue_chunk(m);
+                }
+            }
 
             // ---- row statistics: every warp combines the CTA partials, in the same order -------------
             const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
@@ -571,10 +580,10 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             const float c = (float)cd;
             const float kappa = (float)(cd * (double)(Zq / Zp));
 
-            if (tid == 0) {
+            if (chain_thread && n + 1 < nrows) {
                 // c of the next row of the walk: c_{i+1} = c_i p_i(tok_i)/q_i(tok_i), or 1 at the start
                 // of the next chain; publishing it arms the next row's exchange
-                if (n + 1 < nrows) {
+                {
                     double c_next = 1.0;
                     if (i + 1 < s.gamma) {
                         const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
@@ -584,6 +593,8 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     ctl->c[par ^ 1] = c_next;
                     mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
                 }
+            }
+            if (tid == 0) {
                 if (rank == 0) {
                     // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
                     // -inf only has Z = 0
