@@ -36,7 +36,7 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
 }
 
 struct Carve {
-    size_t rows, part, wpart, dpart, mpart, h, resmass, status, error, total;
+    size_t rows, part, wpart, dpart, mpart, bonus, h, resmass, status, error, total;
 };
 
 Carve carve(const Shape &s) {
@@ -48,6 +48,7 @@ Carve carve(const Shape &s) {
     c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.mpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.bonus = off;     off += align_up((size_t)s.B * 2 * s.ntiles * sizeof(float));
     c.h = off;         off += align_up(NR * sizeof(double));
     c.resmass = off;   off += align_up(NR * sizeof(double));
     c.status = off;    off += align_up((size_t)s.B * sizeof(int32_t));
@@ -137,6 +138,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     L.ws.wpart = (float *)(base + c.wpart);
     L.ws.dpart = (float *)(base + c.dpart);
     L.ws.mpart = (float *)(base + c.mpart);
+    L.ws.bonus = (float *)(base + c.bonus);
     L.ws.h = out_h ? out_h : (double *)(base + c.h);
     L.ws.resmass = out_resmass ? out_resmass : (double *)(base + c.resmass);
     L.ws.status = out_status ? out_status : (int32_t *)(base + c.status);
@@ -156,14 +158,18 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         L.ev_end = g_prof.end[g_prof.used];
         ++g_prof.used;
     }
-    if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
-    if (cudaMemsetAsync(L.ws.error, 0, sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+    // the fused kernel needs nothing cleared: it reports through the row records and zeroes the
+    // error word itself; the two-sweep kernels set status bits with atomics, so those start at zero
     bool fused = g_opt_path != 1 && fused_supported(L);
+    L.ws.prestatus = nullptr;
     int n1 = fused ? launch_fused(L, L.ws.error) : 0;
     if (n1 < 0) return n1;
     if (n1 == 0) {
         if (g_opt_path == 2) return SGBV_ERR_SHAPE;
         fused = false;
+        L.ws.prestatus = L.ws.status;
+        if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+        if (cudaMemsetAsync(L.ws.error, 0, sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
         n1 = launch_twopass(L);
         if (n1 < 0) return n1;
     }

@@ -26,6 +26,8 @@ struct RowInfo {
     float kappa;    // c * Zq / Zp with c = b/a: ratio c*p(x)/q(x) = kappa * ep/eq in row-max units
     float c;        // c = p(x_k^i)/q(x_k^i), ratio of the joint prefix probabilities (c < 1 selects
                     // the cancellation-free numerator)
+    int32_t flags;  // SGBV_STATUS_NONFINITE_LOGIT if the streaming pass found the row pair unusable
+    int32_t pad_;
 };
 
 struct Workspace {
@@ -34,9 +36,12 @@ struct Workspace {
     float *wpart;       // [B*K*gamma][ntiles]: sum over the tile of eq * max(1 - kappa ep/eq, 0)^K
     float *dpart;       // [B*K*gamma][ntiles]: sum of max(kappa ep - eq, 0)               (c < 1)
     float *mpart;       // [B*K*gamma][ntiles]: sum of eq (c - t)^2 Q(t)                    (c < 1)
+    float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     double *h;          // [B][K][gamma]
     double *resmass;    // [B][K][gamma]
-    int32_t *status;    // [B]
+    int32_t *status;    // [B]: final per-row status, written by the finishing kernel
+    int32_t *prestatus; // [B] bits set by earlier kernels with atomics (zeroed first), or NULL when the
+                        // streaming pass reports through RowInfo::flags instead
     int32_t *error;     // [1]: set when a bounded device-side wait expired
 };
 
@@ -92,6 +97,36 @@ __device__ __forceinline__ void element_terms(float eq, float ep, float kappa, f
         m2 = eq * ct * ct * acc;
     }
 }
+
+// 2^x in double precision: x = n + f with |f| <= 1/2, e^(f ln 2) by its Taylor series to degree 13
+// (remainder below 1e-17), scaled by 2^n.  A short dependent chain, unlike the library routine's.
+__device__ __forceinline__ double exp2_short(double x) {
+    if (x != x) return x;
+    if (x < -1100.0) return 0.0;
+    if (x > 1100.0) return INFINITY;
+    const double n = rint(x);
+    const double t = (x - n) * 0.6931471805599453094;
+    double pl = 1.0 / 6227020800.0;
+    pl = fma(pl, t, 1.0 / 479001600.0);
+    pl = fma(pl, t, 1.0 / 39916800.0);
+    pl = fma(pl, t, 1.0 / 3628800.0);
+    pl = fma(pl, t, 1.0 / 362880.0);
+    pl = fma(pl, t, 1.0 / 40320.0);
+    pl = fma(pl, t, 1.0 / 5040.0);
+    pl = fma(pl, t, 1.0 / 720.0);
+    pl = fma(pl, t, 1.0 / 120.0);
+    pl = fma(pl, t, 1.0 / 24.0);
+    pl = fma(pl, t, 1.0 / 6.0);
+    pl = fma(pl, t, 0.5);
+    pl = fma(pl, t, 1.0);
+    pl = fma(pl, t, 1.0);
+    // 2^n built from its bit pattern where it is a normal number, else the library's scaling
+    const int ni = (int)n;
+    if (ni > -1000 && ni < 1000) return pl * __longlong_as_double((long long)(ni + 1023) << 52);
+    return scalbn(pl, ni);
+}
+// e^x through the same short chain.
+__device__ __forceinline__ double exp_short(double x) { return exp2_short(x * 1.4426950408889634074); }
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

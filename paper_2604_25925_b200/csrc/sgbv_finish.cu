@@ -19,10 +19,15 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kEpt = kTile / kThreads;  // elements per thread inside one tile
 static_assert(kEpt >= 1 && kEpt * kThreads == kTile, "a tile is a whole number of elements per thread");
 
-__device__ __forceinline__ double gfun(double u, int K) {  // 1 - (1-u)^K
+// 1 - (1-u)^K as the geometric sum u (1 + (1-u) + ... + (1-u)^(K-1)): all terms are positive, so
+// a tiny u keeps its full relative accuracy, and no transcendental function is needed.
+__device__ __forceinline__ double gfun(double u, int K) {
     if (u >= 1.0) return 1.0;
     if (!(u > 0.0)) return 0.0;
-    return -expm1((double)K * log1p(-u));
+    const double v = 1.0 - u;
+    double sum = 1.0;
+    for (int j = 1; j < K; ++j) sum = fma(sum, v, 1.0);
+    return u * sum;
 }
 
 __device__ __forceinline__ double clamp01(double x) {
@@ -36,7 +41,7 @@ __device__ __forceinline__ double clamp01(double x) {
 //               = M + K (1-c)^(K-1) Dp               (c <  1; equals R - (1-c)^K term by term)
 // denominator/a = numerator/a + g(b)/a - g(min(c,1))
 __device__ double weight_sub(double la, double lb, double R, double Dp, double M, int K, bool below_one) {
-    const double a = exp(la), b = exp(lb), c = exp(lb - la);
+    const double a = exp_short(la), b = exp_short(lb), c = exp_short(lb - la);
     const double gb = gfun(b, K);
     if (!(a > 0.0)) return gb > 0.0 ? 0.0 : 1.0;
     double num, extra;
@@ -57,8 +62,8 @@ __device__ double weight_sub(double la, double lb, double R, double Dp, double M
 
 // Eq. 3.
 __device__ double weight_full(double la, double lb, int K) {
-    const double a = exp(la), b = exp(lb);
-    double c = exp(lb - la);
+    const double a = exp_short(la), b = exp_short(lb);
+    double c = exp_short(lb - la);
     if (!(a > 0.0) || c > 1.0) c = 1.0;
     const double den = gfun(b, K);
     if (!(den > 0.0)) return 0.0;
@@ -113,30 +118,58 @@ __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun,
     return p;
 }
 
-// First tile whose inclusive prefix of the cached tile sums exceeds the target (sequential,
-// float64, ascending: the same order as the total).  If rounding leaves none, the last tile
-// with positive mass, with a base that makes the in-tile search fall back to its last
-// positive element.  Results: sh_i[2] = tile, sh_d[0] = mass before it, sh_d[1] = target.
-__device__ void locate_tile(const float *partials, int ntiles, double target, int *sh_i, double *sh_d) {
-    double cum = 0.0, base = 0.0;
-    int sel = -1, lastpos = 0;
-    for (int t = 0; t < ntiles; ++t) {
-        const double v = (double)partials[t];
+// First tile whose inclusive prefix of the tile sums exceeds the target (float64, ascending
+// vocabulary order), found by the whole block: every thread owns a contiguous run of tiles, the
+// runs' totals are scanned across the block, and each thread searches its own run.  If rounding
+// leaves no such tile, the last tile with positive mass is taken, with a base that makes the
+// in-tile search fall back to its last positive element.  scale[t] (may be NULL) multiplies tile
+// t's sum.  All threads must call.  Results: sh_i[2] = tile, sh_d[0] = mass before it,
+// sh_d[1] = target.
+__device__ void locate_tile(const float *partials, const float *scale, int ntiles, double target, int *sh_i,
+                            double *sh_d, double *sh_warp) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int per = (ntiles + kThreads - 1) / kThreads;
+    const int t0 = min(ntiles, tid * per), t1 = min(ntiles, t0 + per);
+    double local = 0.0;
+    for (int t = t0; t < t1; ++t) local += (double)partials[t] * (scale ? (double)scale[t] : 1.0);
+    double incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (tid == 0) {
+        sh_i[2] = INT_MAX;  // first tile that crosses the target
+        sh_i[3] = -1;       // last tile with positive mass
+    }
+    if (lane == 31) sh_warp[wid] = incl;
+    __syncthreads();
+    double cum = incl - local;
+    for (int w = 0; w < wid; ++w) cum += sh_warp[w];
+    int first = INT_MAX, lastpos = -1;
+    double base = 0.0;
+    for (int t = t0; t < t1; ++t) {
+        const double v = (double)partials[t] * (scale ? (double)scale[t] : 1.0);
         if (v > 0.0) lastpos = t;
-        if (cum + v > target) {
-            sel = t;
+        if (first == INT_MAX && cum + v > target) {
+            first = t;
             base = cum;
-            break;
         }
         cum += v;
     }
-    if (sel < 0) {
-        sel = lastpos;
-        base = -INFINITY;
+    if (first != INT_MAX) atomicMin(&sh_i[2], first);
+    if (lastpos >= 0) atomicMax(&sh_i[3], lastpos);
+    __syncthreads();
+    if (first != INT_MAX && sh_i[2] == first) sh_d[0] = base;  // exactly one thread owns that tile
+    __syncthreads();
+    if (tid == 0) {
+        if (sh_i[2] == INT_MAX) {
+            sh_i[2] = max(sh_i[3], 0);
+            sh_d[0] = -INFINITY;
+        }
+        sh_d[1] = target;
     }
-    sh_i[2] = sel;
-    sh_d[0] = base;
-    sh_d[1] = target;
+    __syncthreads();
 }
 
 template <typename T>
@@ -148,11 +181,17 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int K = s.K, g = s.gamma, KG = K * g;
     double *h_s = reinterpret_cast<double *>(smem_raw);                       // [K*g]
     double *W_s = h_s + KG;                                                   // [K*g] sum of wpart
-    double *la_s = W_s + KG;                                                  // [K*(g+1)] log q(x_k^i)
+    double *D_s = W_s + KG;                                                   // [K*g] sum of dpart
+    double *M_s = D_s + KG;                                                   // [K*g] sum of mpart
+    double *la_s = M_s + KG;                                                  // [K*(g+1)] log q(x_k^i)
     double *lb_s = la_s + K * (g + 1);                                        // [K*(g+1)] log p(x_k^i)
     unsigned long long *rej_s = reinterpret_cast<unsigned long long *>(lb_s + K * (g + 1));  // [K]
-    float *tile_s = reinterpret_cast<float *>(rej_s + K);                     // [ntiles]
-    unsigned char *lcp_s = reinterpret_cast<unsigned char *>(tile_s + s.ntiles);  // [K*K]
+    int32_t *tok_s = reinterpret_cast<int32_t *>(rej_s + K);                  // [K*g] the draft tokens
+    float *u_s = reinterpret_cast<float *>(tok_s + KG);                       // [K*g+1] the uniforms
+    unsigned char *lcp_s = reinterpret_cast<unsigned char *>(u_s + KG + 1);   // [K*K]
+    // per-tile (sum, maximum -> factor) of the target row a bonus token is drawn from: global scratch
+    float *tile_s = ws.bonus + (size_t)blockIdx.x * 2 * s.ntiles;             // [ntiles]
+    float *tile_m = tile_s + s.ntiles;                                        // [ntiles]
     __shared__ double sh_warp[kWarps];
     __shared__ float sh_redf[kWarps];
     __shared__ int sh_pick[2];
@@ -163,27 +202,45 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int32_t *tok = tok_all + (size_t)b * KG;
     const float *u = u_all + (size_t)b * (KG + 1);
-    const int status_in = ws.status[b];
     const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
-    const bool invalid = lost || (status_in & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT)) != 0;
+    int myflags = ws.prestatus ? ws.prestatus[b] : 0;
 
-    // ---- 0. joint prefix probabilities (logs), one thread per draft -----------------------------
+    // the uniforms are needed by the serial scan: fetch them now, with threads other than those
+    // that start the token work below
+    for (int n = (tid + kThreads / 2) % kThreads; n <= KG; n += kThreads) u_s[n] = u[n];
+
+    // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
+    //         running sum per draft ------------------------------------------------------------
+    for (int n = tid; n < KG; n += kThreads) {
+        const int k = n / g, i = n % g;
+        const size_t r = ((size_t)b * K + k) * g + i;
+        const RowInfo ri = ws.rows[r];
+        int t = tok[n];
+        tok_s[n] = t;
+        myflags |= ri.flags;
+        if (t < 0 || t >= s.V) {  // the row is flagged and produces no output
+            myflags |= SGBV_STATUS_TOKEN_RANGE;
+            t = 0;
+        }
+        const float zqt = ld_logit(zq_all, (((size_t)b * K + k) * (g + 1) + i) * s.V + t);
+        const float zpt = ld_logit(zp_all, r * s.V + t);
+        la_s[k * (g + 1) + i + 1] = ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
+        lb_s[k * (g + 1) + i + 1] = ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
+    }
+    // block-wide OR of the flags (these also are the barrier after the loop)
+    const int status_in = (__syncthreads_or(myflags & SGBV_STATUS_TOKEN_RANGE) ? SGBV_STATUS_TOKEN_RANGE : 0) |
+                          (__syncthreads_or(myflags & SGBV_STATUS_NONFINITE_LOGIT) ? SGBV_STATUS_NONFINITE_LOGIT : 0);
+    const bool invalid = lost || status_in != 0;
     for (int k = tid; k < K; k += kThreads) {
         double la = 0.0, lb = 0.0;
-        for (int i = 0; i < g; ++i) {
+        la_s[k * (g + 1)] = 0.0;
+        lb_s[k * (g + 1)] = 0.0;
+        for (int i = 1; i <= g; ++i) {
+            la += la_s[k * (g + 1) + i];
+            lb += lb_s[k * (g + 1) + i];
             la_s[k * (g + 1) + i] = la;
             lb_s[k * (g + 1) + i] = lb;
-            const size_t r = ((size_t)b * K + k) * g + i;
-            const RowInfo ri = ws.rows[r];
-            int t = tok[k * g + i];
-            if (t < 0 || t >= s.V) t = 0;  // the row is flagged and produces no output
-            const float zqt = ld_logit(zq_all, (((size_t)b * K + k) * (g + 1) + i) * s.V + t);
-            const float zpt = ld_logit(zp_all, r * s.V + t);
-            la += ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
-            lb += ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
         }
-        la_s[k * (g + 1) + g] = la;
-        lb_s[k * (g + 1) + g] = lb;
     }
     __syncthreads();
 
@@ -195,40 +252,59 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const bool aux = ri.c < 1.0f;
         const float *wp = ws.wpart + r * s.ntiles, *dp = ws.dpart + r * s.ntiles, *mp = ws.mpart + r * s.ntiles;
         double sw = 0.0, sd = 0.0, sm = 0.0;
-        for (int t = lane; t < s.ntiles; t += 32) {
-            sw += (double)wp[t];
-            if (aux) {
-                sd += (double)dp[t];
-                sm += (double)mp[t];
+        for (int t0 = 0; t0 < s.ntiles; t0 += 128) {  // four independent loads per array in flight
+            float w4[4], d4[4], m4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int t = t0 + lane + 32 * e;
+                const bool in = t < s.ntiles;
+                w4[e] = in ? wp[t] : 0.0f;
+                d4[e] = (in && aux) ? dp[t] : 0.0f;
+                m4[e] = (in && aux) ? mp[t] : 0.0f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                sw += (double)w4[e];
+                sd += (double)d4[e];
+                sm += (double)m4[e];
             }
         }
         sw = warp_sum(sw);
         sd = warp_sum(sd);
         sm = warp_sum(sm);
         if (lane == 0) {
-            const double R = sw / ri.Zq;
             W_s[n] = sw;
-            const double la = la_s[k * (g + 1) + i], lb = lb_s[k * (g + 1) + i];
-            const double S = exp(la) * R;
-            ws.resmass[(size_t)b * KG + n] = invalid ? NAN : S;
-            if (i >= 1) {
-                const double hv = weight_sub(la, lb, R, sd / ri.Zq, sm / ri.Zq, K, aux);
-                h_s[k * g + i - 1] = hv;
-                ws.h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
-            }
+            D_s[n] = sd;
+            M_s[n] = sm;
         }
     }
-    for (int k = tid; k < K; k += kThreads) {
+    __syncthreads();
+    // the float64 transcendentals of Eq. 2, one thread per (k,i) so that they run side by side
+    for (int n = tid; n < KG; n += kThreads) {
+        const int k = n / g, i = n % g;
+        const size_t r = ((size_t)b * K + k) * g + i;
+        const RowInfo ri = ws.rows[r];
+        const double R = W_s[n] / ri.Zq;
+        const double la = la_s[k * (g + 1) + i], lb = lb_s[k * (g + 1) + i];
+        const double S = exp_short(la) * R;
+        ws.resmass[(size_t)b * KG + n] = invalid ? NAN : S;
+        if (i >= 1) {
+            const double hv = weight_sub(la, lb, R, D_s[n] / ri.Zq, M_s[n] / ri.Zq, K, ri.c < 1.0f);
+            h_s[k * g + i - 1] = hv;
+            ws.h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
+        }
+    }
+    for (int k = kThreads - 1 - tid; k < K; k += kThreads) {  // the last threads, while the first ones do Eq. 2
         const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
         h_s[k * g + g - 1] = hv;
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
         rej_s[k] = 0ull;
     }
     // longest common prefix of every pair of drafts (for the membership test in H)
-    for (int n = tid; n < K * K; n += kThreads) {
+    for (int n = (tid + kThreads / 2) % kThreads; n < K * K; n += kThreads) {
         const int k = n / K, kp = n % K;
         int l = 0;
-        while (l < g && tok[k * g + l] == tok[kp * g + l]) ++l;
+        while (l < g && tok_s[k * g + l] == tok_s[kp * g + l]) ++l;
         lcp_s[n] = (unsigned char)l;
     }
     __syncthreads();
@@ -237,7 +313,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         if (tid == 0) {
             out_tau[b] = -1;
             out_f[b] = -1;
-            if (lost) ws.status[b] = status_in | SGBV_STATUS_TIMEOUT;
+            ws.status[b] = status_in | (lost ? SGBV_STATUS_TIMEOUT : 0);
         }
         for (int j = tid; j <= g; j += kThreads) out_tokens[(size_t)b * (g + 1) + j] = -1;
         return;
@@ -251,7 +327,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             const int start = tau + 1;
             for (int i = start; i <= g; ++i) {
                 const double hv = h_s[k * g + i - 1];
-                const double eta = (double)u[k * g + i - 1];
+                const double eta = (double)u_s[k * g + i - 1];
                 bool inH = false;  // an earlier draft with the same i-token prefix was rejected at length i
                 for (int kp = lane; kp < k; kp += 32)
                     inH |= (lcp_s[k * K + kp] >= i) && ((rej_s[kp] >> (i - 1)) & 1ull);
@@ -278,7 +354,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __syncthreads();
     const int tau = sh_i[0], f = sh_i[1];
     const int kk = (tau == 0) ? 0 : f;
-    const double us = (double)u[KG];
+    const double us = (double)u_s[KG];
 
     // ---- 3. extra token -------------------------------------------------------------------------
     int y = -1;
@@ -290,8 +366,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const double W = W_s[kk * g + tau];
         if (W > 0.0) {
             const float *wp = ws.wpart + r * s.ntiles;
-            if (tid == 0) locate_tile(wp, s.ntiles, us * W, sh_i, sh_d);
-            __syncthreads();
+            locate_tile(wp, nullptr, s.ntiles, us * W, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
             const RowInfo ri = ws.rows[r];
             const T *zp = zp_all + (((size_t)b * K + kk) * g + tau) * s.V;
@@ -311,15 +386,44 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         }
     }
     if (from_q) {
-        // softmax(zq/T) of one row, block-wide: max, per-tile sums, locate, pick
-        float m = -INFINITY;
+        // softmax(zq/T) of one row in a single pass over memory: every tile's maximum and its
+        // sum of exponentials relative to that maximum, then the row maximum, the factors that move
+        // the tile sums to it, the tile search and the pick inside the tile
         bool bad = false;
-        for (int x = tid; x < s.V; x += kThreads) {
-            const float z = ld_logit(zq, x);
-            bad |= (z != z) | (z == INFINITY);
-            m = fmaxf(m, z);
+        float m = -INFINITY;
+        constexpr int kNT = 4;  // tiles a warp has in flight
+        for (int tb = wid * kNT; tb < s.ntiles; tb += kWarps * kNT) {
+            float z[kNT][kTile / 32];
+#pragma unroll
+            for (int q = 0; q < kNT; ++q)
+#pragma unroll
+                for (int e = 0; e < kTile / 32; ++e) {
+                    const int x = (tb + q) * kTile + lane + 32 * e;
+                    z[q][e] = (tb + q < s.ntiles && x < s.V) ? ld_logit(zq, x) : -INFINITY;
+                }
+#pragma unroll
+            for (int q = 0; q < kNT; ++q) {
+                if (tb + q >= s.ntiles) break;
+                float mt = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < kTile / 32; ++e) {
+                    bad |= (z[q][e] != z[q][e]) | (z[q][e] == INFINITY);
+                    mt = fmaxf(mt, z[q][e]);
+                }
+                mt = warp_max(mt);
+                float acc = 0.0f;
+                if (mt > -INFINITY) {
+#pragma unroll
+                    for (int e = 0; e < kTile / 32; ++e) acc += expo(z[q][e], mt, s.scale);
+                }
+                acc = warp_sum(acc);
+                if (lane == 0) {
+                    tile_s[tb + q] = acc;
+                    tile_m[tb + q] = mt;
+                }
+                m = fmaxf(m, mt);
+            }
         }
-        m = warp_max(m);
         if (lane == 0) sh_redf[wid] = m;
         bad = __syncthreads_or(bad);
         m = sh_redf[0];
@@ -327,20 +431,18 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         if (bad || !(m > -INFINITY)) {
             flags |= SGBV_STATUS_NONFINITE_LOGIT;
         } else {
-            for (int t = wid; t < s.ntiles; t += kWarps) {
-                const int x0 = t * kTile, x1 = min(s.V, x0 + kTile);
-                float acc = 0.0f;
-                for (int x = x0 + lane; x < x1; x += 32) acc += expo(ld_logit(zq, x), m, s.scale);
-                acc = warp_sum(acc);
-                if (lane == 0) tile_s[t] = acc;
-            }
+            // tile_m becomes the factor exp((m_t - m)/T) of its tile
+            for (int t = tid; t < s.ntiles; t += kThreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
             __syncthreads();
-            if (tid == 0) {
-                double W = 0.0;
-                for (int t = 0; t < s.ntiles; ++t) W += (double)tile_s[t];
-                locate_tile(tile_s, s.ntiles, us * W, sh_i, sh_d);
-            }
+            double W = 0.0;
+            for (int t = tid; t < s.ntiles; t += kThreads) W += (double)tile_s[t] * (double)tile_m[t];
+            W = warp_sum(W);
+            if (lane == 0) sh_warp[wid] = W;
             __syncthreads();
+            W = 0.0;
+            for (int w = 0; w < kWarps; ++w) W += sh_warp[w];
+            __syncthreads();
+            locate_tile(tile_s, tile_m, s.ntiles, us * W, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
             const int x0 = sel * kTile, x1 = min(s.V, x0 + kTile);
             auto wfun = [&](int x) { return expo(ld_logit(zq, x), m, s.scale); };
@@ -354,7 +456,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     if (tid == 0) {
         out_tau[b] = failed ? -1 : tau;
         out_f[b] = failed ? -1 : f;
-        if (flags) ws.status[b] = status_in | flags;
+        ws.status[b] = status_in | flags;
     }
     for (int j = tid; j <= g; j += kThreads) {
         int v = -1;
@@ -370,8 +472,8 @@ template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
     const size_t KG = (size_t)s.K * s.gamma;
-    const size_t smem = 2 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
-                        s.K * sizeof(unsigned long long) + (size_t)s.ntiles * sizeof(float) + (size_t)s.K * s.K;
+    const size_t smem = 4 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
+                        s.K * sizeof(unsigned long long) + KG * sizeof(int32_t) + (KG + 1) * sizeof(float) + (size_t)s.K * s.K;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;

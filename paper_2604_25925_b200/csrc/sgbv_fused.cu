@@ -164,33 +164,6 @@ __device__ __forceinline__ float warp_max_redux(float v) {
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-// 2^x in double precision: x = n + f with |f| <= 1/2, e^(f ln 2) by its Taylor series to degree 13
-// (remainder below 1e-17), scaled by 2^n.  A short dependent chain, unlike the library routine's.
-__device__ __forceinline__ double exp2_short(double x) {
-    if (x != x) return x;
-    if (x < -1100.0) return 0.0;
-    if (x > 1100.0) return INFINITY;
-    const double n = rint(x);
-    const double t = (x - n) * 0.6931471805599453094;
-    double pl = 1.0 / 6227020800.0;
-    pl = fma(pl, t, 1.0 / 479001600.0);
-    pl = fma(pl, t, 1.0 / 39916800.0);
-    pl = fma(pl, t, 1.0 / 3628800.0);
-    pl = fma(pl, t, 1.0 / 362880.0);
-    pl = fma(pl, t, 1.0 / 40320.0);
-    pl = fma(pl, t, 1.0 / 5040.0);
-    pl = fma(pl, t, 1.0 / 720.0);
-    pl = fma(pl, t, 1.0 / 120.0);
-    pl = fma(pl, t, 1.0 / 24.0);
-    pl = fma(pl, t, 1.0 / 6.0);
-    pl = fma(pl, t, 0.5);
-    pl = fma(pl, t, 1.0);
-    pl = fma(pl, t, 1.0);
-    // 2^n built from its bit pattern where it is a normal number, else the library's scaling
-    const int ni = (int)n;
-    if (ni > -1000 && ni < 1000) return pl * __longlong_as_double((long long)(ni + 1023) << 52);
-    return scalbn(pl, ni);
-}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -387,6 +360,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
+    if (blockIdx.x == 0 && tid == 0) *p.error_flag = 0;  // set again only by a wait that expires (about a second later)
     const int my_chains = (p.nchains - cid + G - 1) / G;
     const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
     const int total_loads = nrows * nchunks;    // chunk pairs this CTA loads
@@ -427,7 +401,6 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     int n = 0;  // row number in this cluster's walk
     for (int cl = 0; cl < my_chains; ++cl) {
         const size_t bk = (size_t)cid + (size_t)cl * G;
-        const int brow = (int)(bk / s.K);
         for (int i = 0; i < s.gamma; ++i, ++n) {
             const size_t r = bk * s.gamma + i;
             const int par = n & 1;
@@ -437,10 +410,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
             if (chain_thread) {
                 int t = tok_next;
-                if (t < 0 || t >= s.V) {
-                    if (rank == 0) atomicOr(p.ws.status + brow, SGBV_STATUS_TOKEN_RANGE);
-                    t = 0;
-                }
+                if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
                 zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
                 zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
                 if (n + 1 < nrows) {
@@ -600,8 +570,9 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     // -inf only has Z = 0
                     const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
                                      !(bq_row < INFINITY) || !(bp_row < INFINITY);
-                    if (bad) atomicOr(p.ws.status + brow, SGBV_STATUS_NONFINITE_LOGIT);
                     RowInfo ri;
+                    ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
+                    ri.pad_ = 0;
                     ri.Zq = (double)Zq;
                     ri.Zp = (double)Zp;
                     ri.mq = bq_row;

@@ -113,6 +113,8 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
         ri.mp = mp;
         double c = exp(lb - la);
         ri.c = (float)c;
+        ri.flags = 0;
+        ri.pad_ = 0;
         ri.kappa = (float)(c * Zq / Zp);
         rows[r] = ri;
         int t = tok[r];
