@@ -1,4 +1,4 @@
-// Finishing kernel: one CTA per batch row.
+// Finishing kernel: one CTA of 1024 threads per batch row.
 //   0. log a_i = log q(x_k^i), log b_i = log p(x_k^i) of every draft by running sums of the token
 //      log-probabilities (row maxima and normalisers come from the streaming pass);
 //   1. combine the cached per-tile sums of every (k,i) row into S_i and the acceptance weights
@@ -14,10 +14,11 @@ namespace sgbv {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-constexpr int kEpt = kTile / kThreads;  // elements per thread inside one tile
-static_assert(kEpt >= 1 && kEpt * kThreads == kTile, "a tile is a whole number of elements per thread");
+constexpr int kMaxThreads = 1024;  // CTA size when few batch rows leave most SMs idle (the kernel is a
+constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps per row help); else 256
+constexpr int kMaxWarps = kMaxThreads / 32;
+constexpr int kEpt = 1;  // elements per thread inside one tile (threads beyond the tile hold none)
+static_assert(kMinThreads >= kTile, "one thread per element of a tile");
 
 // 1 - (1-u)^K as the geometric sum u (1 + (1-u) + ... + (1-u)^(K-1)): all terms are positive, so
 // a tiny u keeps its full relative accuracy, and no transcendental function is needed.
@@ -128,7 +129,8 @@ __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun,
 __device__ void locate_tile(const float *partials, const float *scale, int ntiles, double target, int *sh_i,
                             double *sh_d, double *sh_warp) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const int per = (ntiles + kThreads - 1) / kThreads;
+    const int nthreads = blockDim.x;
+    const int per = (ntiles + nthreads - 1) / nthreads;
     const int t0 = min(ntiles, tid * per), t1 = min(ntiles, t0 + per);
     double local = 0.0;
     for (int t = t0; t < t1; ++t) local += (double)partials[t] * (scale ? (double)scale[t] : 1.0);
@@ -173,7 +175,7 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kMaxThreads)
 finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const int32_t *__restrict__ tok_all,
               const float *__restrict__ u_all, Shape s, Workspace ws, int32_t *__restrict__ out_tau,
               int32_t *__restrict__ out_f, int32_t *__restrict__ out_tokens) {
@@ -192,14 +194,15 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     // per-tile (sum, maximum -> factor) of the target row a bonus token is drawn from: global scratch
     float *tile_s = ws.bonus + (size_t)blockIdx.x * 2 * s.ntiles;             // [ntiles]
     float *tile_m = tile_s + s.ntiles;                                        // [ntiles]
-    __shared__ double sh_warp[kWarps];
-    __shared__ float sh_redf[kWarps];
+    __shared__ double sh_warp[kMaxWarps];
+    __shared__ float sh_redf[kMaxWarps];
     __shared__ int sh_pick[2];
     __shared__ int sh_i[4];
     __shared__ double sh_d[2];
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int nthreads = blockDim.x, nwarps = nthreads / 32;
     const int32_t *tok = tok_all + (size_t)b * KG;
     const float *u = u_all + (size_t)b * (KG + 1);
     const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
@@ -207,11 +210,11 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // the uniforms are needed by the serial scan: fetch them now, with threads other than those
     // that start the token work below
-    for (int n = (tid + kThreads / 2) % kThreads; n <= KG; n += kThreads) u_s[n] = u[n];
+    for (int n = (tid + nthreads / 2) % nthreads; n <= KG; n += nthreads) u_s[n] = u[n];
 
     // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
     //         running sum per draft ------------------------------------------------------------
-    for (int n = tid; n < KG; n += kThreads) {
+    for (int n = tid; n < KG; n += nthreads) {
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
@@ -231,7 +234,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int status_in = (__syncthreads_or(myflags & SGBV_STATUS_TOKEN_RANGE) ? SGBV_STATUS_TOKEN_RANGE : 0) |
                           (__syncthreads_or(myflags & SGBV_STATUS_NONFINITE_LOGIT) ? SGBV_STATUS_NONFINITE_LOGIT : 0);
     const bool invalid = lost || status_in != 0;
-    for (int k = tid; k < K; k += kThreads) {
+    for (int k = tid; k < K; k += nthreads) {
         double la = 0.0, lb = 0.0;
         la_s[k * (g + 1)] = 0.0;
         lb_s[k * (g + 1)] = 0.0;
@@ -245,7 +248,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __syncthreads();
 
     // ---- 1. weights ---------------------------------------------------------------------------
-    for (int n = wid; n < KG; n += kWarps) {
+    for (int n = wid; n < KG; n += nwarps) {
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
@@ -280,7 +283,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     }
     __syncthreads();
     // the float64 transcendentals of Eq. 2, one thread per (k,i) so that they run side by side
-    for (int n = tid; n < KG; n += kThreads) {
+    for (int n = tid; n < KG; n += nthreads) {
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
@@ -294,14 +297,14 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             ws.h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
         }
     }
-    for (int k = kThreads - 1 - tid; k < K; k += kThreads) {  // the last threads, while the first ones do Eq. 2
+    for (int k = nthreads - 1 - tid; k < K; k += nthreads) {  // the last threads, while the first ones do Eq. 2
         const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
         h_s[k * g + g - 1] = hv;
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
         rej_s[k] = 0ull;
     }
     // longest common prefix of every pair of drafts (for the membership test in H)
-    for (int n = (tid + kThreads / 2) % kThreads; n < K * K; n += kThreads) {
+    for (int n = (tid + nthreads / 2) % nthreads; n < K * K; n += nthreads) {
         const int k = n / K, kp = n % K;
         int l = 0;
         while (l < g && tok_s[k * g + l] == tok_s[kp * g + l]) ++l;
@@ -315,7 +318,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             out_f[b] = -1;
             ws.status[b] = status_in | (lost ? SGBV_STATUS_TIMEOUT : 0);
         }
-        for (int j = tid; j <= g; j += kThreads) out_tokens[(size_t)b * (g + 1) + j] = -1;
+        for (int j = tid; j <= g; j += nthreads) out_tokens[(size_t)b * (g + 1) + j] = -1;
         return;
     }
 
@@ -392,7 +395,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         bool bad = false;
         float m = -INFINITY;
         constexpr int kNT = 4;  // tiles a warp has in flight
-        for (int tb = wid * kNT; tb < s.ntiles; tb += kWarps * kNT) {
+        for (int tb = wid * kNT; tb < s.ntiles; tb += nwarps * kNT) {
             float z[kNT][kTile / 32];
 #pragma unroll
             for (int q = 0; q < kNT; ++q)
@@ -427,20 +430,20 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         if (lane == 0) sh_redf[wid] = m;
         bad = __syncthreads_or(bad);
         m = sh_redf[0];
-        for (int w = 1; w < kWarps; ++w) m = fmaxf(m, sh_redf[w]);
+        for (int w = 1; w < nwarps; ++w) m = fmaxf(m, sh_redf[w]);
         if (bad || !(m > -INFINITY)) {
             flags |= SGBV_STATUS_NONFINITE_LOGIT;
         } else {
             // tile_m becomes the factor exp((m_t - m)/T) of its tile
-            for (int t = tid; t < s.ntiles; t += kThreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
+            for (int t = tid; t < s.ntiles; t += nthreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
             __syncthreads();
             double W = 0.0;
-            for (int t = tid; t < s.ntiles; t += kThreads) W += (double)tile_s[t] * (double)tile_m[t];
+            for (int t = tid; t < s.ntiles; t += nthreads) W += (double)tile_s[t] * (double)tile_m[t];
             W = warp_sum(W);
             if (lane == 0) sh_warp[wid] = W;
             __syncthreads();
             W = 0.0;
-            for (int w = 0; w < kWarps; ++w) W += sh_warp[w];
+            for (int w = 0; w < nwarps; ++w) W += sh_warp[w];
             __syncthreads();
             locate_tile(tile_s, tile_m, s.ntiles, us * W, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
@@ -458,7 +461,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         out_f[b] = failed ? -1 : f;
         ws.status[b] = status_in | flags;
     }
-    for (int j = tid; j <= g; j += kThreads) {
+    for (int j = tid; j <= g; j += nthreads) {
         int v = -1;
         if (!failed) {
             if (j < tau) v = tok[f * g + j];
@@ -478,7 +481,7 @@ int run(const Launch &L) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;
     }
-    finish_kernel<T><<<s.B, kThreads, smem, L.stream>>>((const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, L.ws,
+    finish_kernel<T><<<s.B, s.B <= 148 ? kMaxThreads : kMinThreads, smem, L.stream>>>((const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, L.ws,
                                                         L.out_tau, L.out_f, L.out_tokens);
     return cudaGetLastError() == cudaSuccess ? 1 : SGBV_ERR_CUDA;
 }
