@@ -45,6 +45,27 @@ def algorithmic_bytes(cfg, n_bonus: float) -> dict:
     return {"sweep": sweep, "step": sweep + bonus + small}
 
 
+def kernel_traffic(workload: str):
+    """DRAM bytes per launch of the logit-streaming kernel from the committed ncu capture
+    (profiles/fused_chain_kernel_traffic.txt), or None if there is no capture for this workload or the
+    kernel source has changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "fused_chain_kernel_traffic.txt")
+    src = os.path.join(ROOT, "paper_2604_25925_b200", "csrc", "sgbv_fused.cu")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+        vals = {}
+        for line in open(path):
+            if ":" in line and not line.startswith("#"):
+                k, v = line.split(":", 1)
+                vals[k.strip()] = v.strip()
+        if vals.get("source_sha256") != sha or workload not in vals:
+            return None
+        return int(vals[workload].split()[0])
+    except Exception:
+        return None
+
+
 def hbm_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -187,7 +208,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2604_25925_b200 import binding, workloads
+    from paper_2604_25925_b200 import binding, sharding, workloads
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -256,10 +277,7 @@ def main():
         dist.barrier()
     ms_total = ev0.elapsed_time(ev1)
     kern_ms, kern_n = binding.profile_end()
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(ms_total, device=dev)   # a step takes as long as its slowest rank
     clocks = sampler.stop(t0, t1) if sampler else None
 
     # parity-relevant facts of the timed outputs, and the end-to-end / CPU legs (rank 0)
@@ -286,7 +304,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": binding.last_main_kernel(), "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                          "peak_source": f"of {which}", "kernel_ms": kern_avg_ms, "launches_timed": kern_n,
-                         "algorithmic_bytes_per_launch": ab["sweep"], "traffic": None},
+                         "algorithmic_bytes_per_launch": ab["sweep"], "traffic": kernel_traffic(cfg.name)},
             "gpu_launches": launches_per_step * steps,
             "clocks": clocks,
         }
