@@ -370,19 +370,19 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     // Loads are numbered in consumption order: chunk m of this CTA's walk is chunk m % nchunks of
     // row m / nchunks and lands in ring stage m % S.  issue_chunk is stateless, so any lane can issue
     // any chunk: lanes of one warp issue the chunks of a whole row side by side.
-    auto issue_chunk = [&](int m) {
-        const int row = m / nchunks, jc = m - row * nchunks;
-        const int chain = row / s.gamma, pos = row - chain * s.gamma;
-        const size_t bkc = (size_t)cid + (size_t)chain * G;
+    auto issue_at = [&](size_t bkc, int pos, int jc, int stage) {
         const int x0 = x_begin + jc * kChunk;  // first element of the chunk
         const T *zq = reinterpret_cast<const T *>(p.zq) + (bkc * (s.gamma + 1) + pos) * s.V + x0;
         const T *zp = reinterpret_cast<const T *>(p.zp) + (bkc * s.gamma + pos) * s.V + x0;
         const uint32_t bytes = (uint32_t)min(kChunk, cta_len - jc * kChunk) * (uint32_t)sizeof(T);
-        const int stage = m % S;
         unsigned char *dst = ring + (size_t)stage * kStageBytes;
         mbar_expect_tx(&full[stage], 2 * bytes);
         bulk_load(dst, zq, bytes, &full[stage]);
         bulk_load(dst + kChunkBytes, zp, bytes, &full[stage]);
+    };
+    auto issue_chunk = [&](int m) {
+        const int row = m / nchunks, chain = row / s.gamma;
+        issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S);
     };
     if (warp == 0 && lane < S && lane < total_loads) issue_chunk(lane);  // fill the ring
 
@@ -534,9 +534,22 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             // chain thread's warp 0 has enough to do), so the copy requests are issued side by side.
             {
                 const int jc = (warp + kFWarps - 1) % kFWarps;  // warp 1 -> chunk 0, ..., warp 0 -> chunk 7
-                if (lane == 0 && jc < nchunks) {
-                    const int m = n * nchunks + jc + S;
-                    if (m < total_loads) issue_chunk(m);
+                if (lane == 0 && jc < nchunks && n * nchunks + jc + S < total_loads) {
+                    // chunk jc of this row sits in stage (st - nchunks + jc) mod S; the chunk that replaces it
+                    // is S chunks further along the walk: a few rows on, maybe in the next chain
+                    int stage = st - nchunks + jc;
+                    while (stage < 0) stage += S;
+                    int jc2 = jc + S, pos = i;
+                    while (jc2 >= nchunks) {
+                        jc2 -= nchunks;
+                        ++pos;
+                    }
+                    size_t bkc = bk;
+                    while (pos >= s.gamma) {
+                        pos -= s.gamma;
+                        bkc += G;
+                    }
+                    issue_at(bkc, pos, jc2, stage);
                 }
             }
 
