@@ -205,12 +205,16 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     const int nthreads = blockDim.x, nwarps = nthreads / 32;
     const int32_t *tok = tok_all + (size_t)b * KG;
     const float *u = u_all + (size_t)b * (KG + 1);
-    const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
-    int myflags = ws.prestatus ? ws.prestatus[b] : 0;
-
     // the uniforms are needed by the serial scan: fetch them now, with threads other than those
     // that start the token work below
     for (int n = (tid + nthreads / 2) % nthreads; n <= KG; n += nthreads) u_s[n] = u[n];
+    for (int n = tid; n < KG; n += nthreads) tok_s[n] = tok[n];
+    // Everything above reads only the caller's inputs.  The kernel may have been scheduled while the
+    // streaming kernel was still running (programmatic dependent launch): wait for it to complete
+    // before touching the row records and cell sums.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
+    int myflags = ws.prestatus ? ws.prestatus[b] : 0;
 
     // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
     //         running sum per draft ------------------------------------------------------------
@@ -218,8 +222,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
-        int t = tok[n];
-        tok_s[n] = t;
+        int t = tok_s[n];
         myflags |= ri.flags;
         if (t < 0 || t >= s.V) {  // the row is flagged and produces no output
             myflags |= SGBV_STATUS_TOKEN_RANGE;
@@ -481,9 +484,25 @@ int run(const Launch &L) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;
     }
-    finish_kernel<T><<<s.B, s.B <= 148 ? kMaxThreads : kMinThreads, smem, L.stream>>>((const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, L.ws,
-                                                        L.out_tau, L.out_f, L.out_tokens);
-    return cudaGetLastError() == cudaSuccess ? 1 : SGBV_ERR_CUDA;
+    // programmatic stream serialisation: the kernel may be scheduled before the one ahead of it in the
+    // stream has finished; it waits for that kernel itself (griddepcontrol.wait) once it needs its results
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(s.B);
+    cfg.blockDim = dim3(s.B <= 148 ? kMaxThreads : kMinThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = L.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, finish_kernel<T>, (const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, L.ws,
+                                       L.out_tau, L.out_f, L.out_tokens);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return SGBV_ERR_CUDA;
+    }
+    return 1;
 }
 
 }  // namespace

@@ -360,6 +360,9 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
+    // the finishing kernel is launched with programmatic stream serialisation: let it be scheduled now
+    // (it waits for this grid to complete before it reads anything this grid writes)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (blockIdx.x == 0 && tid == 0) *p.error_flag = 0;  // set again only by a wait that expires (about a second later)
     const int my_chains = (p.nchains - cid + G - 1) / G;
     const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
