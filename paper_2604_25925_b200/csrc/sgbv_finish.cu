@@ -304,7 +304,6 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
         h_s[k * g + g - 1] = hv;
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
-        rej_s[k] = 0ull;
     }
     // longest common prefix of every pair of drafts (for the membership test in H)
     for (int n = (tid + nthreads / 2) % nthreads; n < K * K; n += nthreads) {
@@ -327,29 +326,41 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // ---- 2. scan (Algorithm 1), warp 0 ---------------------------------------------------------
     if (wid == 0) {
+        // All state lives in registers.  Lane l owns drafts l and l + 32: pass = the lengths whose
+        // Bernoulli trial succeeds (eta < h), rej = the lengths at which the draft entered H.
+        unsigned long long pass0 = 0, pass1 = 0, rej0 = 0, rej1 = 0;
+        for (int i = 1; i <= g; ++i) {
+            if (lane < K && (double)u_s[lane * g + i - 1] < h_s[lane * g + i - 1]) pass0 |= 1ull << (i - 1);
+            if (lane + 32 < K && (double)u_s[(lane + 32) * g + i - 1] < h_s[(lane + 32) * g + i - 1])
+                pass1 |= 1ull << (i - 1);
+        }
         int tau = 0, f = -1;
         bool done = false;
         for (int k = 0; k < K && !done; ++k) {
-            const int start = tau + 1;
-            for (int i = start; i <= g; ++i) {
-                const double hv = h_s[k * g + i - 1];
-                const double eta = (double)u_s[k * g + i - 1];
-                bool inH = false;  // an earlier draft with the same i-token prefix was rejected at length i
-                for (int kp = lane; kp < k; kp += 32)
-                    inH |= (lcp_s[k * K + kp] >= i) && ((rej_s[kp] >> (i - 1)) & 1ull);
-                inH = __any_sync(0xffffffffu, inH);
-                const bool accept = (eta < hv) && !inH;
-                if (accept) {
+            const unsigned long long passk = __shfl_sync(0xffffffffu, k < 32 ? pass0 : pass1, k & 31);
+            // common prefix of draft k with this lane's drafts; only earlier drafts can be in H
+            const int l0 = (lane < k) ? lcp_s[k * K + lane] : 0;
+            const int l1 = (lane + 32 < k) ? lcp_s[k * K + lane + 32] : 0;
+            unsigned long long rejk = 0;
+            for (int i = tau + 1; i <= g; ++i) {  // the start is fixed when the draft is entered
+                const unsigned long long bit = 1ull << (i - 1);
+                // an earlier draft with the same i-token prefix was rejected at length i
+                const bool mine = (l0 >= i && (rej0 & bit)) || (l1 >= i && (rej1 & bit));
+                const bool inH = __any_sync(0xffffffffu, mine);
+                if ((passk & bit) && !inH) {
                     tau = i;
                     f = k;
                     if (i == g) {
                         done = true;
                         break;
                     }
-                } else if (lane == 0) {
-                    rej_s[k] |= 1ull << (i - 1);
+                } else {
+                    rejk |= bit;
                 }
-                __syncwarp();
+            }
+            if (lane == (k & 31)) {
+                if (k < 32) rej0 = rejk;
+                else rej1 = rejk;
             }
         }
         if (lane == 0) {
