@@ -128,7 +128,7 @@ struct Control {
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
     // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
     float4 wslots[2][kFWarps];
-    int warps_in[2];                     // warps of this CTA whose partial of the row is in wslots
+    int arrivals;                        // partials left in wslots so far, over all rows (never reset)
     float4 slots[2][kMaxCluster];
     double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
 };
@@ -353,7 +353,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
         for (int i = 0; i < S; ++i) mbar_init(&ctl->full[i], 1);
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
-        ctl->warps_in[0] = ctl->warps_in[1] = 0;
+        ctl->arrivals = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -516,11 +516,10 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             if (lane == 0) {
                 ctl->wslots[par][warp] = make_float4(bqw, sq, bpw, sp);
                 __threadfence_block();
-                last_warp = atomicAdd(&ctl->warps_in[par], 1) == kFWarps - 1;
+                last_warp = atomicAdd(&ctl->arrivals, 1) + 1 == kFWarps * (n + 1);
             }
             if (__shfl_sync(0xffffffffu, last_warp, 0)) {
                 __threadfence_block();
-                if (lane == 0) ctl->warps_in[par] = 0;
                 const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
                 const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
                 const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
@@ -530,12 +529,12 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
             }
 
-            if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
-
-            // The exchange is complete, so every warp of this CTA has turned this row's ring stages into
-            // registers: refill them with the chunks S ahead.  Warps 1, 2, ... take one chunk each (the
-            // chain thread's warp 0 has enough to do), so the copy requests are issued side by side.
-            {
+            // Ring refill.  Once all warps of this CTA have left their partials, all of them have turned
+            // this row's ring stages into registers, and the stages can take the chunks S ahead.  Warps
+            // 1, 2, ... take one chunk each, so the copy requests are issued side by side; a warp that
+            // sees the condition already now does it while it would otherwise wait for the exchange,
+            // the others do it after the exchange (whose completion implies the condition).
+            auto do_refill = [&]() {
                 const int jc = (warp + kFWarps - 1) % kFWarps;  // warp 1 -> chunk 0, ..., warp 0 -> chunk 7
                 if (lane == 0 && jc < nchunks && n * nchunks + jc + S < total_loads) {
                     // chunk jc of this row sits in stage (st - nchunks + jc) mod S; the chunk that replaces it
@@ -554,7 +553,20 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     }
                     issue_at(bkc, pos, jc2, stage);
                 }
+            };
+            bool refilled = false;
+            {
+                int seen = 0;
+                if (lane == 0) seen = *reinterpret_cast<volatile int *>(&ctl->arrivals);
+                if (__shfl_sync(0xffffffffu, seen, 0) >= kFWarps * (n + 1)) {
+                    do_refill();
+                    refilled = true;
+                }
             }
+            if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
+
+            // Refill (see do_refill above) if it could not be done while waiting.
+            if (!refilled) do_refill();
 
             // ---- row statistics: every warp combines the CTA partials, in the same order -------------
             const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
