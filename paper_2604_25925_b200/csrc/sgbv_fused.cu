@@ -788,7 +788,9 @@ int launch_fused(const Launch &L, int *error_flag) {
     const size_t budget = kSmemPerSm / occ - kSmemReserved - sizeof(Control);
     if ((size_t)S * stage_bytes > budget) S = (int)(budget / stage_bytes);
     if (S > kMaxStages) S = kMaxStages;
-    if (S < 2) return SGBV_ERR_SHAPE;
+    // a whole row slice is moved to registers before any of its stages is refilled, so the ring must
+    // hold all chunks of a row at once
+    if (S < 2 || S < plan.nch) return g_opt_stages ? SGBV_ERR_SHAPE : 0;
     plan.stages = S;
     plan.smem = (size_t)S * stage_bytes + sizeof(Control);
     plan.grid_clusters = g_opt_max_clusters;

@@ -154,7 +154,7 @@ def _slice_fits(V, cluster):
 
 @pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 4),
                                     ("cluster", 8), ("cluster", 16), ("stages", 2), ("stages", 3),
-                                    ("max_clusters", 3)])
+                                    ("max_clusters", 3), ("occupancy", 3), ("occupancy", 4)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / ring depth /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
@@ -167,6 +167,10 @@ def test_every_kernel_path_and_launch_shape_matches(option):
         for cfg in cfgs:
             if option[0] == "cluster" and not _slice_fits(cfg.V, option[1]):
                 continue   # forced cluster size whose slices do not fit the registers
+            if option[0] == "stages" and -(-(-(-cfg.V // 256) // 8) // 8) > option[1]:
+                continue   # the ring must hold all chunks of a row slice (clusters of at most 8 here)
+            if option[0] == "occupancy" and -(-cfg.V // 256) > 16 * 8 * (2 if option[1] == 3 else 1):
+                continue   # with 3 (4) CTAs per SM a warp holds 2 (1) cells: the row must fit 16 CTAs
             inp = workloads.make_inputs(cfg, device="cuda")
             rep, _, _ = run_both(inp)
             assert_parity(rep)
