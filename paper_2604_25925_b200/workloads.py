@@ -56,6 +56,10 @@ CONFIGS = {
     "c3": VerifyConfig("c3", B=32, K=4, gamma=5, V=128256, dtype="bf16", temperature=0.7,
                        alpha=0.7, seed=1236),
     "c4": VerifyConfig("c4", B=64, K=8, gamma=8, V=151936, alpha=0.9, seed=1237),
+    # the paper's own operating points (Table 2): one prompt, K = 3 drafts, L = 12 or 8, T = 0.4,
+    # a 32k vocabulary (DeepSeek-coder's 32256)
+    "paper_l12": VerifyConfig("paper_l12", B=1, K=3, gamma=12, V=32256, temperature=0.4, alpha=0.85, seed=1240),
+    "paper_l8": VerifyConfig("paper_l8", B=1, K=3, gamma=8, V=32256, temperature=0.4, alpha=0.85, seed=1241),
 }
 
 

@@ -129,6 +129,27 @@ def test_config5_sweep_parity_sampled_rows(K):
                     assert int(out.accept_len[b]) == tau
 
 
+@pytest.mark.parametrize("name", ["paper_l12", "paper_l8"])
+def test_paper_operating_points(name):
+    """K = 3 drafts of 12 or 8 tokens at T = 0.4 over a 32k vocabulary (the paper's Table 2 settings),
+    as a batch of 6 prompts so that several chains share the machine."""
+    cfg = workloads.with_batch(workloads.CONFIGS[name], 6)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+
+
+@pytest.mark.parametrize("K,dtype", [(5, "fp32"), (6, "bf16"), (7, "fp32"), (16, "fp32")])
+def test_draft_counts_without_a_specialised_kernel(K, dtype):
+    """K outside {1,2,3,4,8} takes the run-time-K code of the fused kernel (rows are 16-byte aligned)."""
+    cfg = workloads.VerifyConfig(f"k{K}", B=3, K=K, gamma=3, V=8192, dtype=dtype, temperature=0.8, alpha=0.85,
+                                 seed=500 + K)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+    assert binding.last_main_kernel() == "fused_chain_kernel"
+
+
 EDGE_SHAPES = [
     # B, K, gamma, V
     (3, 1, 1, 1), (2, 2, 3, 7), (5, 3, 2, 1000), (2, 2, 2, 1025), (2, 4, 3, 32001), (1, 1, 1, 5000),
