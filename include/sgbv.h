@@ -160,6 +160,7 @@ int sgbv_profile_end(double *out_total_ms, int *out_records);
  *   "cluster"      CTAs per cluster of the fused kernel (1, 2, 4, 8 or 16)
  *   "stages"       depth of its shared-memory ring (2..12)
  *   "max_clusters" cap on the number of resident clusters it launches
+ *   "walk"         1 = a cluster of the fused kernel walks whole draft chains, 2 = single rows
  *   "occupancy"    CTAs of the fused kernel per SM (2, 3 or 4; more CTAs hold fewer cells each)
  * Returns SGBV_ERR_SHAPE for an unknown name or a value out of range.
  */

@@ -36,7 +36,7 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
 }
 
 struct Carve {
-    size_t rows, part, wpart, dpart, mpart, bonus, h, resmass, status, error, total;
+    size_t rows, part, wpart, dpart, mpart, ratio, bonus, h, resmass, status, error, total;
 };
 
 Carve carve(const Shape &s) {
@@ -48,6 +48,7 @@ Carve carve(const Shape &s) {
     c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.mpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.ratio = off;     off += align_up(NR * sizeof(double));
     c.bonus = off;     off += align_up((size_t)s.B * 2 * s.ntiles * sizeof(float));
     c.h = off;         off += align_up(NR * sizeof(double));
     c.resmass = off;   off += align_up(NR * sizeof(double));
@@ -93,7 +94,7 @@ int grow(void **ptr, size_t *have, size_t need) {
 
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
-int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_occupancy = 0;
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_occupancy = 0, g_opt_walk = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -138,6 +139,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     L.ws.wpart = (float *)(base + c.wpart);
     L.ws.dpart = (float *)(base + c.dpart);
     L.ws.mpart = (float *)(base + c.mpart);
+    L.ws.ratio = (double *)(base + c.ratio);
     L.ws.bonus = (float *)(base + c.bonus);
     L.ws.h = out_h ? out_h : (double *)(base + c.h);
     L.ws.resmass = out_resmass ? out_resmass : (double *)(base + c.resmass);
@@ -291,13 +293,16 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;
         g_opt_max_clusters = value;
+    } else if (!strcmp(name, "walk")) {
+        if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
+        g_opt_walk = value;
     } else if (!strcmp(name, "occupancy")) {
         if (value != 0 && (value < 2 || value > 4)) return SGBV_ERR_SHAPE;
         g_opt_occupancy = value;
     } else {
         return SGBV_ERR_SHAPE;
     }
-    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_occupancy);
+    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_occupancy, g_opt_walk);
     return SGBV_OK;
 }
 

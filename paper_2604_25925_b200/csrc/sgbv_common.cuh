@@ -36,6 +36,8 @@ struct Workspace {
     float *wpart;       // [B*K*gamma][ntiles]: sum over the tile of eq * max(1 - kappa ep/eq, 0)^K
     float *dpart;       // [B*K*gamma][ntiles]: sum of max(kappa ep - eq, 0)               (c < 1)
     float *mpart;       // [B*K*gamma][ntiles]: sum of eq (c - t)^2 Q(t)                    (c < 1)
+    double *ratio;      // [B*K*gamma]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel);
+                        // preset to a NaN pattern before each launch, which reads as "not published yet"
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     double *h;          // [B][K][gamma]
     double *resmass;    // [B][K][gamma]
@@ -167,6 +169,6 @@ bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0
 int launch_fused(const Launch &L, int *error_flag);
-void fused_set_options(int cluster, int stages, int max_clusters, int occupancy);
+void fused_set_options(int cluster, int stages, int max_clusters, int occupancy, int walk);
 
 }  // namespace sgbv

@@ -50,6 +50,7 @@ struct FusedParams {
     int slice_len;    // vocabulary elements per CTA (multiple of kCell)
     int stages;       // ring depth
     int nchains;      // B*K
+    int row_mode;     // 0: a cluster walks whole chains; 1: a cluster walks single rows (see the kernel)
     int *error_flag;  // set to 1 if a bounded wait expired
 };
 
@@ -61,6 +62,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
@@ -124,7 +128,8 @@ __device__ __forceinline__ float rcp(float x) {
 // [ring: stages x (chunk of zq, chunk of zp)] [Control]
 struct Control {
     uint64_t full[kMaxStages];           // per ring stage: "both chunks have landed"
-    uint64_t xbar[2];                    // by row parity: "all partials of the row and c_i are here"
+    uint64_t xbar[2];                    // by row parity: "all partials of the row (chain walk: and c_i) are here"
+    uint64_t cbar[2];                    // by row parity, row walk only: "c_i is here"
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
     // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
     float4 wslots[2][kFWarps];
@@ -323,7 +328,7 @@ __device__ __forceinline__ void sweep_two_dispatch(const float2 (&eq)[NCH][4], c
 
 // OCC = CTAs of this kernel that share an SM (2, 3 or 4): more co-resident CTAs hide more of each
 // other's exchange and pipeline latency, but leave each thread fewer registers, hence fewer cells.
-template <typename T, int NCH, int OCC>
+template <typename T, int NCH, int OCC, bool kRow>
 __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const FusedParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
@@ -353,6 +358,8 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
         for (int i = 0; i < S; ++i) mbar_init(&ctl->full[i], 1);
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
+        mbar_init(&ctl->cbar[0], 1);
+        mbar_init(&ctl->cbar[1], 1);
         ctl->arrivals = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -360,12 +367,25 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
-    // the finishing kernel is launched with programmatic stream serialisation: let it be scheduled now
-    // (it waits for this grid to complete before it reads anything this grid writes)
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The finishing kernel is launched with programmatic stream serialisation: let it be scheduled now
+    // (it waits for this grid to complete before it reads anything this grid writes).  Not in row mode:
+    // there clusters wait for one another, so no CTA of this grid may find its place on an SM taken by
+    // a kernel that in turn waits for this grid.
+    if (!kRow) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (blockIdx.x == 0 && tid == 0) *p.error_flag = 0;  // set again only by a wait that expires (about a second later)
-    const int my_chains = (p.nchains - cid + G - 1) / G;
-    const int nrows = my_chains * s.gamma;      // rows this cluster walks, in order
+    // The walk of this cluster: position n = 0, 1, ... is row (bk, i).
+    //   chain mode: chains cid, cid+G, ... each from i = 0 to gamma-1 (c_i is carried along the chain);
+    //   row mode:   rows u = cid, cid+G, ... of the list of all rows, u = bk*gamma + i.  Used when there
+    //               are few chains: all rows of a chain then run at the same time on different clusters,
+    //               and c_i comes from the ratios p_j(tok_j)/q_j(tok_j) that the clusters of rows j < i
+    //               publish in global memory.  A row only waits for rows earlier in the list, which are
+    //               walked no later by clusters that are all resident, so every wait ends.
+    // One step of the walk: bk += step_bk, i += step_i, and on i >= gamma: i -= gamma, bk += wrap_bk.
+    constexpr bool row_mode = kRow;
+    const int step_bk = row_mode ? G / s.gamma : 0, step_i = row_mode ? G % s.gamma : 1, wrap_bk = row_mode ? 1 : G;
+    const long total_rows = (long)p.nchains * s.gamma;
+    const int nrows = row_mode ? (int)((total_rows - cid + G - 1) / G)
+                               : ((p.nchains - cid + G - 1) / G) * s.gamma;  // rows this cluster walks
     const int total_loads = nrows * nchunks;    // chunk pairs this CTA loads
     const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
     bool timed_out = false;
@@ -384,8 +404,14 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
         bulk_load(dst + kChunkBytes, zp, bytes, &full[stage]);
     };
     auto issue_chunk = [&](int m) {
-        const int row = m / nchunks, chain = row / s.gamma;
-        issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S);
+        const int row = m / nchunks;  // position in the walk
+        if (row_mode) {
+            const long u = (long)cid + (long)row * G;
+            issue_at((size_t)(u / s.gamma), (int)(u % s.gamma), m - row * nchunks, m % S);
+        } else {
+            const int chain = row / s.gamma;
+            issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S);
+        }
     };
     if (warp == 0 && lane < S && lane < total_loads) issue_chunk(lane);  // fill the ring
 
@@ -393,8 +419,8 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     // ahead: tok_next is the token of the next row of the walk.
     const bool chain_thread = tid == kFThreads - 32;  // lane 0 of the last warp; thread 0 writes the row records
     int tok_next = 0;
-    if (chain_thread && nrows > 0) tok_next = p.tok[(size_t)cid * s.gamma];
-    if (chain_thread && nrows > 0) {  // the first row of the walk starts a chain: c_0 = 1
+    if (chain_thread && nrows > 0) tok_next = p.tok[row_mode ? (size_t)cid : (size_t)cid * s.gamma];
+    if (chain_thread && nrows > 0 && !row_mode) {  // the first row of the walk starts a chain: c_0 = 1
         ctl->c[0] = 1.0;
         mbar_expect_tx(&ctl->xbar[0], xbytes);
     }
@@ -402,9 +428,10 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     int st = 0;
     uint32_t ph = 0;
     int n = 0;  // row number in this cluster's walk
-    for (int cl = 0; cl < my_chains; ++cl) {
-        const size_t bk = (size_t)cid + (size_t)cl * G;
-        for (int i = 0; i < s.gamma; ++i, ++n) {
+    size_t bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
+    int i = row_mode ? cid % s.gamma : 0;
+    {
+        for (; n < nrows; ++n) {
             const size_t r = bk * s.gamma + i;
             const int par = n & 1;
             const uint32_t xph = (uint32_t)(n >> 1) & 1u;
@@ -412,13 +439,18 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
             float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
             if (chain_thread) {
+                if (row_mode) mbar_expect_tx(&ctl->xbar[par], xbytes);  // the exchange does not wait for c_i here
                 int t = tok_next;
                 if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
                 zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
                 zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
                 if (n + 1 < nrows) {
-                    const size_t bk_n = (i + 1 < s.gamma) ? bk : bk + G;
-                    const int i_n = (i + 1 < s.gamma) ? i + 1 : 0;
+                    size_t bk_n = bk + step_bk;
+                    int i_n = i + step_i;
+                    if (i_n >= s.gamma) {
+                        i_n -= s.gamma;
+                        bk_n += wrap_bk;
+                    }
                     tok_next = p.tok[bk_n * s.gamma + i_n];
                 }
             }
@@ -542,14 +574,15 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     int stage = st - nchunks + jc;
                     while (stage < 0) stage += S;
                     int jc2 = jc + S, pos = i;
-                    while (jc2 >= nchunks) {
-                        jc2 -= nchunks;
-                        ++pos;
-                    }
                     size_t bkc = bk;
-                    while (pos >= s.gamma) {
-                        pos -= s.gamma;
-                        bkc += G;
+                    while (jc2 >= nchunks) {  // one step of the walk per row
+                        jc2 -= nchunks;
+                        bkc += step_bk;
+                        pos += step_i;
+                        if (pos >= s.gamma) {
+                            pos -= s.gamma;
+                            bkc += wrap_bk;
+                        }
                     }
                     issue_at(bkc, pos, jc2, stage);
                 }
@@ -574,24 +607,69 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
             const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
             const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
-            const double cd = ctl->c[par];
-            const float c = (float)cd;
-            const float kappa = (float)(cd * (double)(Zq / Zp));
-
-            if (chain_thread && n + 1 < nrows) {
-                // c of the next row of the walk: c_{i+1} = c_i p_i(tok_i)/q_i(tok_i), or 1 at the start
-                // of the next chain; publishing it arms the next row's exchange
-                {
-                    double c_next = 1.0;
-                    if (i + 1 < s.gamma) {
-                        const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
-                        const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
-                        c_next = cd * exp2_short(lp - lq) * (double)(Zq / Zp);
+            // the ratio p_i(tok_i)/q_i(tok_i) of this row (chain thread)
+            auto token_ratio = [&]() {
+                const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
+                const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
+                return exp2_short(lp - lq) * (double)(Zq / Zp);
+            };
+            double cd;
+            if (row_mode) {
+                // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
+                // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
+                // NaN (a row that produces one is flagged invalid anyway).
+                if (chain_thread && rank == 0 && i + 1 < s.gamma) {
+                    double ratio = token_ratio();
+                    if (ratio != ratio) ratio = 0.0;
+                    *reinterpret_cast<volatile double *>(p.ws.ratio + r) = ratio;
+                }
+                // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
+                // butterfly over the lanes).  Those rows are walked by other clusters at about the same
+                // time and publish right after their own statistics, which do not depend on c: no chain of
+                // waits forms.  Every lane of the last warp polls one of them.  Bounded waits.
+                if (warp == kFWarps - 1) {
+                    double cprod = 1.0;
+                    const size_t r0 = bk * s.gamma;
+                    for (int j0 = 0; j0 < i; j0 += 32) {
+                        double v = 1.0;
+                        if (j0 + lane < i) {
+                            const volatile double *word =
+                                reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
+                            v = *word;
+                            if (v != v) {
+                                const long long t0 = clock64();
+                                while ((v = *word) != v) {
+                                    if (clock64() - t0 > kWaitLimitCycles) {
+                                        timed_out = true;
+                                        v = 0.0;
+                                        break;
+                                    }
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) v *= __shfl_xor_sync(0xffffffffu, v, o);
+                        cprod *= v;
                     }
-                    ctl->c[par ^ 1] = c_next;
+                    if (lane == 0) {
+                        ctl->c[par] = cprod;
+                        mbar_arrive(&ctl->cbar[par]);  // c_i is there
+                    }
+                }
+                if (!mbar_wait(&ctl->cbar[par], xph)) timed_out = true;
+                cd = ctl->c[par];
+            } else {
+                cd = ctl->c[par];
+                if (chain_thread && n + 1 < nrows) {
+                    // c of the next row of the walk: c_{i+1} = c_i ratio, or 1 at the start of the next
+                    // chain; publishing it arms the next row's exchange
+                    ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * token_ratio() : 1.0;
                     mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
                 }
             }
+            const float c = (float)cd;
+            const float kappa = (float)(cd * (double)(Zq / Zp));
+
             if (tid == 0) {
                 if (rank == 0) {
                     // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
@@ -637,6 +715,14 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                 sweep_two_dispatch<NCH, true>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
             else
                 sweep_two_dispatch<NCH, false>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
+
+            // one step of the walk
+            bk += step_bk;
+            i += step_i;
+            if (i >= s.gamma) {
+                i -= s.gamma;
+                bk += wrap_bk;
+            }
         }
     }
     if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(p.error_flag, 1);
@@ -646,7 +732,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
 
 // ---- host side ----------------------------------------------------------------------------------------
 struct Plan {
-    int cluster, slice_len, nch, occ, stages, grid_clusters;
+    int cluster, slice_len, nch, occ, stages, grid_clusters, row_mode;
     size_t smem;
 };
 
@@ -654,6 +740,7 @@ int g_opt_cluster = 0;     // 0 = automatic
 int g_opt_stages = 0;
 int g_opt_max_clusters = 0;
 int g_opt_occupancy = 0;
+int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
 
 constexpr int kSmemPerSm = 228 * 1024;     // shared memory of one SM
 constexpr int kSmemReserved = 1024;        // per resident CTA, taken by the system
@@ -664,9 +751,9 @@ int max_nch(int occ) { return occ <= 2 ? kMaxNch : occ == 3 ? 2 : 1; }
 int cells_of(int V) { return (V + kCell - 1) / kCell; }
 int slice_cells(int cells, int C) { return (cells + C - 1) / C; }
 
-template <typename T, int NCH, int OCC>
+template <typename T, int NCH, int OCC, bool kRow>
 int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
-    auto kernel = fused_chain_kernel<T, NCH, OCC>;
+    auto kernel = fused_chain_kernel<T, NCH, OCC, kRow>;
     static bool attr_done[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGBV_ERR_CUDA;
@@ -688,6 +775,7 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     fp.slice_len = plan.slice_len;
     fp.stages = plan.stages;
     fp.nchains = L.s.B * L.s.K;
+    fp.row_mode = plan.row_mode;
     fp.error_flag = error_flag;
 
     cudaLaunchConfig_t cfg = {};
@@ -718,7 +806,11 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
         }
         clusters = slot;
     }
-    if (clusters > fp.nchains) clusters = fp.nchains;
+    const long units = plan.row_mode ? (long)fp.nchains * L.s.gamma : (long)fp.nchains;  // what the clusters share out
+    if (clusters > units) clusters = (int)units;
+    if (plan.row_mode &&
+        cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
+        return SGBV_ERR_CUDA;
     cfg.gridDim = dim3(clusters * plan.cluster);
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, fp);
@@ -732,22 +824,34 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
 
 template <typename T>
 int launch_t(const Launch &L, const Plan &plan, int *error_flag) {
+    if (plan.row_mode) {  // the row walk exists for two CTAs per SM
+        if (plan.occ != 2) return SGBV_ERR_SHAPE;
+        switch (plan.nch) {
+            case 1: return launch_nch<T, 1, 2, true>(L, plan, error_flag);
+            case 2: return launch_nch<T, 2, 2, true>(L, plan, error_flag);
+            case 3: return launch_nch<T, 3, 2, true>(L, plan, error_flag);
+            case 4: return launch_nch<T, 4, 2, true>(L, plan, error_flag);
+            case 5: return launch_nch<T, 5, 2, true>(L, plan, error_flag);
+            default: return SGBV_ERR_SHAPE;
+        }
+    }
     switch (plan.occ * 10 + plan.nch) {
-        case 21: return launch_nch<T, 1, 2>(L, plan, error_flag);
-        case 22: return launch_nch<T, 2, 2>(L, plan, error_flag);
-        case 23: return launch_nch<T, 3, 2>(L, plan, error_flag);
-        case 24: return launch_nch<T, 4, 2>(L, plan, error_flag);
-        case 25: return launch_nch<T, 5, 2>(L, plan, error_flag);
-        case 31: return launch_nch<T, 1, 3>(L, plan, error_flag);
-        case 32: return launch_nch<T, 2, 3>(L, plan, error_flag);
-        case 41: return launch_nch<T, 1, 4>(L, plan, error_flag);
+        case 21: return launch_nch<T, 1, 2, false>(L, plan, error_flag);
+        case 22: return launch_nch<T, 2, 2, false>(L, plan, error_flag);
+        case 23: return launch_nch<T, 3, 2, false>(L, plan, error_flag);
+        case 24: return launch_nch<T, 4, 2, false>(L, plan, error_flag);
+        case 25: return launch_nch<T, 5, 2, false>(L, plan, error_flag);
+        case 31: return launch_nch<T, 1, 3, false>(L, plan, error_flag);
+        case 32: return launch_nch<T, 2, 3, false>(L, plan, error_flag);
+        case 41: return launch_nch<T, 1, 4, false>(L, plan, error_flag);
         default: return SGBV_ERR_SHAPE;
     }
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int stages, int max_clusters, int occupancy) {
+void fused_set_options(int cluster, int stages, int max_clusters, int occupancy, int walk) {
+    g_opt_walk = walk;
     g_opt_cluster = cluster;
     g_opt_stages = stages;
     g_opt_max_clusters = max_clusters;
@@ -772,11 +876,23 @@ int launch_fused(const Launch &L, int *error_flag) {
     const int cap = max_nch(occ) * kChunk;  // elements of a row one CTA can hold
     const long cta_slots = (long)occ * kSms;
     int C = g_opt_cluster;
+    int Cmin = 1;
+    while (Cmin < kMaxCluster && slice_cells(cells, Cmin) * kCell > cap) Cmin *= 2;  // smallest cluster whose slices fit
     if (C == 0) {
-        C = 1;
-        while (C < kMaxCluster && slice_cells(cells, C) * kCell > cap) C *= 2;  // smallest cluster whose slices fit
+        C = Cmin;
         // few chains: spread each over more CTAs while they all stay co-resident in one wave
         while (C < kMaxCluster && nchains * 2 * C <= cta_slots && cells / (2 * C) >= 4) C *= 2;
+    }
+    // Few rows in all: when every ROW can have a cluster of its own in one wave, share out single rows
+    // instead of chains (their only coupling, c_i, is looked up), so that the gamma rows of a chain run
+    // side by side instead of one after the other.
+    {
+        const long units = nchains * s.gamma;
+        int Crow = g_opt_cluster ? g_opt_cluster : Cmin;
+        if (g_opt_cluster == 0)
+            while (Crow < kMaxCluster && units * 2 * Crow <= cta_slots && cells / (2 * Crow) >= 4) Crow *= 2;
+        plan.row_mode = occ == 2 && s.gamma > 1 && (g_opt_walk == 2 || (g_opt_walk == 0 && units * Crow <= cta_slots));
+        if (plan.row_mode) C = Crow;
     }
     if (C < 1 || C > kMaxCluster || slice_cells(cells, C) * kCell > cap) return g_opt_occupancy ? SGBV_ERR_SHAPE : 0;
     plan.cluster = C;

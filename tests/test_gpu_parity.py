@@ -167,6 +167,10 @@ def test_edge_shapes(B, K, gamma, V, dtype):
     assert_parity(rep)
 
 
+def _cdiv(a, b):
+    return -(-a // b)
+
+
 def _slice_fits(V, cluster):
     """A CTA of the fused kernel holds at most five chunks of 2048 elements of a row in registers."""
     cells = -(-V // 256)
@@ -175,7 +179,7 @@ def _slice_fits(V, cluster):
 
 @pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 4),
                                     ("cluster", 8), ("cluster", 16), ("stages", 2), ("stages", 3),
-                                    ("max_clusters", 3), ("occupancy", 3), ("occupancy", 4)])
+                                    ("max_clusters", 3), ("occupancy", 3), ("occupancy", 4), ("walk", 1), ("walk", 2)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / ring depth /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
@@ -184,12 +188,14 @@ def test_every_kernel_path_and_launch_shape_matches(option):
                                    seed=22),
             workloads.VerifyConfig("paths_c", B=2, K=2, gamma=5, V=1000, alpha=0.9, seed=23)]
     binding.set_option(*option)
+    if option[0] == "stages":
+        binding.set_option("cluster", 8)   # fixes the number of chunks per row slice that the ring must hold
     try:
         for cfg in cfgs:
             if option[0] == "cluster" and not _slice_fits(cfg.V, option[1]):
                 continue   # forced cluster size whose slices do not fit the registers
-            if option[0] == "stages" and -(-(-(-cfg.V // 256) // 8) // 8) > option[1]:
-                continue   # the ring must hold all chunks of a row slice (clusters of at most 8 here)
+            if option[0] == "stages" and (not _slice_fits(cfg.V, 8) or _cdiv(_cdiv(_cdiv(cfg.V, 256), 8), 8) > option[1]):
+                continue   # the ring must hold all chunks of a row slice (clusters of 8 here)
             if option[0] == "occupancy" and -(-cfg.V // 256) > 16 * 8 * (2 if option[1] == 3 else 1):
                 continue   # with 3 (4) CTAs per SM a warp holds 2 (1) cells: the row must fit 16 CTAs
             inp = workloads.make_inputs(cfg, device="cuda")
@@ -197,6 +203,7 @@ def test_every_kernel_path_and_launch_shape_matches(option):
             assert_parity(rep)
     finally:
         binding.set_option(option[0], 0)
+        binding.set_option("cluster", 0)
 
 
 def test_unaligned_views_and_repeated_calls_are_deterministic():
