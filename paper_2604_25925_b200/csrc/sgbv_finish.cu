@@ -213,44 +213,12 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     // streaming kernel was still running (programmatic dependent launch): wait for it to complete
     // before touching the row records and cell sums.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    __syncthreads();  // the staged tokens and uniforms are read by other threads than those that fetched them
     const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
     int myflags = ws.prestatus ? ws.prestatus[b] : 0;
 
-    // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
-    //         running sum per draft ------------------------------------------------------------
-    for (int n = tid; n < KG; n += nthreads) {
-        const int k = n / g, i = n % g;
-        const size_t r = ((size_t)b * K + k) * g + i;
-        const RowInfo ri = ws.rows[r];
-        int t = tok_s[n];
-        myflags |= ri.flags;
-        if (t < 0 || t >= s.V) {  // the row is flagged and produces no output
-            myflags |= SGBV_STATUS_TOKEN_RANGE;
-            t = 0;
-        }
-        const float zqt = ld_logit(zq_all, (((size_t)b * K + k) * (g + 1) + i) * s.V + t);
-        const float zpt = ld_logit(zp_all, r * s.V + t);
-        la_s[k * (g + 1) + i + 1] = ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
-        lb_s[k * (g + 1) + i + 1] = ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
-    }
-    // block-wide OR of the flags (these also are the barrier after the loop)
-    const int status_in = (__syncthreads_or(myflags & SGBV_STATUS_TOKEN_RANGE) ? SGBV_STATUS_TOKEN_RANGE : 0) |
-                          (__syncthreads_or(myflags & SGBV_STATUS_NONFINITE_LOGIT) ? SGBV_STATUS_NONFINITE_LOGIT : 0);
-    const bool invalid = lost || status_in != 0;
-    for (int k = tid; k < K; k += nthreads) {
-        double la = 0.0, lb = 0.0;
-        la_s[k * (g + 1)] = 0.0;
-        lb_s[k * (g + 1)] = 0.0;
-        for (int i = 1; i <= g; ++i) {
-            la += la_s[k * (g + 1) + i];
-            lb += lb_s[k * (g + 1) + i];
-            la_s[k * (g + 1) + i] = la;
-            lb_s[k * (g + 1) + i] = lb;
-        }
-    }
-    __syncthreads();
-
-    // ---- 1. weights ---------------------------------------------------------------------------
+    // ---- cell sums of every row (k,i), one warp per row, first warps first; the token work of step 0
+    //      below starts with the LAST threads, so that for small K*gamma both run side by side ----
     for (int n = wid; n < KG; n += nwarps) {
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
@@ -284,6 +252,42 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             M_s[n] = sm;
         }
     }
+
+    // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
+    //         running sum per draft ------------------------------------------------------------
+    for (int n = nthreads - 1 - tid; n < KG; n += nthreads) {
+        const int k = n / g, i = n % g;
+        const size_t r = ((size_t)b * K + k) * g + i;
+        const RowInfo ri = ws.rows[r];
+        int t = tok_s[n];
+        myflags |= ri.flags;
+        if (t < 0 || t >= s.V) {  // the row is flagged and produces no output
+            myflags |= SGBV_STATUS_TOKEN_RANGE;
+            t = 0;
+        }
+        const float zqt = ld_logit(zq_all, (((size_t)b * K + k) * (g + 1) + i) * s.V + t);
+        const float zpt = ld_logit(zp_all, r * s.V + t);
+        la_s[k * (g + 1) + i + 1] = ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
+        lb_s[k * (g + 1) + i + 1] = ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
+    }
+    // block-wide OR of the flags (these also are the barrier after the loop)
+    const int status_in = (__syncthreads_or(myflags & SGBV_STATUS_TOKEN_RANGE) ? SGBV_STATUS_TOKEN_RANGE : 0) |
+                          (__syncthreads_or(myflags & SGBV_STATUS_NONFINITE_LOGIT) ? SGBV_STATUS_NONFINITE_LOGIT : 0);
+    const bool invalid = lost || status_in != 0;
+    for (int k = tid; k < K; k += nthreads) {
+        double la = 0.0, lb = 0.0;
+        la_s[k * (g + 1)] = 0.0;
+        lb_s[k * (g + 1)] = 0.0;
+        for (int i = 1; i <= g; ++i) {
+            la += la_s[k * (g + 1) + i];
+            lb += lb_s[k * (g + 1) + i];
+            la_s[k * (g + 1) + i] = la;
+            lb_s[k * (g + 1) + i] = lb;
+        }
+    }
+    __syncthreads();
+
+    // ---- 1. weights ---------------------------------------------------------------------------
     __syncthreads();
     // the float64 transcendentals of Eq. 2, one thread per (k,i) so that they run side by side
     for (int n = tid; n < KG; n += nthreads) {
