@@ -39,6 +39,7 @@ struct Workspace {
     double *ratio;      // [B*K*gamma]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel);
                         // preset to a NaN pattern before each launch, which reads as "not published yet"
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
+    int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory
     double *h;          // [B][K][gamma]
     double *resmass;    // [B][K][gamma]
     int32_t *status;    // [B]: final per-row status, written by the finishing kernel

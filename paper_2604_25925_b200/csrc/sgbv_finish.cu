@@ -17,6 +17,7 @@ namespace {
 constexpr int kMaxThreads = 1024;  // CTA size when few batch rows leave most SMs idle (the kernel is a
 constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps per row help); else 256
 constexpr int kMaxWarps = kMaxThreads / 32;
+constexpr int kTilesInSmem = 4096;  // rows up to 2^20 entries keep the bonus row's tile sums in shared memory
 constexpr int kEpt = 1;  // elements per thread inside one tile (threads beyond the tile hold none)
 static_assert(kMinThreads >= kTile, "one thread per element of a tile");
 
@@ -132,8 +133,17 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
     const int nthreads = blockDim.x;
     const int per = (ntiles + nthreads - 1) / nthreads;
     const int t0 = min(ntiles, tid * per), t1 = min(ntiles, t0 + per);
+    // the thread's tile sums: the first four stay in registers for the search below
+    constexpr int kKeep = 4;
+    double kept[kKeep];
     double local = 0.0;
-    for (int t = t0; t < t1; ++t) local += (double)partials[t] * (scale ? (double)scale[t] : 1.0);
+#pragma unroll
+    for (int e = 0; e < kKeep; ++e) {
+        const int t = t0 + e;
+        kept[e] = (t < t1) ? (double)partials[t] * (scale ? (double)scale[t] : 1.0) : 0.0;
+        local += kept[e];
+    }
+    for (int t = t0 + kKeep; t < t1; ++t) local += (double)partials[t] * (scale ? (double)scale[t] : 1.0);
     double incl = local;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -151,7 +161,15 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
     int first = INT_MAX, lastpos = -1;
     double base = 0.0;
     for (int t = t0; t < t1; ++t) {
-        const double v = (double)partials[t] * (scale ? (double)scale[t] : 1.0);
+        double v;
+        if (t - t0 < kKeep) {
+            v = kept[0];
+#pragma unroll
+            for (int e = 1; e < kKeep; ++e)
+                if (t - t0 == e) v = kept[e];
+        } else {
+            v = (double)partials[t] * (scale ? (double)scale[t] : 1.0);
+        }
         if (v > 0.0) lastpos = t;
         if (first == INT_MAX && cum + v > target) {
             first = t;
@@ -191,8 +209,10 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     int32_t *tok_s = reinterpret_cast<int32_t *>(rej_s + K);                  // [K*g] the draft tokens
     float *u_s = reinterpret_cast<float *>(tok_s + KG);                       // [K*g+1] the uniforms
     unsigned char *lcp_s = reinterpret_cast<unsigned char *>(u_s + KG + 1);   // [K*K]
-    // per-tile (sum, maximum -> factor) of the target row a bonus token is drawn from: global scratch
-    float *tile_s = ws.bonus + (size_t)blockIdx.x * 2 * s.ntiles;             // [ntiles]
+    // per-tile (sum, maximum -> factor) of the target row a bonus token is drawn from: shared memory
+    // when the row has few enough tiles (the launcher then reserves the space), else global scratch
+    float *tile_s = ws.bonus_in_smem ? reinterpret_cast<float *>(lcp_s + ((K * K + 15) / 16) * 16)
+                                               : ws.bonus + (size_t)blockIdx.x * 2 * s.ntiles;  // [ntiles]
     float *tile_m = tile_s + s.ntiles;                                        // [ntiles]
     __shared__ double sh_warp[kMaxWarps];
     __shared__ float sh_redf[kMaxWarps];
@@ -493,8 +513,13 @@ template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
     const size_t KG = (size_t)s.K * s.gamma;
-    const size_t smem = 4 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
-                        s.K * sizeof(unsigned long long) + KG * sizeof(int32_t) + (KG + 1) * sizeof(float) + (size_t)s.K * s.K;
+    size_t smem = 4 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
+                  s.K * sizeof(unsigned long long) + KG * sizeof(int32_t) + (KG + 1) * sizeof(float) +
+                  ((size_t)s.K * s.K + 15) / 16 * 16;
+    Workspace ws = L.ws;
+    const size_t tiles = 2 * (size_t)s.ntiles * sizeof(float);
+    ws.bonus_in_smem = (s.ntiles <= kTilesInSmem && smem + tiles <= 160 * 1024) ? 1 : 0;
+    if (ws.bonus_in_smem) smem += tiles;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(finish_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return SGBV_ERR_CUDA;
@@ -511,7 +536,7 @@ int run(const Launch &L) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, finish_kernel<T>, (const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, L.ws,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, finish_kernel<T>, (const T *)L.zq, (const T *)L.zp, L.tok, L.u, s, ws,
                                        L.out_tau, L.out_f, L.out_tokens);
     if (e != cudaSuccess) {
         cudaGetLastError();
