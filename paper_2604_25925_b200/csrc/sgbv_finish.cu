@@ -125,10 +125,11 @@ __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun,
 // runs' totals are scanned across the block, and each thread searches its own run.  If rounding
 // leaves no such tile, the last tile with positive mass is taken, with a base that makes the
 // in-tile search fall back to its last positive element.  scale[t] (may be NULL) multiplies tile
-// t's sum.  All threads must call.  Results: sh_i[2] = tile, sh_d[0] = mass before it,
+// t's sum.  relative: `target` is a fraction of the total of all tile sums (computed here on the
+// way) instead of a mass.  All threads must call.  Results: sh_i[2] = tile, sh_d[0] = mass before it,
 // sh_d[1] = target.
-__device__ void locate_tile(const float *partials, const float *scale, int ntiles, double target, int *sh_i,
-                            double *sh_d, double *sh_warp) {
+__device__ void locate_tile(const float *partials, const float *scale, int ntiles, double target, bool relative,
+                            int *sh_i, double *sh_d, double *sh_warp) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int nthreads = blockDim.x;
     const int per = (ntiles + nthreads - 1) / nthreads;
@@ -158,6 +159,11 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
     __syncthreads();
     double cum = incl - local;
     for (int w = 0; w < wid; ++w) cum += sh_warp[w];
+    if (relative) {  // the target is given as a fraction of the total of all tiles
+        double total = 0.0;
+        for (int w = 0; w < (nthreads >> 5); ++w) total += sh_warp[w];
+        target *= total;
+    }
     int first = INT_MAX, lastpos = -1;
     double base = 0.0;
     for (int t = t0; t < t1; ++t) {
@@ -407,7 +413,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const double W = W_s[kk * g + tau];
         if (W > 0.0) {
             const float *wp = ws.wpart + r * s.ntiles;
-            locate_tile(wp, nullptr, s.ntiles, us * W, sh_i, sh_d, sh_warp);
+            locate_tile(wp, nullptr, s.ntiles, us * W, false, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
             const RowInfo ri = ws.rows[r];
             const T *zp = zp_all + (((size_t)b * K + kk) * g + tau) * s.V;
@@ -442,27 +448,40 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
                     const int x = (tb + q) * kTile + lane + 32 * e;
                     z[q][e] = (tb + q < s.ntiles && x < s.V) ? ld_logit(zq, x) : -INFINITY;
                 }
+            // the four tiles are reduced side by side (independent shuffle chains)
+            float mt[kNT], acc[kNT];
 #pragma unroll
             for (int q = 0; q < kNT; ++q) {
-                if (tb + q >= s.ntiles) break;
-                float mt = -INFINITY;
+                mt[q] = -INFINITY;
 #pragma unroll
                 for (int e = 0; e < kTile / 32; ++e) {
                     bad |= (z[q][e] != z[q][e]) | (z[q][e] == INFINITY);
-                    mt = fmaxf(mt, z[q][e]);
+                    mt[q] = fmaxf(mt[q], z[q][e]);
                 }
-                mt = warp_max(mt);
-                float acc = 0.0f;
-                if (mt > -INFINITY) {
+            }
 #pragma unroll
-                    for (int e = 0; e < kTile / 32; ++e) acc += expo(z[q][e], mt, s.scale);
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int q = 0; q < kNT; ++q) mt[q] = fmaxf(mt[q], __shfl_xor_sync(0xffffffffu, mt[q], o));
+#pragma unroll
+            for (int q = 0; q < kNT; ++q) {
+                acc[q] = 0.0f;
+                if (mt[q] > -INFINITY) {
+#pragma unroll
+                    for (int e = 0; e < kTile / 32; ++e) acc[q] += expo(z[q][e], mt[q], s.scale);
                 }
-                acc = warp_sum(acc);
-                if (lane == 0) {
-                    tile_s[tb + q] = acc;
-                    tile_m[tb + q] = mt;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                for (int q = 0; q < kNT; ++q) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
+#pragma unroll
+            for (int q = 0; q < kNT; ++q) {
+                if (lane == 0 && tb + q < s.ntiles) {
+                    tile_s[tb + q] = acc[q];
+                    tile_m[tb + q] = mt[q];
                 }
-                m = fmaxf(m, mt);
+                m = fmaxf(m, mt[q]);
             }
         }
         if (lane == 0) sh_redf[wid] = m;
@@ -475,15 +494,8 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             // tile_m becomes the factor exp((m_t - m)/T) of its tile
             for (int t = tid; t < s.ntiles; t += nthreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
             __syncthreads();
-            double W = 0.0;
-            for (int t = tid; t < s.ntiles; t += nthreads) W += (double)tile_s[t] * (double)tile_m[t];
-            W = warp_sum(W);
-            if (lane == 0) sh_warp[wid] = W;
-            __syncthreads();
-            W = 0.0;
-            for (int w = 0; w < nwarps; ++w) W += sh_warp[w];
-            __syncthreads();
-            locate_tile(tile_s, tile_m, s.ntiles, us * W, sh_i, sh_d, sh_warp);
+            // the target is us times the row's total, which the tile search computes on its way
+            locate_tile(tile_s, tile_m, s.ntiles, us, true, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
             const int x0 = sel * kTile, x1 = min(s.V, x0 + kTile);
             auto wfun = [&](int x) { return expo(ld_logit(zq, x), m, s.scale); };
