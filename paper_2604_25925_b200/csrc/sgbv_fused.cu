@@ -413,7 +413,10 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S);
         }
     };
-    if (warp == 0 && lane < S && lane < total_loads) issue_chunk(lane);  // fill the ring
+    // Fill the ring in two goes: the first row's chunks now, so that they do not share the memory system
+    // with later rows' chunks and the first row can start as early as possible; the rest of the ring once
+    // the first row has landed (see the load phase of the first row).
+    if (warp == 0 && lane < nchunks && lane < total_loads) issue_chunk(lane);
 
     // The chain thread of this CTA carries c_i and fetches the token logits one row
     // ahead: tok_next is the token of the next row of the walk.
@@ -486,6 +489,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     }
                 }
             }
+            if (n == 0 && warp == 0 && lane >= nchunks && lane < S && lane < total_loads) issue_chunk(lane);  // rest of the ring
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 if (j < nchunks) {  // uniform over the CTA
