@@ -38,6 +38,7 @@ constexpr int kMaxNch = 5;                 // cells per warp: what one thread ca
 constexpr int kMaxStages = 12;             // ring depth
 constexpr int kMaxCluster = 16;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
+constexpr uint32_t kSuspendNs = 20000u;               // longest single suspension inside a wait
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
 
 struct FusedParams {
@@ -77,11 +78,24 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// The same test, but the thread may be suspended for up to about `kSuspendNs` until the phase completes
+// (the hardware wakes it when it does), instead of coming back at once.
+__device__ __forceinline__ bool mbar_test_suspend(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait: returns false if the phase did not complete within about a second.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
     if (mbar_test(bar, parity)) return true;
     const long long t0 = clock64();
-    while (!mbar_test(bar, parity))
+    while (!mbar_test_suspend(bar, parity))
         if (clock64() - t0 > kWaitLimitCycles) return false;
     return true;
 }

@@ -167,6 +167,27 @@ def test_edge_shapes(B, K, gamma, V, dtype):
     assert_parity(rep)
 
 
+@pytest.mark.parametrize("T", [0.05, 0.2, 3.0, 25.0])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_temperature_extremes(T, dtype):
+    """Very low temperatures turn rows into near point masses (exponentials underflow to zero away from the
+    maximum, residual masses become tiny); very high ones flatten them (every CDF cell is narrow)."""
+    cfg = workloads.VerifyConfig(f"temp_{T}_{dtype}", B=4, K=3, gamma=4, V=12288, dtype=dtype, temperature=T,
+                                 alpha=0.9, seed=int(1000 * T) + 77)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+
+
+def test_vocabulary_beyond_the_fused_kernel_capacity():
+    """Rows longer than 16 CTAs x 10,240 entries take the generic two-sweep kernels, aligned or not."""
+    cfg = workloads.VerifyConfig("bigv", B=2, K=2, gamma=2, V=163840 + 4096, alpha=0.85, seed=606)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+    assert binding.last_main_kernel() == "otreduce_kernel"
+
+
 def _cdiv(a, b):
     return -(-a // b)
 
