@@ -188,6 +188,21 @@ def test_vocabulary_beyond_the_fused_kernel_capacity():
     assert binding.last_main_kernel() == "otreduce_kernel"
 
 
+def test_more_than_2_to_the_31_logits_per_tensor():
+    """Element offsets beyond 32 bits: 2.8e9 bf16 logits in the target tensor (5.6 GB), 2.5e9 in the draft tensor.
+    The oracle recomputes sampled batch rows from both ends of the tensors."""
+    cfg = workloads.VerifyConfig("huge", B=256, K=8, gamma=8, V=151936, dtype="bf16", temperature=0.9, alpha=0.9,
+                                 seed=808)
+    assert cfg.B * cfg.K * (cfg.gamma + 1) * cfg.V > 2 ** 31
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, out, _ = run_both(inp, rows=[0, 131, 255])
+    assert_parity(rep)
+    tau = out.accept_len.cpu().numpy()
+    assert ((tau >= 0) & (tau <= cfg.gamma)).all() and (out.status.cpu().numpy() == 0).all()
+    del inp, out
+    torch.cuda.empty_cache()
+
+
 def _cdiv(a, b):
     return -(-a // b)
 
