@@ -36,6 +36,7 @@ constexpr int kCell = kTile;               // 256 contiguous elements: one warp'
 constexpr int kChunk = kFWarps * kCell;    // 2048 elements: one cell of every warp
 constexpr int kMaxNch = 5;                 // cells per warp: what one thread can hold in registers (5 x 8 pairs)
 constexpr int kMaxStages = 12;             // ring depth
+constexpr int kRowBars = 16;               // "row has landed" barriers: more than the rows the ring can hold
 constexpr int kMaxCluster = 16;
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 constexpr uint32_t kSuspendNs = 20000u;               // longest single suspension inside a wait
@@ -141,7 +142,7 @@ __device__ __forceinline__ float rcp(float x) {
 // ---- shared memory layout ------------------------------------------------------------------------
 // [ring: stages x (chunk of zq, chunk of zp)] [Control]
 struct Control {
-    uint64_t full[kMaxStages];           // per ring stage: "both chunks have landed"
+    uint64_t rowbar[kRowBars];           // by row of the walk (mod 16): "all chunks of the row have landed"
     uint64_t xbar[2];                    // by row parity: "all partials of the row (chain walk: and c_i) are here"
     uint64_t cbar[2];                    // by row parity, row walk only: "c_i is here"
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
@@ -357,7 +358,6 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     constexpr int kStageBytes = 2 * kChunkBytes;  // one chunk of zq, then the same chunk of zp
     unsigned char *ring = smem;
     Control *ctl = reinterpret_cast<Control *>(smem + (size_t)S * kStageBytes);
-    uint64_t *full = ctl->full;
 
     // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 8, ...
     const int x_begin = rank * p.slice_len;
@@ -369,7 +369,8 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     const int x_warp = x_begin + warp * kCell;  // first element of this warp's first cell
 
     if (tid == 0) {
-        for (int i = 0; i < S; ++i) mbar_init(&ctl->full[i], 1);
+        // one arrival (with its byte count) per chunk of the row
+        for (int i = 0; i < kRowBars; ++i) mbar_init(&ctl->rowbar[i], (uint32_t)max(nchunks, 1));
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
         mbar_init(&ctl->cbar[0], 1);
@@ -406,25 +407,27 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
 
     // Loads are numbered in consumption order: chunk m of this CTA's walk is chunk m % nchunks of
     // row m / nchunks and lands in ring stage m % S.  issue_chunk is stateless, so any lane can issue
-    // any chunk: lanes of one warp issue the chunks of a whole row side by side.
-    auto issue_at = [&](size_t bkc, int pos, int jc, int stage) {
+    // any chunk: lanes of one warp issue the chunks of a whole row side by side.  All chunks of walk
+    // position `row` complete on the barrier of that row (one wait per row instead of one per chunk).
+    auto issue_at = [&](size_t bkc, int pos, int jc, int stage, int row) {
         const int x0 = x_begin + jc * kChunk;  // first element of the chunk
         const T *zq = reinterpret_cast<const T *>(p.zq) + (bkc * (s.gamma + 1) + pos) * s.V + x0;
         const T *zp = reinterpret_cast<const T *>(p.zp) + (bkc * s.gamma + pos) * s.V + x0;
         const uint32_t bytes = (uint32_t)min(kChunk, cta_len - jc * kChunk) * (uint32_t)sizeof(T);
         unsigned char *dst = ring + (size_t)stage * kStageBytes;
-        mbar_expect_tx(&full[stage], 2 * bytes);
-        bulk_load(dst, zq, bytes, &full[stage]);
-        bulk_load(dst + kChunkBytes, zp, bytes, &full[stage]);
+        uint64_t *bar = &ctl->rowbar[row & (kRowBars - 1)];
+        mbar_expect_tx(bar, 2 * bytes);
+        bulk_load(dst, zq, bytes, bar);
+        bulk_load(dst + kChunkBytes, zp, bytes, bar);
     };
     auto issue_chunk = [&](int m) {
         const int row = m / nchunks;  // position in the walk
         if (row_mode) {
             const long u = (long)cid + (long)row * G;
-            issue_at((size_t)(u / s.gamma), (int)(u % s.gamma), m - row * nchunks, m % S);
+            issue_at((size_t)(u / s.gamma), (int)(u % s.gamma), m - row * nchunks, m % S, row);
         } else {
             const int chain = row / s.gamma;
-            issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S);
+            issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S, row);
         }
     };
     // Fill the ring in two goes: the first row's chunks now, so that they do not share the memory system
@@ -443,7 +446,6 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     }
 
     int st = 0;
-    uint32_t ph = 0;
     int n = 0;  // row number in this cluster's walk
     size_t bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
     int i = row_mode ? cid % s.gamma : 0;
@@ -475,35 +477,9 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
             // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
             float2 eq[NCH][4], ep[NCH][4];  // two neighbouring vocabulary entries per register pair
             float mq = -INFINITY, mp = -INFINITY;
-            {
-                // all stages of the row are tested at once (one shared-memory round trip when the data
-                // is there, which is the normal case); only a stage that is late is waited for
-                bool ready = true;
-                int stj = st;
-                uint32_t phj = ph;
-#pragma unroll
-                for (int j = 0; j < NCH; ++j) {
-                    if (j < nchunks) {
-                        ready &= mbar_test(&full[stj], phj);
-                        if (++stj == S) {
-                            stj = 0;
-                            phj ^= 1u;
-                        }
-                    }
-                }
-                if (!ready) {
-                    stj = st;
-                    phj = ph;
-                    for (int j = 0; j < nchunks; ++j) {
-                        if (!mbar_wait(&full[stj], phj)) timed_out = true;
-                        if (++stj == S) {
-                            stj = 0;
-                            phj ^= 1u;
-                        }
-                    }
-                }
-            }
+            if (nchunks > 0 && !mbar_wait(&ctl->rowbar[n & (kRowBars - 1)], (uint32_t)(n / kRowBars) & 1u)) timed_out = true;
             if (n == 0 && warp == 0 && lane >= nchunks && lane < S && lane < total_loads) issue_chunk(lane);  // rest of the ring
+            // all loads first, so that their latencies overlap; the maxima afterwards
 #pragma unroll
             for (int j = 0; j < NCH; ++j) {
                 if (j < nchunks) {  // uniform over the CTA
@@ -511,23 +487,25 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                         const unsigned char *base = ring + (size_t)st * kStageBytes + warp * kCellBytes;
                         read_cell<T>(base, lane, eq[j]);
                         read_cell<T>(base + kChunkBytes, lane, ep[j]);
-                        const int cell_x = x_warp + j * kChunk;
-                        if (cell_x + kCell > s.V) {  // the row ends inside this cell
+                    }
+                    if (++st == S) st = 0;
+                }
+            }
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[j][e].x = ep[j][e].x = -INFINITY;
-                                if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[j][e].y = ep[j][e].y = -INFINITY;
-                            }
-                        }
+            for (int j = 0; j < NCH; ++j) {
+                if (j < nj) {
+                    const int cell_x = x_warp + j * kChunk;
+                    if (cell_x + kCell > s.V) {  // the row ends inside this cell
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            mq = max3(mq, eq[j][e].x, eq[j][e].y);
-                            mp = max3(mp, ep[j][e].x, ep[j][e].y);
+                            if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[j][e].x = ep[j][e].x = -INFINITY;
+                            if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[j][e].y = ep[j][e].y = -INFINITY;
                         }
                     }
-                    if (++st == S) {
-                        st = 0;
-                        ph ^= 1u;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        mq = max3(mq, eq[j][e].x, eq[j][e].y);
+                        mp = max3(mp, ep[j][e].x, ep[j][e].y);
                     }
                 }
             }
@@ -591,10 +569,11 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                     // is S chunks further along the walk: a few rows on, maybe in the next chain
                     int stage = st - nchunks + jc;
                     while (stage < 0) stage += S;
-                    int jc2 = jc + S, pos = i;
+                    int jc2 = jc + S, pos = i, row2 = n;
                     size_t bkc = bk;
                     while (jc2 >= nchunks) {  // one step of the walk per row
                         jc2 -= nchunks;
+                        ++row2;
                         bkc += step_bk;
                         pos += step_i;
                         if (pos >= s.gamma) {
@@ -602,7 +581,7 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
                             bkc += wrap_bk;
                         }
                     }
-                    issue_at(bkc, pos, jc2, stage);
+                    issue_at(bkc, pos, jc2, stage, row2);
                 }
             };
             bool refilled = false;
