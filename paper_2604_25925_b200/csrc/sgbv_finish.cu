@@ -205,14 +205,13 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
               int32_t *__restrict__ out_f, int32_t *__restrict__ out_tokens) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int K = s.K, g = s.gamma, KG = K * g;
-    double *h_s = reinterpret_cast<double *>(smem_raw);                       // [K*g]
-    double *W_s = h_s + KG;                                                   // [K*g] sum of wpart
+    double *W_s = reinterpret_cast<double *>(smem_raw);                       // [K*g] sum of wpart
     double *D_s = W_s + KG;                                                   // [K*g] sum of dpart
     double *M_s = D_s + KG;                                                   // [K*g] sum of mpart
     double *la_s = M_s + KG;                                                  // [K*(g+1)] log q(x_k^i)
     double *lb_s = la_s + K * (g + 1);                                        // [K*(g+1)] log p(x_k^i)
-    unsigned long long *rej_s = reinterpret_cast<unsigned long long *>(lb_s + K * (g + 1));  // [K]
-    int32_t *tok_s = reinterpret_cast<int32_t *>(rej_s + K);                  // [K*g] the draft tokens
+    unsigned long long *pass_s = reinterpret_cast<unsigned long long *>(lb_s + K * (g + 1));  // [K] bit i-1: eta < h for length i
+    int32_t *tok_s = reinterpret_cast<int32_t *>(pass_s + K);                 // [K*g] the draft tokens
     float *u_s = reinterpret_cast<float *>(tok_s + KG);                       // [K*g+1] the uniforms
     unsigned char *lcp_s = reinterpret_cast<unsigned char *>(u_s + KG + 1);   // [K*K]
     // per-tile (sum, maximum -> factor) of the target row a bonus token is drawn from: shared memory
@@ -235,6 +234,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     // that start the token work below
     for (int n = (tid + nthreads / 2) % nthreads; n <= KG; n += nthreads) u_s[n] = u[n];
     for (int n = tid; n < KG; n += nthreads) tok_s[n] = tok[n];
+    for (int k = tid; k < K; k += nthreads) pass_s[k] = 0ull;
     // Everything above reads only the caller's inputs.  The kernel may have been scheduled while the
     // streaming kernel was still running (programmatic dependent launch): wait for it to complete
     // before touching the row records and cell sums.
@@ -281,10 +281,17 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // ---- 0. joint prefix probabilities (logs): token log-probabilities in parallel, then one
     //         running sum per draft ------------------------------------------------------------
-    for (int n = nthreads - 1 - tid; n < KG; n += nthreads) {
+    const int n_first = nthreads - 1 - tid;  // this thread's first (k,i), here and in the weights below
+    double inv_Zq_first = 0.0;
+    bool below_first = false;
+    for (int n = n_first; n < KG; n += nthreads) {
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
+        if (n == n_first) {
+            inv_Zq_first = 1.0 / ri.Zq;
+            below_first = ri.c < 1.0f;
+        }
         int t = tok_s[n];
         myflags |= ri.flags;
         if (t < 0 || t >= s.V) {  // the row is flagged and produces no output
@@ -316,23 +323,30 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     // ---- 1. weights ---------------------------------------------------------------------------
     __syncthreads();
     // the float64 transcendentals of Eq. 2, one thread per (k,i) so that they run side by side
-    for (int n = tid; n < KG; n += nthreads) {
+    // (the thread that fetched the row's record for step 0 still has what it needs of it); each weight
+    // leaves the outcome of its trial, eta < h, as one bit for the scan
+    for (int n = n_first; n < KG; n += nthreads) {
         const int k = n / g, i = n % g;
-        const size_t r = ((size_t)b * K + k) * g + i;
-        const RowInfo ri = ws.rows[r];
-        const double R = W_s[n] / ri.Zq;
+        double inv_Zq = inv_Zq_first;
+        bool below = below_first;
+        if (n != n_first) {
+            const RowInfo ri = ws.rows[((size_t)b * K + k) * g + i];
+            inv_Zq = 1.0 / ri.Zq;
+            below = ri.c < 1.0f;
+        }
+        const double R = W_s[n] * inv_Zq;
         const double la = la_s[k * (g + 1) + i], lb = lb_s[k * (g + 1) + i];
         const double S = exp_short(la) * R;
         ws.resmass[(size_t)b * KG + n] = invalid ? NAN : S;
         if (i >= 1) {
-            const double hv = weight_sub(la, lb, R, D_s[n] / ri.Zq, M_s[n] / ri.Zq, K, ri.c < 1.0f);
-            h_s[k * g + i - 1] = hv;
+            const double hv = weight_sub(la, lb, R, D_s[n] * inv_Zq, M_s[n] * inv_Zq, K, below);
+            if ((double)u_s[k * g + i - 1] < hv) atomicOr(&pass_s[k], 1ull << (i - 1));
             ws.h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
         }
     }
-    for (int k = nthreads - 1 - tid; k < K; k += nthreads) {  // the last threads, while the first ones do Eq. 2
+    for (int k = tid; k < K; k += nthreads) {  // the first threads, while the last ones do Eq. 2
         const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
-        h_s[k * g + g - 1] = hv;
+        if ((double)u_s[k * g + g - 1] < hv) atomicOr(&pass_s[k], 1ull << (g - 1));
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
     }
     // longest common prefix of every pair of drafts (for the membership test in H)
@@ -356,42 +370,38 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // ---- 2. scan (Algorithm 1), warp 0 ---------------------------------------------------------
     if (wid == 0) {
-        // All state lives in registers.  Lane l owns drafts l and l + 32: pass = the lengths whose
-        // Bernoulli trial succeeds (eta < h), rej = the lengths at which the draft entered H.
-        unsigned long long pass0 = 0, pass1 = 0, rej0 = 0, rej1 = 0;
-        for (int i = 1; i <= g; ++i) {
-            if (lane < K && (double)u_s[lane * g + i - 1] < h_s[lane * g + i - 1]) pass0 |= 1ull << (i - 1);
-            if (lane + 32 < K && (double)u_s[(lane + 32) * g + i - 1] < h_s[(lane + 32) * g + i - 1])
-                pass1 |= 1ull << (i - 1);
-        }
+        // All state lives in registers, as bit sets over the lengths 1..gamma (bit i-1 = length i).
+        // Lane l owns drafts l and l + 32: pass = the lengths whose Bernoulli trial succeeds (eta < h),
+        // rej = the lengths at which the draft entered H.  A draft's walk over i = tau+1..gamma does not
+        // depend on its own progress (the start is fixed when the draft is entered, H only holds earlier
+        // drafts), so it is evaluated for all lengths at once: the accepted length is the largest one in
+        // the range whose trial passes and whose sub-block is not in H.
+        auto low = [](int l) { return l >= 64 ? ~0ull : (1ull << l) - 1ull; };  // lengths 1..l
+        const unsigned long long pass0 = lane < K ? pass_s[lane] : 0ull, pass1 = lane + 32 < K ? pass_s[lane + 32] : 0ull;
+        unsigned long long rej0 = 0, rej1 = 0;
         int tau = 0, f = -1;
-        bool done = false;
-        for (int k = 0; k < K && !done; ++k) {
+        for (int k = 0; k < K; ++k) {
             const unsigned long long passk = __shfl_sync(0xffffffffu, k < 32 ? pass0 : pass1, k & 31);
             // common prefix of draft k with this lane's drafts; only earlier drafts can be in H
             const int l0 = (lane < k) ? lcp_s[k * K + lane] : 0;
             const int l1 = (lane + 32 < k) ? lcp_s[k * K + lane + 32] : 0;
-            unsigned long long rejk = 0;
-            for (int i = tau + 1; i <= g; ++i) {  // the start is fixed when the draft is entered
-                const unsigned long long bit = 1ull << (i - 1);
-                // an earlier draft with the same i-token prefix was rejected at length i
-                const bool mine = (l0 >= i && (rej0 & bit)) || (l1 >= i && (rej1 & bit));
-                const bool inH = __any_sync(0xffffffffu, mine);
-                if ((passk & bit) && !inH) {
-                    tau = i;
-                    f = k;
-                    if (i == g) {
-                        done = true;
-                        break;
-                    }
-                } else {
-                    rejk |= bit;
-                }
+            // lengths at which an earlier draft with the same prefix of that length entered H
+            const unsigned long long mine = (rej0 & low(l0)) | (rej1 & low(l1));
+            const unsigned long long inH =
+                ((unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)(mine >> 32)) << 32) |
+                (unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)mine);
+            const unsigned long long range = low(g) & ~low(tau);  // lengths tau+1..gamma
+            const unsigned long long acc = passk & ~inH & range;
+            const unsigned long long rejk = range & ~acc;
+            if (acc != 0ull) {
+                tau = 64 - __clzll((long long)acc);
+                f = k;
             }
             if (lane == (k & 31)) {
                 if (k < 32) rej0 = rejk;
                 else rej1 = rejk;
             }
+            if (tau == g) break;  // the whole block was accepted
         }
         if (lane == 0) {
             sh_i[0] = tau;
@@ -525,7 +535,7 @@ template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
     const size_t KG = (size_t)s.K * s.gamma;
-    size_t smem = 4 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
+    size_t smem = 3 * KG * sizeof(double) + 2 * (size_t)s.K * (s.gamma + 1) * sizeof(double) +
                   s.K * sizeof(unsigned long long) + KG * sizeof(int32_t) + (KG + 1) * sizeof(float) +
                   ((size_t)s.K * s.K + 15) / 16 * 16;
     Workspace ws = L.ws;

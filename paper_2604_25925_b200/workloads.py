@@ -60,6 +60,8 @@ CONFIGS = {
     # a 32k vocabulary (DeepSeek-coder's 32256)
     "paper_l12": VerifyConfig("paper_l12", B=1, K=3, gamma=12, V=32256, temperature=0.4, alpha=0.85, seed=1240),
     "paper_l8": VerifyConfig("paper_l8", B=1, K=3, gamma=8, V=32256, temperature=0.4, alpha=0.85, seed=1241),
+    # the longest draft length of the paper's sweep over L
+    "paper_l24": VerifyConfig("paper_l24", B=1, K=3, gamma=24, V=32256, temperature=0.4, alpha=0.85, seed=1242),
 }
 
 

@@ -129,9 +129,10 @@ def test_config5_sweep_parity_sampled_rows(K):
                     assert int(out.accept_len[b]) == tau
 
 
-@pytest.mark.parametrize("name", ["paper_l12", "paper_l8"])
+@pytest.mark.parametrize("name", ["paper_l12", "paper_l8", "paper_l24"])
 def test_paper_operating_points(name):
-    """K = 3 drafts of 12 or 8 tokens at T = 0.4 over a 32k vocabulary (the paper's Table 2 settings),
+    """K = 3 drafts of 12, 8 or 24 tokens at T = 0.4 over a 32k vocabulary (the paper's Table 2 settings and
+    the longest draft of its sweep over L),
     as a batch of 6 prompts so that several chains share the machine."""
     cfg = workloads.with_batch(workloads.CONFIGS[name], 6)
     inp = workloads.make_inputs(cfg, device="cuda")
