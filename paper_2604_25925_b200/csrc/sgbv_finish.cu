@@ -157,13 +157,12 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
     }
     if (lane == 31) sh_warp[wid] = incl;
     __syncthreads();
-    double cum = incl - local;
-    for (int w = 0; w < wid; ++w) cum += sh_warp[w];
-    if (relative) {  // the target is given as a fraction of the total of all tiles
-        double total = 0.0;
-        for (int w = 0; w < (nthreads >> 5); ++w) total += sh_warp[w];
-        target *= total;
-    }
+    // the warps' totals: every warp adds up those of the warps before it (and all of them) with a butterfly
+    // over its lanes instead of one after the other
+    const double wv = lane < (nthreads >> 5) ? sh_warp[lane] : 0.0;
+    const double cum0 = incl - local + warp_sum(lane < wid ? wv : 0.0);
+    if (relative) target *= warp_sum(wv);  // the target is given as a fraction of the total of all tiles
+    double cum = cum0;
     int first = INT_MAX, lastpos = -1;
     double base = 0.0;
     for (int t = t0; t < t1; ++t) {
@@ -258,15 +257,17 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             for (int e = 0; e < 4; ++e) {
                 const int t = t0 + lane + 32 * e;
                 const bool in = t < s.ntiles;
+                // the two extra arrays are fetched whether or not the row has them (c < 1), so that the
+                // fetches do not wait for the row's record; what they hold otherwise is dropped below
                 w4[e] = in ? wp[t] : 0.0f;
-                d4[e] = (in && aux) ? dp[t] : 0.0f;
-                m4[e] = (in && aux) ? mp[t] : 0.0f;
+                d4[e] = in ? dp[t] : 0.0f;
+                m4[e] = in ? mp[t] : 0.0f;
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 sw += (double)w4[e];
-                sd += (double)d4[e];
-                sm += (double)m4[e];
+                sd += aux ? (double)d4[e] : 0.0;
+                sm += aux ? (double)m4[e] : 0.0;
             }
         }
         sw = warp_sum(sw);
@@ -423,9 +424,9 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const double W = W_s[kk * g + tau];
         if (W > 0.0) {
             const float *wp = ws.wpart + r * s.ntiles;
+            const RowInfo ri = ws.rows[r];  // fetched while the tile is being located
             locate_tile(wp, nullptr, s.ntiles, us * W, false, sh_i, sh_d, sh_warp);
             const int sel = sh_i[2];
-            const RowInfo ri = ws.rows[r];
             const T *zp = zp_all + (((size_t)b * K + kk) * g + tau) * s.V;
             const int x0 = sel * kTile, x1 = min(s.V, x0 + kTile);
             auto wfun = [&](int x) {
