@@ -222,7 +222,8 @@ def main():
 
     cfg = workloads.get_config(args.workload)
     set_bytes = cfg.logit_bytes()
-    nsets = int(max(2, math.ceil(2.2 * L2_BYTES / set_bytes)))
+    # enough input sets to exceed twice the L2; capped for toy shapes, whose line then says that they stay in L2
+    nsets = int(min(512, max(2, math.ceil(2.2 * L2_BYTES / set_bytes))))
     est_ms = max(0.02, set_bytes / 2.5e9)                  # rough step time for choosing defaults
     steps = args.steps if args.steps is not None else int(max(20, min(50000, 4000.0 / est_ms)))
     warmup = args.warmup if args.warmup is not None else max(3, min(50, steps // 10))
@@ -296,7 +297,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": describe(cfg),
                        "l2": f"{nsets} rotating input sets of {set_bytes / 1e6:.1f} MB "
-                             f"({nsets * set_bytes / 1e6:.0f} MB total, L2 is 126 MB)",
+                             f"({nsets * set_bytes / 1e6:.0f} MB total, L2 is 126 MB)"
+                             + ("" if nsets * set_bytes >= 2 * L2_BYTES else ": NOT larger than L2, no flush"),
                        "per_rank_batch": cfg.B},
             "hbm_gbs_step": ab["step"] / (ms_step * 1e-3) / 1e9,
             "algorithmic_bytes_per_step": ab["step"],

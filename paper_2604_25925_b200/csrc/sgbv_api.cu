@@ -71,6 +71,9 @@ struct DeviceBuffers {
     size_t scratch_bytes = 0;
     void *stage = nullptr;
     size_t stage_bytes = 0;
+    // ratio words of the scratch that the last call left holding the "not published yet" pattern
+    const void *preset_ptr = nullptr;
+    size_t preset_words = 0;
 };
 DeviceBuffers g_buf[kMaxDevices];
 std::mutex g_mu;
@@ -123,6 +126,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     L.s = make_shape(B, K, gamma, V, temperature);
     const Carve c = carve(L.s);
     unsigned char *base = nullptr;
+    int own_dev = -1;  // >= 0: the scratch is the library's own (nobody else writes to it between calls)
     if (workspace) {
         if (workspace_bytes < c.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
         base = (unsigned char *)workspace;
@@ -133,6 +137,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total);
         if (rc != SGBV_OK) return rc;
         base = (unsigned char *)g_buf[dev].scratch;
+        own_dev = dev;
     }
     L.ws.rows = (RowInfo *)(base + c.rows);
     L.ws.part = (float *)(base + c.part);
@@ -164,8 +169,19 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     // error word itself; the two-sweep kernels set status bits with atomics, so those start at zero
     bool fused = g_opt_path != 1 && fused_supported(L);
     L.ws.prestatus = nullptr;
-    int n1 = fused ? launch_fused(L, L.ws.error) : 0;
+    // The row walk of the fused kernel needs its ratio words preset.  The finishing kernel puts the pattern
+    // back after use, so on the library's own scratch a call that follows one of the same layout finds them
+    // ready; any other call in between writes elsewhere into the scratch and voids that.
+    const size_t ratio_words = (size_t)B * K * gamma;
+    if (own_dev >= 0) {
+        std::lock_guard<std::mutex> lock(g_mu);
+        L.ratio_preset = g_buf[own_dev].preset_ptr == (const void *)L.ws.ratio && g_buf[own_dev].preset_words == ratio_words;
+        g_buf[own_dev].preset_ptr = nullptr;
+    }
+    bool walked_rows = false;
+    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows) : 0;
     if (n1 < 0) return n1;
+    L.ws.ratio_used = (n1 > 0 && walked_rows) ? 1 : 0;
     if (n1 == 0) {
         if (g_opt_path == 2) return SGBV_ERR_SHAPE;
         fused = false;
@@ -177,6 +193,11 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     }
     int n2 = launch_finish(L);
     if (n2 < 0) return n2;
+    if (own_dev >= 0 && L.ws.ratio_used) {
+        std::lock_guard<std::mutex> lock(g_mu);
+        g_buf[own_dev].preset_ptr = L.ws.ratio;
+        g_buf[own_dev].preset_words = ratio_words;
+    }
     t_last_launches = n1 + n2;
     t_last_kernel = fused ? "fused_chain_kernel" : "otreduce_kernel";
     return SGBV_OK;

@@ -38,6 +38,7 @@ struct Workspace {
     float *mpart;       // [B*K*gamma][ntiles]: sum of eq (c - t)^2 Q(t)                    (c < 1)
     double *ratio;      // [B*K*gamma]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel);
                         // preset to a NaN pattern before each launch, which reads as "not published yet"
+    int ratio_used;     // the streaming kernel walked rows: the finishing kernel puts the NaN pattern back
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory
     double *h;          // [B][K][gamma]
@@ -162,6 +163,7 @@ struct Launch {
     cudaStream_t stream;
     cudaEvent_t ev_begin = nullptr;  // optional: recorded around the dominant kernel
     cudaEvent_t ev_end = nullptr;
+    bool ratio_preset = false;       // ws.ratio already holds the NaN pattern (left by the previous call)
 };
 
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
@@ -169,7 +171,8 @@ int launch_finish(const Launch &L);   // weights, scan, extra token
 bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0
-int launch_fused(const Launch &L, int *error_flag);
+// *walked_rows: the kernel used (and consumed the preset of) ws.ratio
+int launch_fused(const Launch &L, int *error_flag, bool *walked_rows);
 void fused_set_options(int cluster, int stages, int max_clusters, int occupancy, int walk);
 
 }  // namespace sgbv

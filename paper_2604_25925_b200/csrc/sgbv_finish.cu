@@ -222,6 +222,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __shared__ float sh_redf[kMaxWarps];
     __shared__ int sh_pick[2];
     __shared__ int sh_i[4];
+    __shared__ unsigned sh_or[2];
     __shared__ double sh_d[2];
 
     const int b = blockIdx.x;
@@ -240,6 +241,11 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();  // the staged tokens and uniforms are read by other threads than those that fetched them
     const bool lost = *ws.error != 0;  // a bounded wait expired upstream: nothing can be trusted
+    // the streaming kernel has consumed the "not published yet" pattern of this batch row's ratio words:
+    // put it back, so that the next call on this scratch area need not clear them first
+    if (ws.ratio_used)
+        for (int n = tid; n < KG; n += nthreads)
+            reinterpret_cast<unsigned long long *>(ws.ratio)[(size_t)b * KG + n] = ~0ull;
     int myflags = ws.prestatus ? ws.prestatus[b] : 0;
 
     // ---- cell sums of every row (k,i), one warp per row, first warps first; the token work of step 0
@@ -371,26 +377,30 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // ---- 2. scan (Algorithm 1), warp 0 ---------------------------------------------------------
     if (wid == 0) {
-        // All state lives in registers, as bit sets over the lengths 1..gamma (bit i-1 = length i).
-        // Lane l owns drafts l and l + 32: pass = the lengths whose Bernoulli trial succeeds (eta < h),
-        // rej = the lengths at which the draft entered H.  A draft's walk over i = tau+1..gamma does not
+        // The state is bit sets over the lengths 1..gamma (bit i-1 = length i): pass (shared memory, left by
+        // the weights above) = the lengths whose Bernoulli trial succeeds (eta < h); rej (registers, lane l
+        // owns drafts l and l + 32) = the lengths at which the draft entered H.  A draft's walk over i = tau+1..gamma does not
         // depend on its own progress (the start is fixed when the draft is entered, H only holds earlier
         // drafts), so it is evaluated for all lengths at once: the accepted length is the largest one in
         // the range whose trial passes and whose sub-block is not in H.
         auto low = [](int l) { return l >= 64 ? ~0ull : (1ull << l) - 1ull; };  // lengths 1..l
-        const unsigned long long pass0 = lane < K ? pass_s[lane] : 0ull, pass1 = lane + 32 < K ? pass_s[lane + 32] : 0ull;
         unsigned long long rej0 = 0, rej1 = 0;
         int tau = 0, f = -1;
         for (int k = 0; k < K; ++k) {
-            const unsigned long long passk = __shfl_sync(0xffffffffu, k < 32 ? pass0 : pass1, k & 31);
+            const unsigned long long passk = pass_s[k];
             // common prefix of draft k with this lane's drafts; only earlier drafts can be in H
             const int l0 = (lane < k) ? lcp_s[k * K + lane] : 0;
             const int l1 = (lane + 32 < k) ? lcp_s[k * K + lane + 32] : 0;
             // lengths at which an earlier draft with the same prefix of that length entered H
             const unsigned long long mine = (rej0 & low(l0)) | (rej1 & low(l1));
-            const unsigned long long inH =
-                ((unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)(mine >> 32)) << 32) |
-                (unsigned long long)__reduce_or_sync(0xffffffffu, (unsigned)mine);
+            // union over the lanes, through shared memory
+            if (lane == 0) sh_or[0] = sh_or[1] = 0u;
+            __syncwarp();
+            if ((unsigned)mine) atomicOr(&sh_or[0], (unsigned)mine);
+            if ((unsigned)(mine >> 32)) atomicOr(&sh_or[1], (unsigned)(mine >> 32));
+            __syncwarp();
+            const unsigned long long inH = ((unsigned long long)sh_or[1] << 32) | (unsigned long long)sh_or[0];
+            __syncwarp();
             const unsigned long long range = low(g) & ~low(tau);  // lengths tau+1..gamma
             const unsigned long long acc = passk & ~inH & range;
             const unsigned long long rejk = range & ~acc;

@@ -805,7 +805,7 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     }
     const long units = plan.row_mode ? (long)fp.nchains * L.s.gamma : (long)fp.nchains;  // what the clusters share out
     if (clusters > units) clusters = (int)units;
-    if (plan.row_mode &&
+    if (plan.row_mode && !L.ratio_preset &&
         cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
         return SGBV_ERR_CUDA;
     cfg.gridDim = dim3(clusters * plan.cluster);
@@ -863,7 +863,8 @@ bool fused_supported(const Launch &L) {
     return slice_cells(cells_of(L.s.V), kMaxCluster) * kCell <= kMaxNch * kChunk;
 }
 
-int launch_fused(const Launch &L, int *error_flag) {
+int launch_fused(const Launch &L, int *error_flag, bool *walked_rows) {
+    *walked_rows = false;
     const Shape &s = L.s;
     const size_t esz = L.dtype == SGBV_DTYPE_BF16 ? 2 : 4;
     const int cells = cells_of(s.V);
@@ -907,6 +908,7 @@ int launch_fused(const Launch &L, int *error_flag) {
     plan.stages = S;
     plan.smem = (size_t)S * stage_bytes + sizeof(Control);
     plan.grid_clusters = g_opt_max_clusters;
+    *walked_rows = plan.row_mode != 0;
     return L.dtype == SGBV_DTYPE_BF16 ? launch_t<uint16_t>(L, plan, error_flag) : launch_t<float>(L, plan, error_flag);
 }
 

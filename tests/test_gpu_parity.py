@@ -289,6 +289,36 @@ def test_degenerate_and_flagged_rows():
     assert (out.tokens[2:5].cpu().numpy() == -1).all() and (out.accept_len[2:5].cpu().numpy() == -1).all()
 
 
+def test_repeated_calls_on_the_library_scratch_match_calls_on_a_fresh_workspace():
+    """The row walk's "not published yet" words are cleared by a memset on a caller's workspace, but on the
+    library's own scratch they are put back by the finishing kernel for the next call of the same layout.
+    Sequences of calls (same shape repeated, another shape in between) must give what a fresh workspace gives."""
+    row_cfg = workloads.with_batch(workloads.CONFIGS["paper_l8"], 2)
+    other_cfg = workloads.VerifyConfig("other", B=16, K=4, gamma=4, V=8192, alpha=0.85, seed=31)
+    sets = [workloads.make_inputs(row_cfg, device="cuda", set_index=i) for i in range(4)]
+    other = workloads.make_inputs(other_cfg, device="cuda")
+
+    def fresh(inp):
+        ws = torch.empty(binding.workspace_bytes(inp.cfg.B, inp.cfg.K, inp.cfg.gamma, inp.cfg.V) + 256,
+                         dtype=torch.uint8, device="cuda")
+        ws.fill_(0x5a)
+        off = (-ws.data_ptr()) % 256
+        return binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                      inp.cfg.temperature, workspace=ws[off:off + ws.numel() - 256])
+
+    order = [sets[0], sets[1], sets[1], other, sets[2], sets[3], other, other, sets[0]]
+    for inp in order:
+        got = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                     inp.cfg.temperature)
+        want = fresh(inp)
+        torch.cuda.synchronize()
+        assert torch.equal(got.accept_len, want.accept_len) and torch.equal(got.draft_idx, want.draft_idx)
+        assert torch.equal(got.tokens, want.tokens) and torch.equal(got.status, want.status)
+        assert torch.equal(got.h, want.h) and torch.equal(got.resmass, want.resmass)
+    rep, _, _ = run_both(sets[2])
+    assert_parity(rep)
+
+
 def test_plain_bf16_and_host_entry_points_agree_with_extended():
     for name in ("c2",):
         cfg = workloads.CONFIGS[name]
