@@ -223,6 +223,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __shared__ int sh_pick[2];
     __shared__ int sh_i[4];
     __shared__ unsigned sh_or[2];
+    __shared__ int sh_flags;
     __shared__ double sh_d[2];
 
     const int b = blockIdx.x;
@@ -235,6 +236,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     for (int n = (tid + nthreads / 2) % nthreads; n <= KG; n += nthreads) u_s[n] = u[n];
     for (int n = tid; n < KG; n += nthreads) tok_s[n] = tok[n];
     for (int k = tid; k < K; k += nthreads) pass_s[k] = 0ull;
+    if (tid == 0) sh_flags = 0;
     // Everything above reads only the caller's inputs.  The kernel may have been scheduled while the
     // streaming kernel was still running (programmatic dependent launch): wait for it to complete
     // before touching the row records and cell sums.
@@ -246,7 +248,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     if (ws.ratio_used)
         for (int n = tid; n < KG; n += nthreads)
             reinterpret_cast<unsigned long long *>(ws.ratio)[(size_t)b * KG + n] = ~0ull;
-    int myflags = ws.prestatus ? ws.prestatus[b] : 0;
+    int myflags = (tid == 0 && ws.prestatus) ? ws.prestatus[b] : 0;
 
     // ---- cell sums of every row (k,i), one warp per row, first warps first; the token work of step 0
     //      below starts with the LAST threads, so that for small K*gamma both run side by side ----
@@ -310,25 +312,20 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         la_s[k * (g + 1) + i + 1] = ((double)zqt - (double)ri.mq) * s.inv_T - log(ri.Zq);
         lb_s[k * (g + 1) + i + 1] = ((double)zpt - (double)ri.mp) * s.inv_T - log(ri.Zp);
     }
-    // block-wide OR of the flags (these also are the barrier after the loop)
-    const int status_in = (__syncthreads_or(myflags & SGBV_STATUS_TOKEN_RANGE) ? SGBV_STATUS_TOKEN_RANGE : 0) |
-                          (__syncthreads_or(myflags & SGBV_STATUS_NONFINITE_LOGIT) ? SGBV_STATUS_NONFINITE_LOGIT : 0);
-    const bool invalid = lost || status_in != 0;
-    for (int k = tid; k < K; k += nthreads) {
-        double la = 0.0, lb = 0.0;
-        la_s[k * (g + 1)] = 0.0;
-        lb_s[k * (g + 1)] = 0.0;
-        for (int i = 1; i <= g; ++i) {
-            la += la_s[k * (g + 1) + i];
-            lb += lb_s[k * (g + 1) + i];
-            la_s[k * (g + 1) + i] = la;
-            lb_s[k * (g + 1) + i] = lb;
-        }
-    }
+    // block-wide OR of the flags (rarely any), then the barrier after the loop
+    if (myflags) atomicOr(&sh_flags, myflags);
     __syncthreads();
+    const int status_in = sh_flags & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT);
+    const bool invalid = lost || status_in != 0;
+    // la_s/lb_s[k][i+1] now hold log q_i(x_k^i), log p_i(x_k^i); every user below adds up the terms it needs
+    // itself, in the order of a running sum (at most gamma additions, and no pass and barrier of its own)
+    auto prefix = [&](const double *row, int len) {
+        double acc = 0.0;
+        for (int j = 1; j <= len; ++j) acc += row[j];
+        return acc;
+    };
 
     // ---- 1. weights ---------------------------------------------------------------------------
-    __syncthreads();
     // the float64 transcendentals of Eq. 2, one thread per (k,i) so that they run side by side
     // (the thread that fetched the row's record for step 0 still has what it needs of it); each weight
     // leaves the outcome of its trial, eta < h, as one bit for the scan
@@ -342,7 +339,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             below = ri.c < 1.0f;
         }
         const double R = W_s[n] * inv_Zq;
-        const double la = la_s[k * (g + 1) + i], lb = lb_s[k * (g + 1) + i];
+        const double la = prefix(la_s + k * (g + 1), i), lb = prefix(lb_s + k * (g + 1), i);
         const double S = exp_short(la) * R;
         ws.resmass[(size_t)b * KG + n] = invalid ? NAN : S;
         if (i >= 1) {
@@ -352,7 +349,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         }
     }
     for (int k = tid; k < K; k += nthreads) {  // the first threads, while the last ones do Eq. 2
-        const double hv = weight_full(la_s[k * (g + 1) + g], lb_s[k * (g + 1) + g], K);
+        const double hv = weight_full(prefix(la_s + k * (g + 1), g), prefix(lb_s + k * (g + 1), g), K);
         if ((double)u_s[k * g + g - 1] < hv) atomicOr(&pass_s[k], 1ull << (g - 1));
         ws.h[(size_t)b * KG + k * g + g - 1] = invalid ? NAN : hv;
     }
