@@ -10,6 +10,9 @@
 
 namespace sgbv {
 
+// Batches of at most this many rows: the finishing kernel (one CTA per row) leaves most SMs idle, so the next
+// call's streaming kernel is allowed onto them while it runs (programmatic dependent launch across calls).
+constexpr int kChainedLaunchMaxB = 16;
 constexpr int kTile = 256;         // vocabulary elements per tile (granularity of the cached partial sums)
 constexpr int kMaxK = 64;
 constexpr int kMaxGamma = 64;

@@ -226,6 +226,10 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __shared__ int sh_flags;
     __shared__ double sh_d[2];
 
+    // A kernel launched behind this one with programmatic stream serialisation (the next call's streaming
+    // kernel) may be scheduled from now on; it waits for this grid to complete before it touches memory.
+    // Only for small batches, where this grid leaves most SMs idle.
+    if (s.B <= kChainedLaunchMaxB) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads / 32;

@@ -382,6 +382,11 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
+    // Small batches: this grid is itself launched with programmatic stream serialisation, so all of the above may have run while
+    // the kernel ahead of it in the stream was still running (in a sequence of calls that is the previous
+    // call's finishing kernel, which reads the scratch that this grid is about to write).  Nothing in global
+    // memory has been touched so far; from here on that kernel has completed and its writes are visible.
+    if (s.B <= kChainedLaunchMaxB) asm volatile("griddepcontrol.wait;" ::: "memory");
     // The finishing kernel is launched with programmatic stream serialisation: let it be scheduled now
     // (it waits for this grid to complete before it reads anything this grid writes).  Not in row mode:
     // there clusters wait for one another, so no CTA of this grid may find its place on an SM taken by
@@ -779,13 +784,17 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     cfg.blockDim = dim3(kFThreads);
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = L.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = plan.cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the kernel may be scheduled before the one ahead of it in the stream has finished (it waits for it
+    // itself before it touches global memory): its launch and start-up then overlap that kernel's tail
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = L.s.B <= kChainedLaunchMaxB ? 2 : 1;  // small batches only: see kChainedLaunchMaxB
 
     int clusters = plan.grid_clusters;
     if (clusters <= 0) {
