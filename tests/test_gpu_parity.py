@@ -319,6 +319,34 @@ def test_repeated_calls_on_the_library_scratch_match_calls_on_a_fresh_workspace(
     assert_parity(rep)
 
 
+@pytest.mark.parametrize("name", ["c2", "paper_l8"])
+def test_calls_replayed_from_a_cuda_graph_give_the_eager_results(name):
+    """After a warm-up call per shape a call only enqueues kernels (the chain walk of c2, the row walk of the
+    one-prompt shape): a captured sequence of calls, replayed, must reproduce the eager outputs."""
+    cfg = workloads.CONFIGS[name]
+    sets = [workloads.make_inputs(cfg, device="cuda", set_index=i) for i in range(3)]
+    eager = [binding.sgbv_verify(i.target_logits, i.draft_logits, i.draft_tokens, i.uniforms, cfg.temperature)
+             for i in sets]
+    torch.cuda.synchronize()
+    outs = [binding.VerifyOutput(torch.full_like(e.accept_len, -7), torch.full_like(e.draft_idx, -7),
+                                 torch.full_like(e.tokens, -7)) for e in eager]
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i, o in zip(sets, outs):
+                binding.sgbv_verify(i.target_logits, i.draft_logits, i.draft_tokens, i.uniforms, cfg.temperature,
+                                    out=o)
+    for _ in range(2):
+        for o in outs:
+            o.accept_len.fill_(-7), o.draft_idx.fill_(-7), o.tokens.fill_(-7)
+        graph.replay()
+        torch.cuda.synchronize()
+        for e, o in zip(eager, outs):
+            assert torch.equal(e.accept_len, o.accept_len) and torch.equal(e.draft_idx, o.draft_idx)
+            assert torch.equal(e.tokens, o.tokens)
+
+
 def test_plain_bf16_and_host_entry_points_agree_with_extended():
     for name in ("c2",):
         cfg = workloads.CONFIGS[name]
