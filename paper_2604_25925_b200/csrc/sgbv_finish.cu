@@ -102,8 +102,9 @@ __device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun,
     }
     if (lane == 31) sh_warp[wid] = incl;
     __syncthreads();
-    double off = base;
-    for (int k = 0; k < wid; ++k) off += sh_warp[k];
+    // mass of the warps before this one: a butterfly over the lanes instead of a loop over the warps
+    const double wv = lane < (int)(blockDim.x >> 5) ? sh_warp[lane] : 0.0;
+    const double off = base + warp_sum(lane < wid ? wv : 0.0);
     double cum = off + incl - local;
 #pragma unroll
     for (int j = 0; j < kEpt; ++j) {
@@ -508,8 +509,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         }
         if (lane == 0) sh_redf[wid] = m;
         bad = __syncthreads_or(bad);
-        m = sh_redf[0];
-        for (int w = 1; w < nwarps; ++w) m = fmaxf(m, sh_redf[w]);
+        m = warp_max(lane < nwarps ? sh_redf[lane] : -INFINITY);
         if (bad || !(m > -INFINITY)) {
             flags |= SGBV_STATUS_NONFINITE_LOGIT;
         } else {
