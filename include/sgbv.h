@@ -67,7 +67,13 @@ int sgbv_workspace_bytes(int B, int K, int gamma, int V, int dtype, size_t *out_
  * The verify step on float32 logits (problem statement and Algorithm 1; Eqs. 2-4).
  * All tensor pointers are device pointers.  Scratch comes from a per-device buffer that the
  * library grows with cudaMalloc when a larger shape is first seen (so the first call of a
- * shape is not stream-capturable; later ones allocate nothing).
+ * shape is not stream-capturable; later ones allocate nothing).  Calls that use that buffer on
+ * one device must be ordered with respect to one another (one stream, or events between streams):
+ * they share it, and between two such calls of the same shape the library keeps part of it
+ * prepared for the next call.  The kernels are launched with programmatic stream serialisation:
+ * for batches of at most 16 rows the first kernel of a call may be scheduled while the kernel
+ * ahead of it in the stream is still running; it touches no global memory until that kernel has
+ * completed, so the caller sees ordinary stream order.
  */
 int sgbv_verify(const float *target_logits, const float *draft_logits, const int32_t *draft_tokens,
                 const float *uniforms, int B, int K, int gamma, int V, float temperature,
