@@ -249,11 +249,6 @@ def main():
         if rc != 0:
             raise binding.SgbvError(rc)
 
-    for i in range(warmup):
-        step(i)
-    torch.cuda.synchronize()
-    launches_per_step = binding.last_launch_count()
-
     uuid = None
     try:
         uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
@@ -261,7 +256,14 @@ def main():
         pass
     sampler = ClockSampler(uuid) if rank == 0 else None
     time.sleep(0.25)
-    nrec = min(steps, 4000)
+    # the warm-up steps run right before the timed ones (the sampler's start-up pause would let the GPU idle)
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    launches_per_step = binding.last_launch_count()
+    # event pairs around the streaming kernel on a tenth of the timed steps at most: the records sit between
+    # the two kernels of a step and between steps, where they cost the overlap that the launches otherwise have
+    nrec = max(1, min(steps // 10, 4000))
     binding.profile_begin(nrec)
     if world > 1:
         dist.barrier()
