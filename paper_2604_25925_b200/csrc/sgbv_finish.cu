@@ -15,7 +15,7 @@ namespace sgbv {
 namespace {
 
 constexpr int kMaxThreads = 1024;  // CTA size when few batch rows leave most SMs idle (the kernel is a
-constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps per row help); else 256
+constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps per row help); else 512 or 256
 constexpr int kMaxWarps = kMaxThreads / 32;
 constexpr int kTilesInSmem = 4096;  // rows up to 2^20 entries keep the bonus row's tile sums in shared memory
 constexpr int kEpt = 1;  // elements per thread inside one tile (threads beyond the tile hold none)
@@ -562,7 +562,9 @@ int run(const Launch &L) {
     // stream has finished; it waits for that kernel itself (griddepcontrol.wait) once it needs its results
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(s.B);
-    cfg.blockDim = dim3(s.B <= 148 ? kMaxThreads : kMinThreads);
+    // the largest CTA with which all batch rows are still resident at once (64 registers per thread: one CTA of
+    // 1024 threads per SM, two of 512, four of 256)
+    cfg.blockDim = dim3(s.B <= 148 ? kMaxThreads : s.B <= 296 ? 512 : kMinThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = L.stream;
     cudaLaunchAttribute attr[1];
