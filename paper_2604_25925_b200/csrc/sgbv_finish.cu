@@ -198,6 +198,32 @@ __device__ void locate_tile(const float *partials, const float *scale, int ntile
     __syncthreads();
 }
 
+// The 8 entries of a 256-entry tile that one lane takes when the row can be read in 16-byte pieces (the row starts
+// on a 16-byte boundary and V is a multiple of the entries per piece, so a piece lies inside the row or past it).
+template <typename T>
+__device__ __forceinline__ void load_tile_pieces(const T *zq, int tile, bool in, int V, int lane, float (&z)[kTile / 32]);
+template <>
+__device__ __forceinline__ void load_tile_pieces<float>(const float *zq, int tile, bool in, int V, int lane,
+                                                        float (&z)[kTile / 32]) {
+    const float ninf = -INFINITY;
+    const int xa = tile * kTile + lane * 4, xb = xa + kTile / 2;
+    const float4 a = (in && xa < V) ? __ldg(reinterpret_cast<const float4 *>(zq + xa)) : make_float4(ninf, ninf, ninf, ninf);
+    const float4 b = (in && xb < V) ? __ldg(reinterpret_cast<const float4 *>(zq + xb)) : make_float4(ninf, ninf, ninf, ninf);
+    z[0] = a.x; z[1] = a.y; z[2] = a.z; z[3] = a.w;
+    z[4] = b.x; z[5] = b.y; z[6] = b.z; z[7] = b.w;
+}
+template <>
+__device__ __forceinline__ void load_tile_pieces<uint16_t>(const uint16_t *zq, int tile, bool in, int V, int lane,
+                                                           float (&z)[kTile / 32]) {
+    const uint32_t ninf2 = 0xff80ff80u;  // two bf16 -inf
+    const int xa = tile * kTile + lane * 8;
+    const uint4 a = (in && xa < V) ? __ldg(reinterpret_cast<const uint4 *>(zq + xa)) : make_uint4(ninf2, ninf2, ninf2, ninf2);
+    z[0] = __uint_as_float(a.x << 16); z[1] = __uint_as_float(a.x & 0xffff0000u);
+    z[2] = __uint_as_float(a.y << 16); z[3] = __uint_as_float(a.y & 0xffff0000u);
+    z[4] = __uint_as_float(a.z << 16); z[5] = __uint_as_float(a.z & 0xffff0000u);
+    z[6] = __uint_as_float(a.w << 16); z[7] = __uint_as_float(a.w & 0xffff0000u);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kMaxThreads)
 finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const int32_t *__restrict__ tok_all,
@@ -462,15 +488,22 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         bool bad = false;
         float m = -INFINITY;
         constexpr int kNT = 4;  // tiles a warp has in flight
+        static_assert(kTile == 256, "a lane takes 8 entries of a tile");
+        const bool pieces = (reinterpret_cast<uintptr_t>(zq) % 16 == 0) && (s.V % (16 / (int)sizeof(T)) == 0);
         for (int tb = wid * kNT; tb < s.ntiles; tb += nwarps * kNT) {
             float z[kNT][kTile / 32];
+            if (pieces) {  // 16-byte loads
 #pragma unroll
-            for (int q = 0; q < kNT; ++q)
+                for (int q = 0; q < kNT; ++q) load_tile_pieces<T>(zq, tb + q, tb + q < s.ntiles, s.V, lane, z[q]);
+            } else {
 #pragma unroll
-                for (int e = 0; e < kTile / 32; ++e) {
-                    const int x = (tb + q) * kTile + lane + 32 * e;
-                    z[q][e] = (tb + q < s.ntiles && x < s.V) ? ld_logit(zq, x) : -INFINITY;
-                }
+                for (int q = 0; q < kNT; ++q)
+#pragma unroll
+                    for (int e = 0; e < kTile / 32; ++e) {
+                        const int x = (tb + q) * kTile + lane + 32 * e;
+                        z[q][e] = (tb + q < s.ntiles && x < s.V) ? ld_logit(zq, x) : -INFINITY;
+                    }
+            }
             // the four tiles are reduced side by side (independent shuffle chains)
             float mt[kNT], acc[kNT];
 #pragma unroll
