@@ -43,12 +43,14 @@ Carve carve(const Shape &s) {
     const size_t NR = (size_t)s.B * s.K * s.gamma;
     Carve c;
     size_t off = 0;
+    // the ratio words sit at the head, at the same place for every shape: on the library's own scratch
+    // they keep their "not published yet" pattern from call to call, whatever shapes the calls have
+    c.ratio = off;     off += align_up(kRatioWords * sizeof(double));
     c.rows = off;      off += align_up(NR * sizeof(RowInfo));
     c.part = off;      off += align_up(NR * s.nsplit * 4 * sizeof(float));
     c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.mpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
-    c.ratio = off;     off += align_up(NR * sizeof(double));
     c.bonus = off;     off += align_up((size_t)s.B * 2 * s.ntiles * sizeof(float));
     c.h = off;         off += align_up(NR * sizeof(double));
     c.resmass = off;   off += align_up(NR * sizeof(double));
@@ -71,14 +73,16 @@ struct DeviceBuffers {
     size_t scratch_bytes = 0;
     void *stage = nullptr;
     size_t stage_bytes = 0;
-    // ratio words of the scratch that the last call left holding the "not published yet" pattern
-    const void *preset_ptr = nullptr;
-    size_t preset_words = 0;
+    // the ratio words at the head of the scratch may not hold the "not published yet" pattern (a call
+    // failed between the kernel that consumes them and the one that puts them back)
+    bool ratio_dirty = false;
 };
 DeviceBuffers g_buf[kMaxDevices];
 std::mutex g_mu;
 
-int grow(void **ptr, size_t *have, size_t need) {
+// Grows a per-device buffer.  preset_head: the first bytes of a new buffer get the 0xff pattern of unpublished
+// ratio words before anyone uses it (the device is idle then).
+int grow(void **ptr, size_t *have, size_t need, size_t preset_head = 0) {
     if (*have >= need) return SGBV_OK;
     if (*ptr) {
         if (cudaDeviceSynchronize() != cudaSuccess) return SGBV_ERR_CUDA;
@@ -91,13 +95,20 @@ int grow(void **ptr, size_t *have, size_t need) {
         *ptr = nullptr;
         return SGBV_ERR_CUDA;
     }
+    if (preset_head && (cudaMemset(*ptr, 0xff, preset_head) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)) {
+        cudaGetLastError();
+        cudaFree(*ptr);
+        *ptr = nullptr;
+        return SGBV_ERR_CUDA;
+    }
     *have = need;
     return SGBV_OK;
 }
 
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
-int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_occupancy = 0, g_opt_walk = 0;
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_walk = 0, g_opt_poll_us = 0,
+    g_opt_withhold = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -134,10 +145,15 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
         std::lock_guard<std::mutex> lock(g_mu);
-        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total);
+        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total, kRatioWords * sizeof(double));
         if (rc != SGBV_OK) return rc;
         base = (unsigned char *)g_buf[dev].scratch;
         own_dev = dev;
+        // The row walk of the fused kernel needs its ratio words preset.  They sit at a fixed place, are preset
+        // when the buffer is allocated, and every finishing kernel puts the pattern back after use: whatever the
+        // order of eager calls and graph replays, a call finds them ready.  Only a call that failed half-way
+        // leaves them in doubt; the next row walk then clears them itself.
+        L.ratio_preset = !g_buf[dev].ratio_dirty;
     }
     L.ws.rows = (RowInfo *)(base + c.rows);
     L.ws.part = (float *)(base + c.part);
@@ -169,15 +185,6 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     // error word itself; the two-sweep kernels set status bits with atomics, so those start at zero
     bool fused = g_opt_path != 1 && fused_supported(L);
     L.ws.prestatus = nullptr;
-    // The row walk of the fused kernel needs its ratio words preset.  The finishing kernel puts the pattern
-    // back after use, so on the library's own scratch a call that follows one of the same layout finds them
-    // ready; any other call in between writes elsewhere into the scratch and voids that.
-    const size_t ratio_words = (size_t)B * K * gamma;
-    if (own_dev >= 0) {
-        std::lock_guard<std::mutex> lock(g_mu);
-        L.ratio_preset = g_buf[own_dev].preset_ptr == (const void *)L.ws.ratio && g_buf[own_dev].preset_words == ratio_words;
-        g_buf[own_dev].preset_ptr = nullptr;
-    }
     bool walked_rows = false;
     int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows) : 0;
     if (n1 < 0) return n1;
@@ -192,12 +199,16 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         if (n1 < 0) return n1;
     }
     int n2 = launch_finish(L);
-    if (n2 < 0) return n2;
     if (own_dev >= 0 && L.ws.ratio_used) {
+        // a walk that cleared the words itself is followed by a finishing kernel that puts them back: the
+        // doubt ends unless that kernel was not launched, or nothing ran at all (stream capture)
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        const bool capturing = cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone;
         std::lock_guard<std::mutex> lock(g_mu);
-        g_buf[own_dev].preset_ptr = L.ws.ratio;
-        g_buf[own_dev].preset_words = ratio_words;
+        if (n2 < 0) g_buf[own_dev].ratio_dirty = true;
+        else if (!capturing) g_buf[own_dev].ratio_dirty = false;
     }
+    if (n2 < 0) return n2;
     t_last_launches = n1 + n2;
     t_last_kernel = fused ? "fused_chain_kernel" : "otreduce_kernel";
     return SGBV_OK;
@@ -305,11 +316,10 @@ int sgbv_set_option(const char *name, int value) {
         if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
         g_opt_path = value;
     } else if (!strcmp(name, "cluster")) {
-        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16)
-            return SGBV_ERR_SHAPE;
+        if (value < 0 || value > 8) return SGBV_ERR_SHAPE;
         g_opt_cluster = value;
     } else if (!strcmp(name, "stages")) {
-        if (value != 0 && (value < 2 || value > 12)) return SGBV_ERR_SHAPE;
+        if (value < 0 || value > 8) return SGBV_ERR_SHAPE;
         g_opt_stages = value;
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;
@@ -317,13 +327,16 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "walk")) {
         if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
         g_opt_walk = value;
-    } else if (!strcmp(name, "occupancy")) {
-        if (value != 0 && (value < 2 || value > 4)) return SGBV_ERR_SHAPE;
-        g_opt_occupancy = value;
+    } else if (!strcmp(name, "poll_us")) {
+        if (value < 0 || value > 1000000) return SGBV_ERR_SHAPE;
+        g_opt_poll_us = value;
+    } else if (!strcmp(name, "withhold")) {
+        if (value < 0 || value > 1) return SGBV_ERR_SHAPE;
+        g_opt_withhold = value;
     } else {
         return SGBV_ERR_SHAPE;
     }
-    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_occupancy, g_opt_walk);
+    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_walk, g_opt_poll_us, g_opt_withhold);
     return SGBV_OK;
 }
 

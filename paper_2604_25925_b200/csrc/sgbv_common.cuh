@@ -13,6 +13,8 @@ namespace sgbv {
 // Batches of at most this many rows: the finishing kernel (one CTA per row) leaves most SMs idle, so the next
 // call's streaming kernel is allowed onto them while it runs (programmatic dependent launch across calls).
 constexpr int kChainedLaunchMaxB = 16;
+constexpr int kRatioWords = 256;   // ratio words at the head of the scratch: the row walk needs one per row and
+                                   // only runs while every row has a cluster of its own in one wave (<= 148)
 constexpr int kTile = 256;         // vocabulary elements per tile (granularity of the cached partial sums)
 constexpr int kMaxK = 64;
 constexpr int kMaxGamma = 64;
@@ -39,8 +41,9 @@ struct Workspace {
     float *wpart;       // [B*K*gamma][ntiles]: sum over the tile of eq * max(1 - kappa ep/eq, 0)^K
     float *dpart;       // [B*K*gamma][ntiles]: sum of max(kappa ep - eq, 0)               (c < 1)
     float *mpart;       // [B*K*gamma][ntiles]: sum of eq (c - t)^2 Q(t)                    (c < 1)
-    double *ratio;      // [B*K*gamma]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel);
-                        // preset to a NaN pattern before each launch, which reads as "not published yet"
+    double *ratio;      // [kRatioWords]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel, which
+                        // only runs when B*K*gamma <= kRatioWords); every word holds a NaN pattern ("not
+                        // published yet") whenever no call is in flight
     int ratio_used;     // the streaming kernel walked rows: the finishing kernel puts the NaN pattern back
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory
@@ -166,7 +169,7 @@ struct Launch {
     cudaStream_t stream;
     cudaEvent_t ev_begin = nullptr;  // optional: recorded around the dominant kernel
     cudaEvent_t ev_end = nullptr;
-    bool ratio_preset = false;       // ws.ratio already holds the NaN pattern (left by the previous call)
+    bool ratio_preset = false;       // ws.ratio is known to hold the NaN pattern (the library's own scratch)
 };
 
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
@@ -176,6 +179,6 @@ bool fused_supported(const Launch &L);
 // anything (the caller then takes the two-sweep path), or < 0
 // *walked_rows: the kernel used (and consumed the preset of) ws.ratio
 int launch_fused(const Launch &L, int *error_flag, bool *walked_rows);
-void fused_set_options(int cluster, int stages, int max_clusters, int occupancy, int walk);
+void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold);
 
 }  // namespace sgbv

@@ -1,43 +1,50 @@
-// Fused single-read path (steps A1-A3): one thread-block cluster walks one draft chain (b,k).
+// Fused single-read path (steps A1-A3): one thread-block cluster walks one draft chain (b,k), one
+// CTA of 32 warps per SM, the row resident in TENSOR MEMORY between the two sweeps.
 //
 // For every position i = 0..gamma-1 of the chain the cluster
-//   * streams the target row and the draft row from HBM exactly once: bulk asynchronous copies
-//     (cp.async.bulk + mbarrier transaction counts) of 2048-element chunks of both tensors into a
-//     shared-memory ring that runs ahead across rows and chains.  A warp owns the 256-element
-//     cells  warp, warp+8, warp+16, ...  of its CTA's slice.  There is no producer thread and no
-//     "stage free" barrier: once the row's exchange (below) is complete, every warp of the CTA has
-//     moved the row into registers, so its ring stages are refilled right then, by a different warp
-//     for each chunk; the copies stay large (few requests to the copy engine);
-//   * keeps the whole row pair resident in REGISTERS (each thread 8 elements of every cell) as
-//     exponentials relative to the thread's own maximum, so the second
-//     sweep of the coupling sum never re-reads memory;
+//   * streams the target row and the draft row from HBM exactly once.  CTA r of the cluster owns a
+//     contiguous slice of the vocabulary, warp w of the CTA the 256-entry cells  w, w+32, w+64, w+96
+//     of that slice.  Every warp runs its own little ring of bulk asynchronous copies
+//     (cp.async.bulk + mbarrier transaction counts; one cell of both tensors per slot): the warp that
+//     consumes a slot refills it itself, so the load path needs no block-wide synchronisation and
+//     runs ahead across rows and chains;
+//   * first sweep: a thread takes 8 (target, draft) pairs of a cell, turns them into exponentials
+//     relative to its own maxima of that cell (the maximum maps to exactly 1) and parks them in
+//     tensor memory (tcgen05.st; each warp owns 64 of the 512 columns of its lane quarter, 256 KB per
+//     SM in all = 32,768 pairs), keeping only the cell's maximum and sum in registers;
 //   * exchanges (max, sum-exp) partials in two levels: the warps of a CTA leave theirs in shared
 //     memory and the last one to arrive combines them and PUSHES one partial per CTA into every
 //     CTA's shared memory with asynchronous distributed-shared-memory stores that complete on the
 //     receiver's mbarrier; a warp goes on as soon as all CTA partials of the row have landed.
 //     There is no block-wide or cluster-wide barrier inside the row loop;
-//   * runs the second sweep from registers and writes one partial sum per cell.
+//   * second sweep: reads the exponentials back from tensor memory (tcgen05.ld) and writes one
+//     partial sum of the coupling terms per cell.  Shared memory is never read twice and the
+//     registers hold no row data between the sweeps, which is what lets 32 warps share the SM.
 // The joint likelihood ratio c_i = p(x^i)/q(x^i) is carried as a running product by one thread per
 // CTA, which computes c_{i+1} right after the statistics of row i and arms the next row's exchange
-// with it, a whole row before it is needed.  Two CTAs of 256 threads share an SM (different clusters).  The finishing
-// kernel (weights, scan, extra token) consumes the cell sums.
+// with it, a whole row before it is needed.  The finishing kernel (weights, scan, extra token)
+// consumes the cell sums.
 //
-// Every wait on an mbarrier is bounded; on expiry the warp records an error flag and keeps
-// executing the protocol, so a lost copy cannot hang the kernel.
+// Every wait on an mbarrier or on a word in global memory is bounded; on expiry the warp records
+// an error flag and keeps executing the protocol, so a lost copy cannot hang the kernel, and the
+// tensor memory is released on every path.
+#include <algorithm>
+#include <mutex>
+
 #include "sgbv_common.cuh"
 
 namespace sgbv {
 
 namespace {
 
-constexpr int kFThreads = 256;
+constexpr int kFThreads = 1024;
 constexpr int kFWarps = kFThreads / 32;
-constexpr int kCell = kTile;               // 256 contiguous elements: one warp's share of a chunk
-constexpr int kChunk = kFWarps * kCell;    // 2048 elements: one cell of every warp
-constexpr int kMaxNch = 5;                 // cells per warp: what one thread can hold in registers (5 x 8 pairs)
-constexpr int kMaxStages = 12;             // ring depth
-constexpr int kRowBars = 16;               // "row has landed" barriers: more than the rows the ring can hold
-constexpr int kMaxCluster = 16;
+constexpr int kCell = kTile;               // 256 contiguous entries: the unit a warp works on
+constexpr int kCellsPerWarp = 4;           // 4 cells x 16 columns = the 64 tensor-memory columns of a warp
+constexpr int kCtaCells = kFWarps * kCellsPerWarp;  // 128 cells = 32,768 entries of a row per CTA
+constexpr int kTmemCols = 512;             // all of the SM's tensor memory (one CTA per SM)
+constexpr int kMaxSlots = 8;               // ring depth per warp
+constexpr int kMaxCluster = 8;             // portable cluster size
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 constexpr uint32_t kSuspendNs = 20000u;               // longest single suspension inside a wait
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
@@ -49,11 +56,12 @@ struct FusedParams {
     Shape s;
     Workspace ws;
     int cluster;      // CTAs per cluster
-    int slice_len;    // vocabulary elements per CTA (multiple of kCell)
-    int stages;       // ring depth
+    int slice_cells;  // cells of a row per CTA (at most kCtaCells)
+    int slots;        // ring depth per warp
     int nchains;      // B*K
-    int row_mode;     // 0: a cluster walks whole chains; 1: a cluster walks single rows (see the kernel)
     int *error_flag;  // set to 1 if a bounded wait expired
+    long long poll_limit;  // cycles a poll of a published ratio may take (row walk)
+    int withhold;     // failure-detection test: the first row of every chain does not publish its ratio
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -92,13 +100,16 @@ __device__ __forceinline__ bool mbar_test_suspend(uint64_t *bar, uint32_t parity
         : "memory");
     return ok != 0;
 }
-// Bounded wait: returns false if the phase did not complete within about a second.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    if (mbar_test(bar, parity)) return true;
+// Bounded wait: sets `gave_up` if the phase did not complete within about a second.  A thread that has given
+// up once only tests from then on, so that the time a failing kernel takes stays bounded.
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, bool &gave_up) {
+    if (mbar_test(bar, parity) || gave_up) return;
     const long long t0 = clock64();
     while (!mbar_test_suspend(bar, parity))
-        if (clock64() - t0 > kWaitLimitCycles) return false;
-    return true;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            gave_up = true;
+            return;
+        }
 }
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -139,18 +150,58 @@ __device__ __forceinline__ float rcp(float x) {
     return y;
 }
 
+// ---- tensor memory --------------------------------------------------------------------------------
+// One warp allocates all columns for the CTA (the address lands in shared memory), every warp then
+// reads and writes only the lanes of its own quarter (warp index mod 4) and its own columns.
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 16 consecutive columns of this thread's lane: the 8 target and the 8 draft exponentials of a cell
+__device__ __forceinline__ void tmem_st_cell(uint32_t taddr, const float2 (&a)[4], const float2 (&b)[4]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "f"(a[0].x), "f"(a[0].y), "f"(a[1].x), "f"(a[1].y), "f"(a[2].x), "f"(a[2].y), "f"(a[3].x), "f"(a[3].y), "f"(b[0].x),
+        "f"(b[0].y), "f"(b[1].x), "f"(b[1].y), "f"(b[2].x), "f"(b[2].y), "f"(b[3].x), "f"(b[3].y)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_cell(uint32_t taddr, float2 (&a)[4], float2 (&b)[4]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=f"(a[0].x), "=f"(a[0].y), "=f"(a[1].x), "=f"(a[1].y), "=f"(a[2].x), "=f"(a[2].y), "=f"(a[3].x), "=f"(a[3].y),
+          "=f"(b[0].x), "=f"(b[0].y), "=f"(b[1].x), "=f"(b[1].y), "=f"(b[2].x), "=f"(b[2].y), "=f"(b[3].x), "=f"(b[3].y)
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Waits for this thread's tensor-memory loads; the loaded registers pass through the statement, so that no
+// use of them can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_wait_ld(float2 (&a)[4], float2 (&b)[4]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+f"(a[0].x), "+f"(a[0].y), "+f"(a[1].x), "+f"(a[1].y), "+f"(a[2].x), "+f"(a[2].y), "+f"(a[3].x), "+f"(a[3].y),
+                   "+f"(b[0].x), "+f"(b[0].y), "+f"(b[1].x), "+f"(b[1].y), "+f"(b[2].x), "+f"(b[2].y), "+f"(b[3].x), "+f"(b[3].y)
+                 :
+                 : "memory");
+}
+
 // ---- shared memory layout ------------------------------------------------------------------------
-// [ring: stages x (chunk of zq, chunk of zp)] [Control]
+// [rings: 32 warps x slots x (cell of zq, cell of zp)] [full barriers: 32 warps x slots] [Control]
 struct Control {
-    uint64_t rowbar[kRowBars];           // by row of the walk (mod 16): "all chunks of the row have landed"
     uint64_t xbar[2];                    // by row parity: "all partials of the row (chain walk: and c_i) are here"
     uint64_t cbar[2];                    // by row parity, row walk only: "c_i is here"
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
     // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
     float4 wslots[2][kFWarps];
-    int arrivals;                        // partials left in wslots so far, over all rows (never reset)
     float4 slots[2][kMaxCluster];
     double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
+    int arrivals;                        // partials left in wslots so far, over all rows (never reset)
+    uint32_t tmem_base;                  // address of the allocated tensor memory
 };
 
 // Reads this lane's 8 elements of one cell of one tensor from the ring.
@@ -212,16 +263,14 @@ __device__ __forceinline__ float2 ipow2(float2 r, int K) {
     return acc;
 }
 
-// Sums N values over the 32 lanes of a warp at once ("transposed" butterfly: at every step a lane
-// hands half of its values to its partner and keeps the other half).  P = N rounded up to a power
-// of two (<= 16).  On return v[0] of lane l is the warp total of value number owner_index<P>(l).
+// Sums P values over the 32 lanes of a warp at once ("transposed" butterfly: at every step a lane
+// hands half of its values to its partner and keeps the other half).  P is a power of two (<= 4).
+// On return v[0] of lane l is the warp total of value number owner_index<P>(l).
 template <int P>
 __device__ __forceinline__ int owner_index(int lane) {
     int idx = 0;
     if (P >= 2) idx += (lane & 16) ? P / 2 : 0;
     if (P >= 4) idx += (lane & 8) ? P / 4 : 0;
-    if (P >= 8) idx += (lane & 4) ? P / 8 : 0;
-    if (P >= 16) idx += (lane & 2) ? P / 16 : 0;
     return idx;
 }
 template <int P>
@@ -240,26 +289,28 @@ __device__ __forceinline__ void warp_sum_multi(float (&v)[P], int lane) {
     for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
 }
 
-// Second sweep over the register-resident row, two vocabulary entries per instruction (f32x2).
-// eq/ep are exponentials relative to the THREAD's maxima; kt = kappa * (fp_t / fq_t) makes
-// c p(x)/q(x) = kt * ep/eq;  scale_w, scale_d convert the thread's sums to row-max units.
-// nj = number of cells this warp holds; the output pointers address this warp's first cell, its
-// cells are kFWarps apart.  Per cell:
+// What the second sweep needs of a row, the same for every cell.
+struct RowScalars {
+    float rq, rp;   // row maxima (0 where the row has none)
+    float kappa;    // c_i Zq / Zp: makes c p(x)/q(x) = kappa ep/eq in row-max units
+    float c;        // c_i
+    float scale;    // log2(e) / T
+};
+
+// Second sweep over the warp's cells, read back from tensor memory, two vocabulary entries per
+// instruction (f32x2).  eq/ep are exponentials relative to the THREAD's maxima of the cell (mq[j],
+// mp[j]); kt = kappa * (fp / fq) makes c p(x)/q(x) = kt * ep/eq, where fq, fp move the thread's
+// units to row-max units.  Per cell:
 //   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
 //   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
 //   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
-template <int NCH, int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(const float2 (&eq)[NCH][4], const float2 (&ep)[NCH][4], float kt,
-                                          float scale_w, float scale_d, float c, int K, int lane, int nj,
-                                          float *wpart, float *dpart, float *mpart) {
-    constexpr int NV = kAux ? 3 * NCH : NCH;
-    constexpr int P = NV <= 1 ? 1 : NV <= 2 ? 2 : NV <= 4 ? 4 : NV <= 8 ? 8 : 16;
-    static_assert(NV <= 16, "at most 16 sums per thread");
-    float sums[P];
-#pragma unroll
-    for (int k = 0; k < P; ++k) sums[k] = 0.0f;
-    const float v1 = 1.0f - c;
-    const float2 nkt = splat(-kt), nv1 = splat(-v1);
+// The output pointers address this warp's first cell; its cells are kFWarps apart.
+template <int KT, bool kAux>
+__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCellsPerWarp], const float (&mp)[kCellsPerWarp],
+                                          const RowScalars &rs, int K, int lane, int ncw, float *wpart, float *dpart,
+                                          float *mpart) {
+    const float v1 = 1.0f - rs.c;
+    const float2 nv1 = splat(-v1);
     // Horner coefficients of Q: (t+1) (1-c)^t, t = 1..K-2 (uniform over the row)
     float2 coef[KT > 2 ? KT - 2 : 1];
     if (kAux && KT > 2) {
@@ -270,14 +321,40 @@ __device__ __forceinline__ void sweep_two(const float2 (&eq)[NCH][4], const floa
             coef[t - 1] = splat((float)(t + 1) * vj);
         }
     }
+    float wsum[kCellsPerWarp];
 #pragma unroll
-    for (int j = 0; j < NCH; ++j) {
-        if (j >= nj) break;  // warp-uniform
+    for (int j = 0; j < kCellsPerWarp; ++j) wsum[j] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kCellsPerWarp; ++j) {
+        if (j >= ncw) break;  // warp-uniform
+        float2 eq[4], ep[4];
+        tmem_ld_cell(taddr + 16u * (uint32_t)j, eq, ep);
+        // thread units -> row units
+        const float fq = (mq[j] > -INFINITY) ? ex2((mq[j] - rs.rq) * rs.scale) : 0.0f;
+        const float fp = (mp[j] > -INFINITY) ? ex2((mp[j] - rs.rp) * rs.scale) : 0.0f;
+        // equal factors (identical rows above all) must give kappa itself: p = q everywhere then leaves an
+        // exactly zero residual
+        float kt = (fp == fq) ? rs.kappa : rs.kappa * fp * rcp(fq);
+        float scale_w = fq, scale_d = fq;
+        const bool tiny = !(fq > 1e-30f);
+        tmem_wait_ld(eq, ep);
+        if (__any_sync(0xffffffffu, tiny)) {
+            // a thread whose share of the target row underflows (or nearly so, which would
+            // overflow kt): its q is 0 in row units, its weights vanish, and max(c p - q, 0) = c p
+            if (tiny) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) eq[e] = splat(0.0f);
+                kt = 1.0f;
+                scale_w = 0.0f;
+                scale_d = rs.kappa * fp;
+            }
+        }
+        const float2 nkt = splat(-kt);
         float2 sw = splat(0.0f), sd = splat(0.0f), sm = splat(0.0f);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float2 q = eq[j][e];
-            const float2 diff = __ffma2_rn(nkt, ep[j][e], q);  // q - c p, thread units
+            const float2 q = eq[e];
+            const float2 diff = __ffma2_rn(nkt, ep[e], q);  // q - c p, thread units
             const float2 pos = make_float2(fmaxf(diff.x, 0.0f), fmaxf(diff.y, 0.0f));
             if (KT == 1) sw = __fadd2_rn(sw, pos);
             if (KT == 1 && !kAux) continue;
@@ -306,30 +383,25 @@ __device__ __forceinline__ void sweep_two(const float2 (&eq)[NCH][4], const floa
                 sm = __ffma2_rn(__fmul2_rn(q, __fmul2_rn(ct, ct)), acc, sm);
             }
         }
-        sums[j] = (sw.x + sw.y) * scale_w;
+        wsum[j] = (sw.x + sw.y) * scale_w;
         if (kAux) {
-            sums[NCH + j] = (sd.x + sd.y) * scale_d;
-            sums[2 * NCH + j] = (sm.x + sm.y) * scale_w;
+            // the two extra sums of the cell leave right away (they are rare: rows with c < 1)
+            float aux[2] = {(sd.x + sd.y) * scale_d, (sm.x + sm.y) * scale_w};
+            warp_sum_multi<2>(aux, lane);
+            if ((lane & 15) == 0) ((lane & 16) ? mpart : dpart)[j * kFWarps] = aux[0];
         }
     }
-    warp_sum_multi<P>(sums, lane);
+    warp_sum_multi<kCellsPerWarp>(wsum, lane);
     // the lane that owns value number idx (and has the low lane bits clear) stores it
-    const int idx = owner_index<P>(lane);
-    constexpr int kLowMask = P >= 16 ? 1 : P >= 8 ? 3 : P >= 4 ? 7 : P >= 2 ? 15 : 31;
-    if ((lane & kLowMask) == 0 && idx < NV) {
-        const int jj = kAux ? idx % NCH : idx, which = kAux ? idx / NCH : 0;
-        if (jj < nj) {
-            float *dst = which == 0 ? wpart : which == 1 ? dpart : mpart;
-            dst[jj * kFWarps] = sums[0];
-        }
-    }
+    const int idx = owner_index<kCellsPerWarp>(lane);
+    if ((lane & 7) == 0 && idx < ncw) wpart[idx * kFWarps] = wsum[0];
 }
 
-template <int NCH, bool kAux>
-__device__ __forceinline__ void sweep_two_dispatch(const float2 (&eq)[NCH][4], const float2 (&ep)[NCH][4], float kt,
-                                                   float scale_w, float scale_d, float c, int K, int lane, int nj,
-                                                   float *wpart, float *dpart, float *mpart) {
-#define SGBV_SWEEP(KT) sweep_two<NCH, KT, kAux>(eq, ep, kt, scale_w, scale_d, c, K, lane, nj, wpart, dpart, mpart)
+template <bool kAux>
+__device__ __forceinline__ void sweep_two_dispatch(uint32_t taddr, const float (&mq)[kCellsPerWarp],
+                                                   const float (&mp)[kCellsPerWarp], const RowScalars &rs, int K, int lane,
+                                                   int ncw, float *wpart, float *dpart, float *mpart) {
+#define SGBV_SWEEP(KT) sweep_two<KT, kAux>(taddr, mq, mp, rs, K, lane, ncw, wpart, dpart, mpart)
     switch (K) {
         case 1: SGBV_SWEEP(1); break;
         case 2: SGBV_SWEEP(2); break;
@@ -341,10 +413,8 @@ __device__ __forceinline__ void sweep_two_dispatch(const float2 (&eq)[NCH][4], c
 #undef SGBV_SWEEP
 }
 
-// OCC = CTAs of this kernel that share an SM (2, 3 or 4): more co-resident CTAs hide more of each
-// other's exchange and pipeline latency, but leave each thread fewer registers, hence fewer cells.
-template <typename T, int NCH, int OCC, bool kRow>
-__global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const FusedParams p) {
+template <typename T, bool kRow>
+__global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -352,33 +422,38 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     const int rank = (int)cluster_ctarank();
     const int cid = blockIdx.x / C;
     const int G = gridDim.x / C;
-    const int S = p.stages;
-    constexpr int kCellBytes = kCell * (int)sizeof(T);
-    constexpr int kChunkBytes = kChunk * (int)sizeof(T);
-    constexpr int kStageBytes = 2 * kChunkBytes;  // one chunk of zq, then the same chunk of zp
-    unsigned char *ring = smem;
-    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)S * kStageBytes);
+    const int NS = p.slots;
+    constexpr int kHalfBytes = kCell * (int)sizeof(T);  // one tensor's cell
+    constexpr int kSlotBytes = 2 * kHalfBytes;          // the cell of zq, then the same cell of zp
+    unsigned char *ring = smem + (size_t)warp * NS * kSlotBytes;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)kFWarps * NS * kSlotBytes) + warp * NS;
+    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * NS * (kSlotBytes + 8));
 
-    // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 8, ...
-    const int x_begin = rank * p.slice_len;
-    const int cta_len = max(0, min(s.V, x_begin + p.slice_len) - x_begin);
-    const int ncells_valid = (cta_len + kCell - 1) / kCell;
-    const int nj = ncells_valid > warp ? (ncells_valid - warp + kFWarps - 1) / kFWarps : 0;
-    const int nchunks = (ncells_valid + kFWarps - 1) / kFWarps;  // chunks per row of this CTA
-    const int first_cell = x_begin / kCell + warp;
-    const int x_warp = x_begin + warp * kCell;  // first element of this warp's first cell
+    // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 32, ...
+    const int cell_begin = rank * p.slice_cells;
+    const int ncells_cta = max(0, min(s.ntiles, cell_begin + p.slice_cells) - cell_begin);
+    const int ncw = ncells_cta > warp ? (ncells_cta - warp + kFWarps - 1) / kFWarps : 0;  // cells of this warp per row
+    const int first_cell = cell_begin + warp;
+    const int x_warp = first_cell * kCell;  // first element of this warp's first cell
 
     if (tid == 0) {
-        // one arrival (with its byte count) per chunk of the row
-        for (int i = 0; i < kRowBars; ++i) mbar_init(&ctl->rowbar[i], (uint32_t)max(nchunks, 1));
         mbar_init(&ctl->xbar[0], 1);
         mbar_init(&ctl->xbar[1], 1);
         mbar_init(&ctl->cbar[0], 1);
         mbar_init(&ctl->cbar[1], 1);
         ctl->arrivals = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (lane == 0)
+        for (int k = 0; k < NS; ++k) mbar_init(&full[k], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
+    tmem_fence_before();
     __syncthreads();
+    tmem_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    // lanes of this warp's quarter, and its 64 columns
+    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(warp >> 2) * (16u * kCellsPerWarp);
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
@@ -406,39 +481,49 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
     const long total_rows = (long)p.nchains * s.gamma;
     const int nrows = row_mode ? (int)((total_rows - cid + G - 1) / G)
                                : ((p.nchains - cid + G - 1) / G) * s.gamma;  // rows this cluster walks
-    const int total_loads = nrows * nchunks;    // chunk pairs this CTA loads
     const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
     bool timed_out = false;
 
-    // Loads are numbered in consumption order: chunk m of this CTA's walk is chunk m % nchunks of
-    // row m / nchunks and lands in ring stage m % S.  issue_chunk is stateless, so any lane can issue
-    // any chunk: lanes of one warp issue the chunks of a whole row side by side.  All chunks of walk
-    // position `row` complete on the barrier of that row (one wait per row instead of one per chunk).
-    auto issue_at = [&](size_t bkc, int pos, int jc, int stage, int row) {
-        const int x0 = x_begin + jc * kChunk;  // first element of the chunk
-        const T *zq = reinterpret_cast<const T *>(p.zq) + (bkc * (s.gamma + 1) + pos) * s.V + x0;
-        const T *zp = reinterpret_cast<const T *>(p.zp) + (bkc * s.gamma + pos) * s.V + x0;
-        const uint32_t bytes = (uint32_t)min(kChunk, cta_len - jc * kChunk) * (uint32_t)sizeof(T);
-        unsigned char *dst = ring + (size_t)stage * kStageBytes;
-        uint64_t *bar = &ctl->rowbar[row & (kRowBars - 1)];
-        mbar_expect_tx(bar, 2 * bytes);
-        bulk_load(dst, zq, bytes, bar);
-        bulk_load(dst + kChunkBytes, zp, bytes, bar);
-    };
-    auto issue_chunk = [&](int m) {
-        const int row = m / nchunks;  // position in the walk
-        if (row_mode) {
-            const long u = (long)cid + (long)row * G;
-            issue_at((size_t)(u / s.gamma), (int)(u % s.gamma), m - row * nchunks, m % S, row);
-        } else {
-            const int chain = row / s.gamma;
-            issue_at((size_t)cid + (size_t)chain * G, row - chain * s.gamma, m - row * nchunks, m % S, row);
+    // ---- this warp's copy ring --------------------------------------------------------------------
+    // Cell loads are numbered in consumption order: load m is cell m % ncw of walk position m / ncw and
+    // lands in slot m % NS.  The cursor below (kept by every lane, used by lane 0) names the next load.
+    // A warp that has given up on a wait issues no further loads and waits for those in flight only.
+    const long total_loads = (long)nrows * ncw;
+    long ld_m = 0;
+    int in_flight = 0;  // loads issued and not consumed yet
+    int ld_j = 0, ld_i = row_mode ? cid % s.gamma : 0, ld_slot = 0;
+    size_t ld_bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
+    auto issue_next = [&]() {
+        if (ld_m < total_loads && !timed_out) {
+            ++in_flight;
+            if (lane == 0) {
+                const int cell = first_cell + ld_j * kFWarps;
+                const size_t x0 = (size_t)cell * kCell;
+                const T *zq = reinterpret_cast<const T *>(p.zq) + (ld_bk * (s.gamma + 1) + ld_i) * s.V + x0;
+                const T *zp = reinterpret_cast<const T *>(p.zp) + (ld_bk * s.gamma + ld_i) * s.V + x0;
+                const uint32_t bytes = (uint32_t)min(kCell, s.V - (int)x0) * (uint32_t)sizeof(T);
+                unsigned char *dst = ring + (size_t)ld_slot * kSlotBytes;
+                mbar_expect_tx(&full[ld_slot], 2 * bytes);
+                bulk_load(dst, zq, bytes, &full[ld_slot]);
+                bulk_load(dst + kHalfBytes, zp, bytes, &full[ld_slot]);
+            }
+            ++ld_m;
+            if (++ld_slot == NS) ld_slot = 0;
+            if (++ld_j == ncw) {  // on to the next row of the walk
+                ld_j = 0;
+                ld_bk += step_bk;
+                ld_i += step_i;
+                if (ld_i >= s.gamma) {
+                    ld_i -= s.gamma;
+                    ld_bk += wrap_bk;
+                }
+            }
         }
     };
-    // Fill the ring in two goes: the first row's chunks now, so that they do not share the memory system
-    // with later rows' chunks and the first row can start as early as possible; the rest of the ring once
-    // the first row has landed (see the load phase of the first row).
-    if (warp == 0 && lane < nchunks && lane < total_loads) issue_chunk(lane);
+    if (ncw > 0)
+        for (int k = 0; k < NS; ++k) issue_next();
+    int c_slot = 0;           // slot of the next cell to consume
+    uint32_t c_phase = 0;     // parity of that slot's barrier
 
     // The chain thread of this CTA carries c_i and fetches the token logits one row
     // ahead: tok_next is the token of the next row of the walk.
@@ -450,323 +535,316 @@ __global__ void __launch_bounds__(kFThreads, OCC) fused_chain_kernel(const Fused
         mbar_expect_tx(&ctl->xbar[0], xbytes);
     }
 
-    int st = 0;
-    int n = 0;  // row number in this cluster's walk
     size_t bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
     int i = row_mode ? cid % s.gamma : 0;
-    {
-        for (; n < nrows; ++n) {
-            const size_t r = bk * s.gamma + i;
-            const int par = n & 1;
-            const uint32_t xph = (uint32_t)(n >> 1) & 1u;
+    for (int n = 0; n < nrows; ++n) {
+        const size_t r = bk * s.gamma + i;
+        const int par = n & 1;
+        const uint32_t xph = (uint32_t)(n >> 1) & 1u;
 
-            // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
-            float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
-            if (chain_thread) {
-                if (row_mode) mbar_expect_tx(&ctl->xbar[par], xbytes);  // the exchange does not wait for c_i here
-                int t = tok_next;
-                if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
-                zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
-                zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
-                if (n + 1 < nrows) {
-                    size_t bk_n = bk + step_bk;
-                    int i_n = i + step_i;
-                    if (i_n >= s.gamma) {
-                        i_n -= s.gamma;
-                        bk_n += wrap_bk;
-                    }
-                    tok_next = p.tok[bk_n * s.gamma + i_n];
+        // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
+        float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
+        if (chain_thread) {
+            if (row_mode) mbar_expect_tx(&ctl->xbar[par], xbytes);  // the exchange does not wait for c_i here
+            int t = tok_next;
+            if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
+            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
+            zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
+            if (n + 1 < nrows) {
+                size_t bk_n = bk + step_bk;
+                int i_n = i + step_i;
+                if (i_n >= s.gamma) {
+                    i_n -= s.gamma;
+                    bk_n += wrap_bk;
                 }
+                tok_next = p.tok[bk_n * s.gamma + i_n];
             }
+        }
 
-            // ---- first sweep, part 1: ring -> registers, running maxima of this thread ---------------
-            float2 eq[NCH][4], ep[NCH][4];  // two neighbouring vocabulary entries per register pair
-            float mq = -INFINITY, mp = -INFINITY;
-            if (nchunks > 0 && !mbar_wait(&ctl->rowbar[n & (kRowBars - 1)], (uint32_t)(n / kRowBars) & 1u)) timed_out = true;
-            if (n == 0 && warp == 0 && lane >= nchunks && lane < S && lane < total_loads) issue_chunk(lane);  // rest of the ring
-            // all loads first, so that their latencies overlap; the maxima afterwards
+        // ---- first sweep: ring -> exponentials in tensor memory, maximum and sum of every cell --------
+        float mq[kCellsPerWarp], mp[kCellsPerWarp], sq[kCellsPerWarp], sp[kCellsPerWarp];
 #pragma unroll
-            for (int j = 0; j < NCH; ++j) {
-                if (j < nchunks) {  // uniform over the CTA
-                    if (j < nj) {  // warp-uniform
-                        const unsigned char *base = ring + (size_t)st * kStageBytes + warp * kCellBytes;
-                        read_cell<T>(base, lane, eq[j]);
-                        read_cell<T>(base + kChunkBytes, lane, ep[j]);
-                    }
-                    if (++st == S) st = 0;
+        for (int j = 0; j < kCellsPerWarp; ++j) {
+            mq[j] = mp[j] = -INFINITY;
+            sq[j] = sp[j] = 0.0f;
+        }
+#pragma unroll
+        for (int j = 0; j < kCellsPerWarp; ++j) {
+            if (j < ncw) {  // warp-uniform
+                if (in_flight > 0) {
+                    mbar_wait(&full[c_slot], c_phase, timed_out);
+                    timed_out = __any_sync(0xffffffffu, timed_out);
+                    --in_flight;
                 }
-            }
-#pragma unroll
-            for (int j = 0; j < NCH; ++j) {
-                if (j < nj) {
-                    const int cell_x = x_warp + j * kChunk;
-                    if (cell_x + kCell > s.V) {  // the row ends inside this cell
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[j][e].x = ep[j][e].x = -INFINITY;
-                            if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[j][e].y = ep[j][e].y = -INFINITY;
-                        }
-                    }
+                float2 eq[4], ep[4];
+                const unsigned char *base = ring + (size_t)c_slot * kSlotBytes;
+                read_cell<T>(base, lane, eq);
+                read_cell<T>(base + kHalfBytes, lane, ep);
+                const int cell_x = x_warp + j * kFWarps * kCell;
+                if (cell_x + kCell > s.V) {  // the row ends inside this cell
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        mq = max3(mq, eq[j][e].x, eq[j][e].y);
-                        mp = max3(mp, ep[j][e].x, ep[j][e].y);
+                        if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[e].x = ep[e].x = -INFINITY;
+                        if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[e].y = ep[e].y = -INFINITY;
                     }
                 }
-            }
-            // reference points of this thread's exponentials: its own maxima (0 if it saw only -inf);
-            // the maximum itself maps to exactly 1, so point-mass rows stay exact
-            const bool has_q = mq > -INFINITY, has_p = mp > -INFINITY;
-            const float bq = has_q ? mq : 0.0f;
-            const float bp = has_p ? mp : 0.0f;
-
-            // ---- first sweep, part 2: exponentials in place, sums ----------------------------------
-            float2 sq2 = splat(0.0f), sp2 = splat(0.0f);
-            const float2 nbq = splat(-bq), nbp = splat(-bp), sc2 = splat(s.scale);
+                float m1 = -INFINITY, m2 = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < NCH; ++j) {
-                if (j < nj) {
+                for (int e = 0; e < 4; ++e) {
+                    m1 = max3(m1, eq[e].x, eq[e].y);
+                    m2 = max3(m2, ep[e].x, ep[e].y);
+                }
+                // every lane holds its share of the slot in registers now: refill it with the cell NS further on
+                __syncwarp();
+                issue_next();
+                if (++c_slot == NS) {
+                    c_slot = 0;
+                    c_phase ^= 1u;
+                }
+                // reference points of this thread's exponentials: its own maxima of the cell (0 if it saw
+                // only -inf); the maximum itself maps to exactly 1, so point-mass rows stay exact
+                const float bq = (m1 > -INFINITY) ? m1 : 0.0f;
+                const float bp = (m2 > -INFINITY) ? m2 : 0.0f;
+                const float2 nbq = splat(-bq), nbp = splat(-bp), sc2 = splat(s.scale);
+                float2 sq2 = splat(0.0f), sp2 = splat(0.0f);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 aq = __fmul2_rn(__fadd2_rn(eq[j][e], nbq), sc2);
-                        const float2 ap = __fmul2_rn(__fadd2_rn(ep[j][e], nbp), sc2);
-                        eq[j][e] = make_float2(ex2(aq.x), ex2(aq.y));
-                        ep[j][e] = make_float2(ex2(ap.x), ex2(ap.y));
-                        sq2 = __fadd2_rn(sq2, eq[j][e]);
-                        sp2 = __fadd2_rn(sp2, ep[j][e]);
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    const float2 aq = __fmul2_rn(__fadd2_rn(eq[e], nbq), sc2);
+                    const float2 ap = __fmul2_rn(__fadd2_rn(ep[e], nbp), sc2);
+                    eq[e] = make_float2(ex2(aq.x), ex2(aq.y));
+                    ep[e] = make_float2(ex2(ap.x), ex2(ap.y));
+                    sq2 = __fadd2_rn(sq2, eq[e]);
+                    sp2 = __fadd2_rn(sp2, ep[e]);
                 }
+                tmem_st_cell(taddr + 16u * (uint32_t)j, eq, ep);
+                mq[j] = m1;
+                mp[j] = m2;
+                sq[j] = sq2.x + sq2.y;
+                sp[j] = sp2.x + sp2.y;
             }
-            float sq = sq2.x + sq2.y, sp = sp2.x + sp2.y;
-            // warp partials relative to the warp's maxima, pushed to every CTA
-            const float bqw = warp_max_redux(has_q ? bq : -INFINITY), bpw = warp_max_redux(has_p ? bp : -INFINITY);
-            const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
-            sq = warp_sum(has_q ? sq * ex2((bq - rqw) * s.scale) : 0.0f);
-            sp = warp_sum(has_p ? sp * ex2((bp - rpw) * s.scale) : 0.0f);
-            // two-level exchange: the warp partials meet in this CTA's shared memory; the warp that
-            // arrives last combines them (fixed order) and pushes ONE partial per CTA to every CTA
-            bool last_warp = false;
-            if (lane == 0) {
-                ctl->wslots[par][warp] = make_float4(bqw, sq, bpw, sp);
-                __threadfence_block();
-                last_warp = atomicAdd(&ctl->arrivals, 1) + 1 == kFWarps * (n + 1);
-            }
-            if (__shfl_sync(0xffffffffu, last_warp, 0)) {
-                __threadfence_block();
-                const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-                const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
-                const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
-                const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
-                const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
-                if (lane < C)
-                    push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
-            }
+        }
+        tmem_wait_st();
 
-            // Ring refill.  Once all warps of this CTA have left their partials, all of them have turned
-            // this row's ring stages into registers, and the stages can take the chunks S ahead.  Warps
-            // 1, 2, ... take one chunk each, so the copy requests are issued side by side; a warp that
-            // sees the condition already now does it while it would otherwise wait for the exchange,
-            // the others do it after the exchange (whose completion implies the condition).
-            auto do_refill = [&]() {
-                const int jc = (warp + kFWarps - 1) % kFWarps;  // warp 1 -> chunk 0, ..., warp 0 -> chunk 7
-                if (lane == 0 && jc < nchunks && n * nchunks + jc + S < total_loads) {
-                    // chunk jc of this row sits in stage (st - nchunks + jc) mod S; the chunk that replaces it
-                    // is S chunks further along the walk: a few rows on, maybe in the next chain
-                    int stage = st - nchunks + jc;
-                    while (stage < 0) stage += S;
-                    int jc2 = jc + S, pos = i, row2 = n;
-                    size_t bkc = bk;
-                    while (jc2 >= nchunks) {  // one step of the walk per row
-                        jc2 -= nchunks;
-                        ++row2;
-                        bkc += step_bk;
-                        pos += step_i;
-                        if (pos >= s.gamma) {
-                            pos -= s.gamma;
-                            bkc += wrap_bk;
-                        }
-                    }
-                    issue_at(bkc, pos, jc2, stage, row2);
-                }
-            };
-            bool refilled = false;
-            {
-                int seen = 0;
-                if (lane == 0) seen = *reinterpret_cast<volatile int *>(&ctl->arrivals);
-                if (__shfl_sync(0xffffffffu, seen, 0) >= kFWarps * (n + 1)) {
-                    do_refill();
-                    refilled = true;
-                }
+        // ---- this thread's partial of the row: cell sums moved to its maximum over the cells ---------
+        float mqt = mq[0], mpt = mp[0];
+#pragma unroll
+        for (int j = 1; j < kCellsPerWarp; ++j) {
+            mqt = fmaxf(mqt, mq[j]);
+            mpt = fmaxf(mpt, mp[j]);
+        }
+        const bool has_q = mqt > -INFINITY, has_p = mpt > -INFINITY;
+        const float bqt = has_q ? mqt : 0.0f, bpt = has_p ? mpt : 0.0f;
+        float sqt = 0.0f, spt = 0.0f;
+#pragma unroll
+        for (int j = 0; j < kCellsPerWarp; ++j) {
+            if (j < ncw) {  // a cell without a finite entry has sum 0 and factor 2^-inf = 0
+                sqt = fmaf(sq[j], ex2((mq[j] - bqt) * s.scale), sqt);
+                spt = fmaf(sp[j], ex2((mp[j] - bpt) * s.scale), spt);
             }
-            if (!mbar_wait(&ctl->xbar[par], xph)) timed_out = true;
+        }
+        // warp partials relative to the warp's maxima
+        const float bqw = warp_max_redux(has_q ? bqt : -INFINITY), bpw = warp_max_redux(has_p ? bpt : -INFINITY);
+        const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
+        sqt = warp_sum(has_q ? sqt * ex2((bqt - rqw) * s.scale) : 0.0f);
+        spt = warp_sum(has_p ? spt * ex2((bpt - rpw) * s.scale) : 0.0f);
+        // two-level exchange: the warp partials meet in this CTA's shared memory; the warp that
+        // arrives last combines them (fixed order) and pushes ONE partial per CTA to every CTA
+        bool last_warp = false;
+        if (lane == 0) {
+            ctl->wslots[par][warp] = make_float4(bqw, sqt, bpw, spt);
+            __threadfence_block();
+            last_warp = atomicAdd(&ctl->arrivals, 1) + 1 == kFWarps * (n + 1);
+        }
+        if (__shfl_sync(0xffffffffu, last_warp, 0)) {
+            __threadfence_block();
+            const float4 v = ctl->wslots[par][lane];  // one warp partial per lane
+            const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
+            const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
+            const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
+            const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
+            if (lane < C)
+                push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
+        }
+        mbar_wait(&ctl->xbar[par], xph, timed_out);
+        timed_out = __any_sync(0xffffffffu, timed_out);  // the warp gives up as one
 
-            // Refill (see do_refill above) if it could not be done while waiting.
-            if (!refilled) do_refill();
-
-            // ---- row statistics: every warp combines the CTA partials, in the same order -------------
-            const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-            const float bq_row = warp_max_redux(cv.x), bp_row = warp_max_redux(cv.z);
-            const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
-            const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
-            const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
-            // the ratio p_i(tok_i)/q_i(tok_i) of this row (chain thread)
-            auto token_ratio = [&]() {
-                const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
-                const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
-                return exp2_short(lp - lq) * (double)(Zq / Zp);
-            };
-            double cd;
-            if (row_mode) {
-                // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
-                // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
-                // NaN (a row that produces one is flagged invalid anyway).
-                if (chain_thread && rank == 0 && i + 1 < s.gamma) {
-                    double ratio = token_ratio();
-                    if (ratio != ratio) ratio = 0.0;
-                    *reinterpret_cast<volatile double *>(p.ws.ratio + r) = ratio;
-                }
-                // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
-                // butterfly over the lanes).  Those rows are walked by other clusters at about the same
-                // time and publish right after their own statistics, which do not depend on c: no chain of
-                // waits forms.  Every lane of the last warp polls one of them.  Bounded waits.
-                if (warp == kFWarps - 1) {
-                    double cprod = 1.0;
-                    const size_t r0 = bk * s.gamma;
-                    for (int j0 = 0; j0 < i; j0 += 32) {
-                        double v = 1.0;
-                        if (j0 + lane < i) {
-                            const volatile double *word =
-                                reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
-                            v = *word;
-                            if (v != v) {
-                                const long long t0 = clock64();
-                                while ((v = *word) != v) {
-                                    if (clock64() - t0 > kWaitLimitCycles) {
-                                        timed_out = true;
-                                        v = 0.0;
-                                        break;
-                                    }
+        // ---- row statistics: every warp combines the CTA partials, in the same order -------------
+        const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+        const float bq_row = warp_max_redux(cv.x), bp_row = warp_max_redux(cv.z);
+        const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
+        const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
+        const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
+        // the ratio p_i(tok_i)/q_i(tok_i) of this row (chain thread)
+        auto token_ratio = [&]() {
+            const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
+            const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
+            return exp2_short(lp - lq) * (double)(Zq / Zp);
+        };
+        double cd;
+        if (row_mode) {
+            // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
+            // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
+            // NaN (a row that produces one is flagged invalid anyway).
+            if (chain_thread && rank == 0 && i + 1 < s.gamma && !(p.withhold && i == 0)) {
+                double ratio = token_ratio();
+                if (ratio != ratio) ratio = 0.0;
+                *reinterpret_cast<volatile double *>(p.ws.ratio + r) = ratio;
+            }
+            // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
+            // butterfly over the lanes).  Those rows are walked by other clusters at about the same
+            // time and publish right after their own statistics, which do not depend on c: no chain of
+            // waits forms.  Every lane of the last warp polls one of them.  Bounded waits.
+            if (warp == kFWarps - 1) {
+                double cprod = 1.0;
+                const size_t r0 = bk * s.gamma;
+                for (int j0 = 0; j0 < i; j0 += 32) {
+                    double v = 1.0;
+                    if (j0 + lane < i) {
+                        const volatile double *word =
+                            reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
+                        v = *word;
+                        if (v != v && timed_out) v = 0.0;
+                        if (v != v) {
+                            const long long t0 = clock64();
+                            while ((v = *word) != v) {
+                                if (clock64() - t0 > p.poll_limit) {
+                                    timed_out = true;
+                                    v = 0.0;
+                                    break;
                                 }
                             }
                         }
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) v *= __shfl_xor_sync(0xffffffffu, v, o);
-                        cprod *= v;
                     }
-                    if (lane == 0) {
-                        ctl->c[par] = cprod;
-                        mbar_arrive(&ctl->cbar[par]);  // c_i is there
-                    }
-                }
-                if (!mbar_wait(&ctl->cbar[par], xph)) timed_out = true;
-                cd = ctl->c[par];
-            } else {
-                cd = ctl->c[par];
-                if (chain_thread && n + 1 < nrows) {
-                    // c of the next row of the walk: c_{i+1} = c_i ratio, or 1 at the start of the next
-                    // chain; publishing it arms the next row's exchange
-                    ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * token_ratio() : 1.0;
-                    mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
-                }
-            }
-            const float c = (float)cd;
-            const float kappa = (float)(cd * (double)(Zq / Zp));
-
-            if (tid == 0) {
-                if (rank == 0) {
-                    // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
-                    // -inf only has Z = 0
-                    const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
-                                     !(bq_row < INFINITY) || !(bp_row < INFINITY);
-                    RowInfo ri;
-                    ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
-                    ri.pad_ = 0;
-                    ri.Zq = (double)Zq;
-                    ri.Zp = (double)Zp;
-                    ri.mq = bq_row;
-                    ri.mp = bp_row;
-                    ri.kappa = kappa;
-                    ri.c = c;
-                    p.ws.rows[r] = ri;
-                }
-            }
-
-            // thread units -> row units
-            const float fq = has_q ? ex2((bq - rq_row) * s.scale) : 0.0f;
-            const float fp = has_p ? ex2((bp - rp_row) * s.scale) : 0.0f;
-            float kt = kappa * fp / fq;
-            float scale_w = fq, scale_d = fq;
-            if (__any_sync(0xffffffffu, !(fq > 1e-30f))) {
-                // a thread whose share of the target row underflows (or nearly so, which would
-                // overflow kt): its q is 0 in row units, its weights vanish, and max(c p - q, 0) = c p
-                if (!(fq > 1e-30f)) {
 #pragma unroll
-                    for (int j = 0; j < NCH; ++j)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) eq[j][e] = splat(0.0f);
-                    kt = 1.0f;
-                    scale_w = 0.0f;
-                    scale_d = kappa * fp;
+                    for (int o = 16; o > 0; o >>= 1) v *= __shfl_xor_sync(0xffffffffu, v, o);
+                    cprod *= v;
+                }
+                if (lane == 0) {
+                    ctl->c[par] = cprod;
+                    mbar_arrive(&ctl->cbar[par]);  // c_i is there
                 }
             }
-
-            // ---- second sweep from registers ---------------------------------------------------------
-            float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
-                  *mpp = p.ws.mpart + r * s.ntiles + first_cell;
-            if (c < 1.0f)
-                sweep_two_dispatch<NCH, true>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
-            else
-                sweep_two_dispatch<NCH, false>(eq, ep, kt, scale_w, scale_d, c, s.K, lane, nj, wp, dp, mpp);
-
-            // one step of the walk
-            bk += step_bk;
-            i += step_i;
-            if (i >= s.gamma) {
-                i -= s.gamma;
-                bk += wrap_bk;
+            mbar_wait(&ctl->cbar[par], xph, timed_out);
+            timed_out = __any_sync(0xffffffffu, timed_out);
+            cd = ctl->c[par];
+        } else {
+            cd = ctl->c[par];
+            if (chain_thread && n + 1 < nrows) {
+                // c of the next row of the walk: c_{i+1} = c_i ratio, or 1 at the start of the next
+                // chain; publishing it arms the next row's exchange
+                ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * token_ratio() : 1.0;
+                mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
             }
+        }
+        RowScalars rs;
+        rs.rq = rq_row;
+        rs.rp = rp_row;
+        rs.c = (float)cd;
+        rs.kappa = (float)(cd * (double)(Zq / Zp));
+        rs.scale = s.scale;
+
+        if (tid == 0 && rank == 0) {
+            // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
+            // -inf only has Z = 0
+            const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
+                             !(bq_row < INFINITY) || !(bp_row < INFINITY);
+            RowInfo ri;
+            ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
+            ri.pad_ = 0;
+            ri.Zq = (double)Zq;
+            ri.Zp = (double)Zp;
+            ri.mq = bq_row;
+            ri.mp = bp_row;
+            ri.kappa = rs.kappa;
+            ri.c = rs.c;
+            p.ws.rows[r] = ri;
+        }
+
+        // ---- second sweep from tensor memory ----------------------------------------------------------
+        float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
+              *mpp = p.ws.mpart + r * s.ntiles + first_cell;
+        if (rs.c < 1.0f)
+            sweep_two_dispatch<true>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+        else
+            sweep_two_dispatch<false>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+
+        // one step of the walk
+        bk += step_bk;
+        i += step_i;
+        if (i >= s.gamma) {
+            i -= s.gamma;
+            bk += wrap_bk;
         }
     }
     if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(p.error_flag, 1);
     cluster_arrive();  // no CTA leaves while a neighbour may still write into its slots
     cluster_wait();
+    tmem_fence_before();
+    __syncthreads();  // every warp of this CTA is done with the tensor memory
+    if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
 struct Plan {
-    int cluster, slice_len, nch, occ, stages, grid_clusters, row_mode;
+    int cluster, slice_cells, slots, grid_clusters, row_mode;
     size_t smem;
 };
 
 int g_opt_cluster = 0;     // 0 = automatic
-int g_opt_stages = 0;
+int g_opt_slots = 0;
 int g_opt_max_clusters = 0;
-int g_opt_occupancy = 0;
 int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
+int g_opt_poll_us = 0;     // 0 = about a second
+int g_opt_withhold = 0;
 
-constexpr int kSmemPerSm = 228 * 1024;     // shared memory of one SM
-constexpr int kSmemReserved = 1024;        // per resident CTA, taken by the system
-constexpr int kSms = 148;
-// cells per warp that fit the registers when OCC CTAs share an SM
-int max_nch(int occ) { return occ <= 2 ? kMaxNch : occ == 3 ? 2 : 1; }
+constexpr int kSmemPerCta = 227 * 1024;    // largest dynamic shared memory of one CTA
+constexpr int kDevices = 64;
+std::mutex g_plan_mu;      // guards the per-device caches below
 
-int cells_of(int V) { return (V + kCell - 1) / kCell; }
-int slice_cells(int cells, int C) { return (cells + C - 1) / C; }
+size_t slot_bytes(int dtype) { return 2 * (size_t)kCell * (dtype == SGBV_DTYPE_BF16 ? 2 : 4); }
+size_t smem_bytes(int dtype, int slots) { return (size_t)kFWarps * slots * (slot_bytes(dtype) + 8) + sizeof(Control); }
+int slice_cells_of(int cells, int C) { return (cells + C - 1) / C; }
 
-template <typename T, int NCH, int OCC, bool kRow>
-int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
-    auto kernel = fused_chain_kernel<T, NCH, OCC, kRow>;
-    static bool attr_done[64];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SGBV_ERR_CUDA;
+template <typename T, bool kRow>
+cudaError_t prepare(int dev) {
+    static bool attr_done[kDevices];
     if (!attr_done[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kSmemPerSm / OCC - kSmemReserved) != cudaSuccess)
-            return SGBV_ERR_CUDA;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
-            return SGBV_ERR_CUDA;
+        cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
+        if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
+    return cudaSuccess;
+}
+
+// Clusters of C CTAs of this kernel that the device runs side by side (queried once per configuration).
+template <typename T, bool kRow>
+int resident_clusters(int dev, int C, int slots, size_t smem) {
+    static int cached[kDevices][kMaxCluster + 1][kMaxSlots + 1];
+    int &slot = cached[dev][C][slots];
+    if (slot == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.blockDim = dim3(kFThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.gridDim = dim3(C * (148 / C));
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = C;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int nmax = 0;
+        if (cudaOccupancyMaxActiveClusters(&nmax, fused_chain_kernel<T, kRow>, &cfg) != cudaSuccess || nmax < 1) {
+            cudaGetLastError();
+            return 0;
+        }
+        slot = nmax;
+    }
+    return slot;
+}
+
+template <typename T, bool kRow>
+int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) {
     FusedParams fp;
     fp.zq = L.zq;
     fp.zp = L.zp;
@@ -774,11 +852,12 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     fp.s = L.s;
     fp.ws = L.ws;
     fp.cluster = plan.cluster;
-    fp.slice_len = plan.slice_len;
-    fp.stages = plan.stages;
+    fp.slice_cells = plan.slice_cells;
+    fp.slots = plan.slots;
     fp.nchains = L.s.B * L.s.K;
-    fp.row_mode = plan.row_mode;
     fp.error_flag = error_flag;
+    fp.poll_limit = g_opt_poll_us > 0 ? (long long)g_opt_poll_us * 2000ll : kWaitLimitCycles;
+    fp.withhold = g_opt_withhold;
 
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kFThreads);
@@ -795,31 +874,12 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = L.s.B <= kChainedLaunchMaxB ? 2 : 1;  // small batches only: see kChainedLaunchMaxB
-
-    int clusters = plan.grid_clusters;
-    if (clusters <= 0) {
-        // persistent grid: as many clusters as can be co-resident (queried once per configuration)
-        static int cached[64][kMaxCluster + 1][kMaxStages + 1];  // [device][cluster size][stages]
-        int &slot = cached[dev][plan.cluster][plan.stages];
-        if (slot == 0) {
-            cfg.gridDim = dim3(plan.cluster * (OCC * kSms / plan.cluster));
-            int nmax = 0;
-            if (cudaOccupancyMaxActiveClusters(&nmax, kernel, &cfg) != cudaSuccess || nmax < 1) {
-                cudaGetLastError();
-                return 0;  // this cluster shape cannot be scheduled here: nothing launched
-            }
-            slot = nmax;
-        }
-        clusters = slot;
-    }
-    const long units = plan.row_mode ? (long)fp.nchains * L.s.gamma : (long)fp.nchains;  // what the clusters share out
-    if (clusters > units) clusters = (int)units;
-    if (plan.row_mode && !L.ratio_preset &&
+    cfg.gridDim = dim3(clusters * plan.cluster);
+    if (kRow && !L.ratio_preset &&
         cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
         return SGBV_ERR_CUDA;
-    cfg.gridDim = dim3(clusters * plan.cluster);
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, fp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_chain_kernel<T, kRow>, fp);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -828,97 +888,91 @@ int launch_nch(const Launch &L, const Plan &plan, int *error_flag) {
     return 1;
 }
 
+// Chooses the cluster size and the walk, then launches.  Returns launches, 0 if declined, or < 0.
 template <typename T>
-int launch_t(const Launch &L, const Plan &plan, int *error_flag) {
-    if (plan.row_mode) {  // the row walk exists for two CTAs per SM
-        if (plan.occ != 2) return SGBV_ERR_SHAPE;
-        switch (plan.nch) {
-            case 1: return launch_nch<T, 1, 2, true>(L, plan, error_flag);
-            case 2: return launch_nch<T, 2, 2, true>(L, plan, error_flag);
-            case 3: return launch_nch<T, 3, 2, true>(L, plan, error_flag);
-            case 4: return launch_nch<T, 4, 2, true>(L, plan, error_flag);
-            case 5: return launch_nch<T, 5, 2, true>(L, plan, error_flag);
-            default: return SGBV_ERR_SHAPE;
-        }
+int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
+    const Shape &s = L.s;
+    const int cells = s.ntiles;
+    const long nchains = (long)s.B * s.K, units = nchains * s.gamma;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDevices) return SGBV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_plan_mu);
+    if (prepare<T, false>(dev) != cudaSuccess || prepare<T, true>(dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SGBV_ERR_CUDA;
     }
-    switch (plan.occ * 10 + plan.nch) {
-        case 21: return launch_nch<T, 1, 2, false>(L, plan, error_flag);
-        case 22: return launch_nch<T, 2, 2, false>(L, plan, error_flag);
-        case 23: return launch_nch<T, 3, 2, false>(L, plan, error_flag);
-        case 24: return launch_nch<T, 4, 2, false>(L, plan, error_flag);
-        case 25: return launch_nch<T, 5, 2, false>(L, plan, error_flag);
-        case 31: return launch_nch<T, 1, 3, false>(L, plan, error_flag);
-        case 32: return launch_nch<T, 2, 3, false>(L, plan, error_flag);
-        case 41: return launch_nch<T, 1, 4, false>(L, plan, error_flag);
-        default: return SGBV_ERR_SHAPE;
+    Plan plan;
+    // ring depth: what fits beside the control block, at most the default (deeper rings keep more bytes
+    // in flight than the memory system rewards)
+    const int max_slots = (int)std::min<size_t>(kMaxSlots, (kSmemPerCta - sizeof(Control)) / ((size_t)kFWarps * (slot_bytes(L.dtype) + 8)));
+    int slots = g_opt_slots ? g_opt_slots : (L.dtype == SGBV_DTYPE_BF16 ? 6 : 3);
+    if (slots > max_slots) {
+        if (g_opt_slots) return SGBV_ERR_SHAPE;
+        slots = max_slots;
     }
+    plan.slots = slots;
+    plan.smem = smem_bytes(L.dtype, slots);
+    int Cmin = (cells + kCtaCells - 1) / kCtaCells;  // smallest cluster whose slices fit the tensor memory
+    if (Cmin > kMaxCluster) return 0;
+    auto fits = [&](int C) { return C >= Cmin && C <= kMaxCluster; };
+    auto resident = [&](int C, bool row) {
+        return row ? resident_clusters<T, true>(dev, C, plan.slots, plan.smem)
+                   : resident_clusters<T, false>(dev, C, plan.slots, plan.smem);
+    };
+    // Few units of work: spread each over more CTAs (at least half the warps keep a cell) while all of them
+    // still run side by side.
+    auto widen = [&](long n_units, bool row) {
+        int C = Cmin;
+        while (2 * C <= kMaxCluster && cells >= C * kFWarps && n_units <= resident(2 * C, row)) C *= 2;
+        return C;
+    };
+    int C = g_opt_cluster ? g_opt_cluster : widen(nchains, false);
+    // Few rows in all: when every ROW can have a cluster of its own in one wave, share out single rows
+    // instead of chains (their only coupling, c_i, is looked up), so that the gamma rows of a chain run
+    // side by side instead of one after the other.
+    const int Crow = g_opt_cluster ? g_opt_cluster : widen(units, true);
+    plan.row_mode = 0;
+    if (g_opt_walk == 2 && units > kRatioWords) return SGBV_ERR_SHAPE;  // one ratio word per row, and only so many
+    if (s.gamma > 1 && fits(Crow) && units <= kRatioWords &&
+        (g_opt_walk == 2 || (g_opt_walk == 0 && units <= resident(Crow, true)))) {
+        plan.row_mode = 1;
+        C = Crow;
+    }
+    if (!fits(C)) return g_opt_cluster ? SGBV_ERR_SHAPE : 0;
+    plan.cluster = C;
+    plan.slice_cells = slice_cells_of(cells, C);
+    int clusters = g_opt_max_clusters > 0 ? g_opt_max_clusters : resident(C, plan.row_mode != 0);
+    if (clusters < 1) return 0;  // this cluster shape cannot be scheduled here: nothing launched
+    const long share = plan.row_mode ? units : nchains;  // what the clusters share out
+    if (clusters > share) clusters = (int)share;
+    *walked_rows = plan.row_mode != 0;
+    return plan.row_mode ? launch_as<T, true>(L, plan, error_flag, clusters) : launch_as<T, false>(L, plan, error_flag, clusters);
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int stages, int max_clusters, int occupancy, int walk) {
+void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold) {
+    std::lock_guard<std::mutex> lock(g_plan_mu);
+    g_opt_withhold = withhold;
     g_opt_walk = walk;
     g_opt_cluster = cluster;
-    g_opt_stages = stages;
+    g_opt_slots = slots;
     g_opt_max_clusters = max_clusters;
-    g_opt_occupancy = occupancy;
+    g_opt_poll_us = poll_us;
 }
 
-// Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and
-// a CTA's slice must fit its registers (at most 5 chunks of 2048 elements, clusters of at most 16).
+// Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and a
+// row must fit the tensor memory of a cluster (8 CTAs x 32,768 entries).
 bool fused_supported(const Launch &L) {
     const size_t esz = L.dtype == SGBV_DTYPE_BF16 ? 2 : 4;
     if (((uintptr_t)L.zq % 16) || ((uintptr_t)L.zp % 16) || (((size_t)L.s.V * esz) % 16)) return false;
-    return slice_cells(cells_of(L.s.V), kMaxCluster) * kCell <= kMaxNch * kChunk;
+    return L.s.ntiles <= kMaxCluster * kCtaCells;
 }
 
 int launch_fused(const Launch &L, int *error_flag, bool *walked_rows) {
     *walked_rows = false;
-    const Shape &s = L.s;
-    const size_t esz = L.dtype == SGBV_DTYPE_BF16 ? 2 : 4;
-    const int cells = cells_of(s.V);
-    const long nchains = (long)s.B * s.K;
-    Plan plan;
-    const int occ = g_opt_occupancy ? g_opt_occupancy : 2;
-    const int cap = max_nch(occ) * kChunk;  // elements of a row one CTA can hold
-    const long cta_slots = (long)occ * kSms;
-    int C = g_opt_cluster;
-    int Cmin = 1;
-    while (Cmin < kMaxCluster && slice_cells(cells, Cmin) * kCell > cap) Cmin *= 2;  // smallest cluster whose slices fit
-    if (C == 0) {
-        C = Cmin;
-        // few chains: spread each over more CTAs while they all stay co-resident in one wave
-        while (C < kMaxCluster && nchains * 2 * C <= cta_slots && cells / (2 * C) >= 4) C *= 2;
-    }
-    // Few rows in all: when every ROW can have a cluster of its own in one wave, share out single rows
-    // instead of chains (their only coupling, c_i, is looked up), so that the gamma rows of a chain run
-    // side by side instead of one after the other.
-    {
-        const long units = nchains * s.gamma;
-        int Crow = g_opt_cluster ? g_opt_cluster : Cmin;
-        if (g_opt_cluster == 0)
-            while (Crow < kMaxCluster && units * 2 * Crow <= cta_slots && cells / (2 * Crow) >= 4) Crow *= 2;
-        plan.row_mode = occ == 2 && s.gamma > 1 && (g_opt_walk == 2 || (g_opt_walk == 0 && units * Crow <= cta_slots));
-        if (plan.row_mode) C = Crow;
-    }
-    if (C < 1 || C > kMaxCluster || slice_cells(cells, C) * kCell > cap) return g_opt_occupancy ? SGBV_ERR_SHAPE : 0;
-    plan.cluster = C;
-    plan.occ = occ;
-    plan.slice_len = slice_cells(cells, C) * kCell;
-    plan.nch = (plan.slice_len + kChunk - 1) / kChunk;
-    const size_t stage_bytes = 2 * kChunk * esz;
-    int S = g_opt_stages ? g_opt_stages : kMaxStages;
-    const size_t budget = kSmemPerSm / occ - kSmemReserved - sizeof(Control);
-    if ((size_t)S * stage_bytes > budget) S = (int)(budget / stage_bytes);
-    if (S > kMaxStages) S = kMaxStages;
-    // a whole row slice is moved to registers before any of its stages is refilled, so the ring must
-    // hold all chunks of a row at once
-    if (S < 2 || S < plan.nch) return g_opt_stages ? SGBV_ERR_SHAPE : 0;
-    plan.stages = S;
-    plan.smem = (size_t)S * stage_bytes + sizeof(Control);
-    plan.grid_clusters = g_opt_max_clusters;
-    *walked_rows = plan.row_mode != 0;
-    return L.dtype == SGBV_DTYPE_BF16 ? launch_t<uint16_t>(L, plan, error_flag) : launch_t<float>(L, plan, error_flag);
+    return L.dtype == SGBV_DTYPE_BF16 ? plan_and_launch<uint16_t>(L, error_flag, walked_rows)
+                                      : plan_and_launch<float>(L, error_flag, walked_rows);
 }
 
 }  // namespace sgbv

@@ -181,12 +181,24 @@ def test_temperature_extremes(T, dtype):
 
 
 def test_vocabulary_beyond_the_fused_kernel_capacity():
-    """Rows longer than 16 CTAs x 10,240 entries take the generic two-sweep kernels, aligned or not."""
-    cfg = workloads.VerifyConfig("bigv", B=2, K=2, gamma=2, V=163840 + 4096, alpha=0.85, seed=606)
+    """Rows longer than 8 CTAs x 32,768 entries (the tensor memory of the largest cluster) take the generic
+    two-sweep kernels, aligned or not."""
+    cfg = workloads.VerifyConfig("bigv", B=2, K=2, gamma=2, V=8 * 32768 + 4096, alpha=0.85, seed=606)
     inp = workloads.make_inputs(cfg, device="cuda")
     rep, _, _ = run_both(inp)
     assert_parity(rep)
     assert binding.last_main_kernel() == "otreduce_kernel"
+
+
+@pytest.mark.parametrize("V,dtype", [(8 * 32768, "fp32"), (8 * 32768 - 8, "bf16"), (5 * 32768 + 264, "fp32")])
+def test_vocabulary_at_the_fused_kernel_capacity(V, dtype):
+    """The longest rows the fused kernel takes (clusters of 8 with every tensor-memory column in use), and a
+    row that needs a cluster of 6."""
+    cfg = workloads.VerifyConfig("capv", B=2, K=2, gamma=2, V=V, dtype=dtype, alpha=0.85, seed=607)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+    assert binding.last_main_kernel() == "fused_chain_kernel"
 
 
 def test_more_than_2_to_the_31_logits_per_tensor():
@@ -204,43 +216,37 @@ def test_more_than_2_to_the_31_logits_per_tensor():
     torch.cuda.empty_cache()
 
 
-def _cdiv(a, b):
-    return -(-a // b)
-
-
 def _slice_fits(V, cluster):
-    """A CTA of the fused kernel holds at most five chunks of 2048 elements of a row in registers."""
+    """A CTA of the fused kernel holds at most 128 cells of 256 entries of a row in tensor memory."""
     cells = -(-V // 256)
-    return -(-cells // cluster) * 256 <= 5 * 2048
+    return -(-cells // cluster) <= 128
 
 
-@pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 4),
-                                    ("cluster", 8), ("cluster", 16), ("stages", 2), ("stages", 3),
-                                    ("max_clusters", 3), ("occupancy", 3), ("occupancy", 4), ("walk", 1), ("walk", 2)])
+@pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 3),
+                                    ("cluster", 4), ("cluster", 5), ("cluster", 8), ("stages", 1), ("stages", 2),
+                                    ("stages", 5), ("max_clusters", 3), ("walk", 1), ("walk", 2)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / ring depth /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
     cfgs = [workloads.VerifyConfig("paths_a", B=5, K=3, gamma=3, V=20480, temperature=0.8, alpha=0.8, seed=21),
             workloads.VerifyConfig("paths_b", B=3, K=2, gamma=2, V=33000, dtype="bf16", temperature=1.1, alpha=0.7,
                                    seed=22),
-            workloads.VerifyConfig("paths_c", B=2, K=2, gamma=5, V=1000, alpha=0.9, seed=23)]
+            workloads.VerifyConfig("paths_c", B=2, K=2, gamma=5, V=1000, alpha=0.9, seed=23),
+            workloads.VerifyConfig("paths_d", B=40, K=2, gamma=3, V=9000, temperature=0.9, alpha=0.85, seed=24)]
     binding.set_option(*option)
-    if option[0] == "stages":
-        binding.set_option("cluster", 8)   # fixes the number of chunks per row slice that the ring must hold
     try:
         for cfg in cfgs:
             if option[0] == "cluster" and not _slice_fits(cfg.V, option[1]):
-                continue   # forced cluster size whose slices do not fit the registers
-            if option[0] == "stages" and (not _slice_fits(cfg.V, 8) or _cdiv(_cdiv(_cdiv(cfg.V, 256), 8), 8) > option[1]):
-                continue   # the ring must hold all chunks of a row slice (clusters of 8 here)
-            if option[0] == "occupancy" and -(-cfg.V // 256) > 16 * 8 * (2 if option[1] == 3 else 1):
-                continue   # with 3 (4) CTAs per SM a warp holds 2 (1) cells: the row must fit 16 CTAs
+                continue   # forced cluster size whose slices do not fit the tensor memory
+            if option[0] == "stages" and option[1] > 3 and cfg.dtype == "fp32":
+                continue   # a ring of that depth does not fit the shared memory with float32 cells
+            if option == ("walk", 2) and cfg.B * cfg.K * cfg.gamma > 256:
+                continue   # the row walk has one ratio word per row, 256 in all
             inp = workloads.make_inputs(cfg, device="cuda")
             rep, _, _ = run_both(inp)
             assert_parity(rep)
     finally:
         binding.set_option(option[0], 0)
-        binding.set_option("cluster", 0)
 
 
 def test_unaligned_views_and_repeated_calls_are_deterministic():
@@ -345,6 +351,121 @@ def test_calls_replayed_from_a_cuda_graph_give_the_eager_results(name):
         for e, o in zip(eager, outs):
             assert torch.equal(e.accept_len, o.accept_len) and torch.equal(e.draft_idx, o.draft_idx)
             assert torch.equal(e.tokens, o.tokens)
+
+
+def _full_out(cfg):
+    dev = "cuda"
+    return binding.VerifyOutput(torch.full((cfg.B,), -7, dtype=torch.int32, device=dev),
+                                torch.full((cfg.B,), -7, dtype=torch.int32, device=dev),
+                                torch.full((cfg.B, cfg.gamma + 1), -7, dtype=torch.int32, device=dev),
+                                torch.zeros((cfg.B, cfg.K, cfg.gamma), dtype=torch.float64, device=dev),
+                                torch.zeros((cfg.B, cfg.K, cfg.gamma), dtype=torch.float64, device=dev),
+                                torch.full((cfg.B,), -7, dtype=torch.int32, device=dev))
+
+
+def _fresh_workspace_result(inp):
+    ws = torch.empty(binding.workspace_bytes(inp.cfg.B, inp.cfg.K, inp.cfg.gamma, inp.cfg.V) + 256,
+                     dtype=torch.uint8, device="cuda")
+    ws.fill_(0x5a)
+    off = (-ws.data_ptr()) % 256
+    out = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                 inp.cfg.temperature, workspace=ws[off:off + ws.numel() - 256])
+    torch.cuda.synchronize()
+    return out
+
+
+def _assert_identical(got, want):
+    assert torch.equal(got.accept_len, want.accept_len) and torch.equal(got.draft_idx, want.draft_idx)
+    assert torch.equal(got.tokens, want.tokens) and torch.equal(got.status, want.status)
+    assert torch.equal(got.h, want.h) and torch.equal(got.resmass, want.resmass)
+
+
+def _capture_call(inp, out):
+    """A CUDA graph holding one verify call on the library's own scratch (warmed up first, so nothing allocates)."""
+    args = (inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, inp.cfg.temperature)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            binding.sgbv_verify_ex(*args, out=out)
+    return graph
+
+
+def test_graph_replays_and_eager_calls_of_other_shapes_in_any_order():
+    """The row walk relies on words of the scratch that hold a "not published yet" pattern when a call starts.
+    That must hold whatever ran before on the library's scratch: captures that never ran, replays of graphs of
+    other shapes, eager calls in between.  Every result equals the one computed on a fresh caller workspace."""
+    row_a = workloads.make_inputs(workloads.with_batch(workloads.CONFIGS["paper_l8"], 2), device="cuda")
+    row_b = workloads.make_inputs(workloads.VerifyConfig("rowb", B=3, K=2, gamma=5, V=12288, temperature=0.7,
+                                                         alpha=0.8, seed=41), device="cuda")
+    c2 = workloads.make_inputs(workloads.CONFIGS["c2"], device="cuda")
+    big = workloads.make_inputs(workloads.VerifyConfig("bigger", B=64, K=4, gamma=4, V=32000, alpha=0.85, seed=42),
+                                device="cuda")
+    want = {id(x): _fresh_workspace_result(x) for x in (row_a, row_b, c2, big)}
+
+    def eager(inp):
+        out = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms,
+                                     inp.cfg.temperature)
+        torch.cuda.synchronize()
+        assert_row_walk = inp is row_a or inp is row_b
+        assert binding.last_main_kernel() == "fused_chain_kernel"
+        _assert_identical(out, want[id(inp)])
+        return assert_row_walk
+
+    for inp in (big, row_a, row_b, c2):   # warm-up: the scratch has its final size from here on
+        eager(inp)
+    # (i) capture the row walk, run another shape eagerly, replay
+    out_a = _full_out(row_a.cfg)
+    graph_a = _capture_call(row_a, out_a)
+    eager(c2)
+    graph_a.replay()
+    torch.cuda.synchronize()
+    _assert_identical(out_a, want[id(row_a)])
+    # (ii) a large shape eagerly, a capture that is not replayed, then the captured shape eagerly
+    eager(big)
+    out_b = _full_out(row_b.cfg)
+    graph_b = _capture_call(row_b, out_b)
+    eager(row_b)
+    eager(row_a)
+    # (iii) graphs of two row-walk shapes replayed alternately, eager calls in between
+    for _ in range(3):
+        graph_a.replay()
+        graph_b.replay()
+        torch.cuda.synchronize()
+        _assert_identical(out_a, want[id(row_a)])
+        _assert_identical(out_b, want[id(row_b)])
+        eager(c2)
+        graph_b.replay()
+        graph_a.replay()
+        torch.cuda.synchronize()
+        _assert_identical(out_a, want[id(row_a)])
+        _assert_identical(out_b, want[id(row_b)])
+
+
+def test_a_bounded_wait_that_runs_out_flags_every_row_and_the_next_call_is_correct():
+    """Failure detection without a fault: in the row walk a row waits (bounded) for the ratios that the rows
+    before it publish.  With the first row of every chain withholding its ratio and the limit of that poll
+    shortened, the poll expires; the kernel runs to its end, every batch row comes back flagged TIMEOUT with
+    -1 outputs, and the next ordinary call on the same scratch is correct."""
+    cfg = workloads.with_batch(workloads.CONFIGS["paper_l8"], 2)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    args = (inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, cfg.temperature)
+    binding.set_option("withhold", 1)
+    binding.set_option("poll_us", 300)
+    try:
+        out = binding.sgbv_verify_ex(*args)
+        torch.cuda.synchronize()
+    finally:
+        binding.set_option("withhold", 0)
+        binding.set_option("poll_us", 0)
+    assert binding.last_main_kernel() == "fused_chain_kernel"
+    st = out.status.cpu().numpy()
+    assert ((st & binding.STATUS_TIMEOUT) != 0).all()
+    assert (out.accept_len.cpu().numpy() == -1).all() and (out.draft_idx.cpu().numpy() == -1).all()
+    assert (out.tokens.cpu().numpy() == -1).all()
+    rep, again, _ = run_both(inp)
+    assert_parity(rep)
+    assert (again.status.cpu().numpy() & binding.STATUS_TIMEOUT == 0).all()
 
 
 def test_plain_bf16_and_host_entry_points_agree_with_extended():

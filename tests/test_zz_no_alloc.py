@@ -36,6 +36,16 @@ def test_static_scratch_entry_point_matches_on_two_calls_in_a_row():
         ref = binding.sgbv_verify_ex(*args)
         torch.cuda.synchronize()
         _same(got, ref)
+    # a shape that takes the row walk of the fused kernel, the one path that reads words of the shared array
+    # before writing them: before and after a larger shape that overwrites that part of the array
+    walk = workloads.make_inputs(workloads.with_batch(workloads.CONFIGS["paper_l8"], 2), device="cuda")
+    for inp in (walk, first, walk, walk):
+        args = (inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, inp.cfg.temperature)
+        got = binding.sgbv_verify_static(*args)
+        assert binding.last_main_kernel() == "fused_chain_kernel"
+        ref = binding.sgbv_verify_ex(*args)
+        torch.cuda.synchronize()
+        _same(got, ref)
     # and once more on the first inputs, now over the second call's leftovers
     args = (first.target_logits, first.draft_logits, first.draft_tokens, first.uniforms, first.cfg.temperature)
     got = binding.sgbv_verify_static(*args)
