@@ -37,16 +37,15 @@ namespace sgbv {
 
 namespace {
 
-constexpr int kFThreads = 1024;
-constexpr int kFWarps = kFThreads / 32;
+constexpr int kMaxWarps = 32;              // warps per CTA: 32 (64 registers each) or 16 (128 registers each)
 constexpr int kCell = kTile;               // 256 contiguous entries: the unit a warp works on
-constexpr int kCellsPerWarp = 4;           // 4 cells x 16 columns = the 64 tensor-memory columns of a warp
-constexpr int kCtaCells = kFWarps * kCellsPerWarp;  // 128 cells = 32,768 entries of a row per CTA
+constexpr int kCtaCells = 128;             // cells of a row per CTA: 512 tensor-memory columns / 16 per cell, x 4 lane quarters
+                                           // = 32,768 entries; a CTA of W warps gives each warp 128 / W cells
 constexpr int kTmemCols = 512;             // all of the SM's tensor memory (one CTA per SM)
-constexpr int kMaxSlots = 8;               // ring depth per warp
+constexpr int kMaxSlots = 12;              // ring depth per warp
 constexpr int kMaxCluster = 8;             // portable cluster size
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
-constexpr uint32_t kSuspendNs = 20000u;               // longest single suspension inside a wait
+constexpr uint32_t kPollNs = 100u;                    // sleep between two tests of a barrier that is not ready
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
 
 struct FusedParams {
@@ -67,55 +66,63 @@ struct FusedParams {
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+// mbarrier operations take the barrier's 32-bit shared-memory address
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
 }
-// The same test, but the thread may be suspended for up to about `kSuspendNs` until the phase completes
-// (the hardware wakes it when it does), instead of coming back at once.
-__device__ __forceinline__ bool mbar_test_suspend(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: sets `gave_up` if the phase did not complete within about a second.  A thread that has given
-// up once only tests from then on, so that the time a failing kernel takes stays bounded.
-__device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, bool &gave_up) {
+// Bounded wait: sets `gave_up` if the phase did not complete within about a second.  Between tests the
+// warp sleeps, so that a waiting warp leaves the issue slots to the working ones; the clock is read only
+// every 64 tests.  A thread that has given up once only tests from then on, so that the time a failing
+// kernel takes stays bounded.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool &gave_up) {
     if (mbar_test(bar, parity) || gave_up) return;
-    const long long t0 = clock64();
-    while (!mbar_test_suspend(bar, parity))
-        if (clock64() - t0 > kWaitLimitCycles) {
-            gave_up = true;
-            return;
+    uint32_t tests = 0;
+    long long t0 = 0;
+    for (;;) {
+        __nanosleep(kPollNs);
+        if (mbar_test(bar, parity)) return;
+        if ((++tests & 63u) == 0u) {
+            const long long t = clock64();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > kWaitLimitCycles) {
+                gave_up = true;
+                return;
+            }
         }
+    }
 }
-__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
+// One cell of both tensors into a ring slot (the draft part `half` bytes behind the target part): the lane
+// with pred != 0 announces 2 x bytes on the slot's barrier and starts the two bulk copies.  Every lane
+// executes the statement (no branch); the copies complete on the barrier.
+__device__ __forceinline__ void issue_cell(uint32_t dst, const void *zq, const void *zp, uint32_t bytes, uint32_t bar,
+                                           uint32_t pred, uint32_t half) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b32 d2, b2;\n\t"
+        "setp.ne.u32 p, %5, 0;\n\t"
+        "shl.b32 b2, %3, 1;\n\t"
+        "add.u32 d2, %0, %6;\n\t"
+        "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%4], b2;\n\t"
+        "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %3, [%4];\n\t"
+        "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [d2], [%2], %3, [%4];\n\t}" ::"r"(dst),
+        "l"(zq), "l"(zp), "r"(bytes), "r"(bar), "r"(pred), "r"(half)
+        : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -131,10 +138,10 @@ __device__ __forceinline__ void cluster_wait() {
 // Asynchronous store of 16 bytes into the shared memory of CTA `rank` of this cluster, at the
 // address that `local` has in this CTA; its completion is counted (16 bytes) on the receiver's
 // mbarrier that sits where `local_bar` sits here.
-__device__ __forceinline__ void push_f4(void *local, uint64_t *local_bar, uint32_t rank, float4 v) {
+__device__ __forceinline__ void push_f4(void *local, uint32_t local_bar, uint32_t rank, float4 v) {
     uint32_t dst, bar;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(smem_u32(local)), "r"(rank));
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(smem_u32(local_bar)), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(bar) : "r"(local_bar), "r"(rank));
     asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1,%2,%3,%4}, [%5];" ::"r"(dst),
                  "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(bar)
                  : "memory");
@@ -197,7 +204,7 @@ struct Control {
     uint64_t cbar[2];                    // by row parity, row walk only: "c_i is here"
     // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
     // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
-    float4 wslots[2][kFWarps];
+    float4 wslots[2][kMaxWarps];
     float4 slots[2][kMaxCluster];
     double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
     int arrivals;                        // partials left in wslots so far, over all rows (never reset)
@@ -264,13 +271,14 @@ __device__ __forceinline__ float2 ipow2(float2 r, int K) {
 }
 
 // Sums P values over the 32 lanes of a warp at once ("transposed" butterfly: at every step a lane
-// hands half of its values to its partner and keeps the other half).  P is a power of two (<= 4).
+// hands half of its values to its partner and keeps the other half).  P is a power of two (<= 8).
 // On return v[0] of lane l is the warp total of value number owner_index<P>(l).
 template <int P>
 __device__ __forceinline__ int owner_index(int lane) {
     int idx = 0;
     if (P >= 2) idx += (lane & 16) ? P / 2 : 0;
     if (P >= 4) idx += (lane & 8) ? P / 4 : 0;
+    if (P >= 8) idx += (lane & 4) ? P / 8 : 0;
     return idx;
 }
 template <int P>
@@ -305,10 +313,11 @@ struct RowScalars {
 //   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
 //   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
 // The output pointers address this warp's first cell; its cells are kFWarps apart.
-template <int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCellsPerWarp], const float (&mp)[kCellsPerWarp],
+template <int W, int KT, bool kAux>
+__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCtaCells / W], const float (&mp)[kCtaCells / W],
                                           const RowScalars &rs, int K, int lane, int ncw, float *wpart, float *dpart,
                                           float *mpart) {
+    constexpr int kCellsPerWarp = kCtaCells / W, kFWarps = W;
     const float v1 = 1.0f - rs.c;
     const float2 nv1 = splat(-v1);
     // Horner coefficients of Q: (t+1) (1-c)^t, t = 1..K-2 (uniform over the row)
@@ -394,27 +403,24 @@ __device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCel
     warp_sum_multi<kCellsPerWarp>(wsum, lane);
     // the lane that owns value number idx (and has the low lane bits clear) stores it
     const int idx = owner_index<kCellsPerWarp>(lane);
-    if ((lane & 7) == 0 && idx < ncw) wpart[idx * kFWarps] = wsum[0];
+    constexpr int kOwnerMask = 32 / kCellsPerWarp - 1;  // lanes that hold the same total
+    if ((lane & kOwnerMask) == 0 && idx < ncw) wpart[idx * kFWarps] = wsum[0];
 }
 
-template <bool kAux>
-__device__ __forceinline__ void sweep_two_dispatch(uint32_t taddr, const float (&mq)[kCellsPerWarp],
-                                                   const float (&mp)[kCellsPerWarp], const RowScalars &rs, int K, int lane,
-                                                   int ncw, float *wpart, float *dpart, float *mpart) {
-#define SGBV_SWEEP(KT) sweep_two<KT, kAux>(taddr, mq, mp, rs, K, lane, ncw, wpart, dpart, mpart)
-    switch (K) {
-        case 1: SGBV_SWEEP(1); break;
-        case 2: SGBV_SWEEP(2); break;
-        case 3: SGBV_SWEEP(3); break;
-        case 4: SGBV_SWEEP(4); break;
-        case 8: SGBV_SWEEP(8); break;
-        default: SGBV_SWEEP(0); break;
-    }
-#undef SGBV_SWEEP
-}
+// A warp's place in its stream of cell loads: cells j = 0..ncw-1 of walk position 0, then of position 1, ...
+// Kept by every lane (the values are warp-uniform); lane 0 starts the copies.
+struct LoadCursor {
+    const unsigned char *q, *p;  // this warp's first cell of the row being requested, in both tensors
+    int rows_left;               // rows whose cells have not all been requested
+    int j, i, slot;              // next cell of the row, position of the row in its chain, next ring slot
+    int bk;                      // chain of the row
+    int in_flight;               // loads issued and not consumed yet
+};
 
-template <typename T, bool kRow>
-__global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedParams p) {
+// KT: the number of drafts K when it has a specialised second sweep (1, 2, 3, 4, 8), else 0 (any K, loops).
+template <typename T, bool kRow, int W, int KT>
+__global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParams p) {
+    constexpr int kFWarps = W, kFThreads = W * 32, kCellsPerWarp = kCtaCells / W;
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -425,26 +431,31 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
     const int NS = p.slots;
     constexpr int kHalfBytes = kCell * (int)sizeof(T);  // one tensor's cell
     constexpr int kSlotBytes = 2 * kHalfBytes;          // the cell of zq, then the same cell of zp
-    unsigned char *ring = smem + (size_t)warp * NS * kSlotBytes;
-    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)kFWarps * NS * kSlotBytes) + warp * NS;
+    constexpr int kStrideBytes = kFWarps * kHalfBytes;  // from one cell of a warp to its next, in a row
+    const unsigned char *ring = smem + (size_t)warp * NS * kSlotBytes;
+    const uint32_t ring_u32 = smem_u32(ring);
+    const uint32_t full_u32 = smem_u32(smem) + (uint32_t)(kFWarps * NS * kSlotBytes + warp * NS * 8);
     Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * NS * (kSlotBytes + 8));
+    const uint32_t xbar_u32 = smem_u32(&ctl->xbar[0]), cbar_u32 = smem_u32(&ctl->cbar[0]);
 
     // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 32, ...
     const int cell_begin = rank * p.slice_cells;
     const int ncells_cta = max(0, min(s.ntiles, cell_begin + p.slice_cells) - cell_begin);
     const int ncw = ncells_cta > warp ? (ncells_cta - warp + kFWarps - 1) / kFWarps : 0;  // cells of this warp per row
     const int first_cell = cell_begin + warp;
-    const int x_warp = first_cell * kCell;  // first element of this warp's first cell
+    // the row's last cell may be a partial one: which of this warp's cells it is (-1: none), and its entries
+    const int tail_valid = s.V - (s.ntiles - 1) * kCell;
+    const int tail_j = (tail_valid < kCell && ncw > 0 && first_cell + (ncw - 1) * kFWarps == s.ntiles - 1) ? ncw - 1 : -1;
 
     if (tid == 0) {
-        mbar_init(&ctl->xbar[0], 1);
-        mbar_init(&ctl->xbar[1], 1);
-        mbar_init(&ctl->cbar[0], 1);
-        mbar_init(&ctl->cbar[1], 1);
+        mbar_init(xbar_u32, 1);
+        mbar_init(xbar_u32 + 8, 1);
+        mbar_init(cbar_u32, 1);
+        mbar_init(cbar_u32 + 8, 1);
         ctl->arrivals = 0;
     }
     if (lane == 0)
-        for (int k = 0; k < NS; ++k) mbar_init(&full[k], 1);
+        for (int k = 0; k < NS; ++k) mbar_init(full_u32 + 8 * k, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncwarp();
     if (warp == 0) tmem_alloc(&ctl->tmem_base, kTmemCols);
@@ -485,43 +496,49 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
     bool timed_out = false;
 
     // ---- this warp's copy ring --------------------------------------------------------------------
-    // Cell loads are numbered in consumption order: load m is cell m % ncw of walk position m / ncw and
-    // lands in slot m % NS.  The cursor below (kept by every lane, used by lane 0) names the next load.
-    // A warp that has given up on a wait issues no further loads and waits for those in flight only.
-    const long total_loads = (long)nrows * ncw;
-    long ld_m = 0;
-    int in_flight = 0;  // loads issued and not consumed yet
-    int ld_j = 0, ld_i = row_mode ? cid % s.gamma : 0, ld_slot = 0;
-    size_t ld_bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
-    auto issue_next = [&]() {
-        if (ld_m < total_loads && !timed_out) {
-            ++in_flight;
-            if (lane == 0) {
-                const int cell = first_cell + ld_j * kFWarps;
-                const size_t x0 = (size_t)cell * kCell;
-                const T *zq = reinterpret_cast<const T *>(p.zq) + (ld_bk * (s.gamma + 1) + ld_i) * s.V + x0;
-                const T *zp = reinterpret_cast<const T *>(p.zp) + (ld_bk * s.gamma + ld_i) * s.V + x0;
-                const uint32_t bytes = (uint32_t)min(kCell, s.V - (int)x0) * (uint32_t)sizeof(T);
-                unsigned char *dst = ring + (size_t)ld_slot * kSlotBytes;
-                mbar_expect_tx(&full[ld_slot], 2 * bytes);
-                bulk_load(dst, zq, bytes, &full[ld_slot]);
-                bulk_load(dst + kHalfBytes, zp, bytes, &full[ld_slot]);
-            }
-            ++ld_m;
-            if (++ld_slot == NS) ld_slot = 0;
-            if (++ld_j == ncw) {  // on to the next row of the walk
-                ld_j = 0;
-                ld_bk += step_bk;
-                ld_i += step_i;
-                if (ld_i >= s.gamma) {
-                    ld_i -= s.gamma;
-                    ld_bk += wrap_bk;
-                }
-            }
-        }
-    };
-    if (ncw > 0)
-        for (int k = 0; k < NS; ++k) issue_next();
+    // Cell loads go out in consumption order: cell j = 0..ncw-1 of walk position 0, then of position 1, ...;
+    // a load lands in the slot that the cell NS before it has just left.  The cursor below (kept by every
+    // lane, the copies are started by lane 0) names the next load.  A warp that has given up on a wait
+    // issues no further loads and waits for those in flight only.
+    const size_t row_bytes = (size_t)s.V * sizeof(T);
+    LoadCursor lc;
+    lc.rows_left = ncw > 0 ? nrows : 0;
+    lc.j = 0;
+    lc.i = row_mode ? cid % s.gamma : 0;
+    lc.slot = 0;
+    lc.bk = row_mode ? cid / s.gamma : cid;
+    lc.in_flight = 0;
+    lc.q = reinterpret_cast<const unsigned char *>(p.zq) + (size_t)first_cell * kHalfBytes +
+           ((size_t)lc.bk * (s.gamma + 1) + lc.i) * row_bytes;
+    lc.p = reinterpret_cast<const unsigned char *>(p.zp) + (size_t)first_cell * kHalfBytes +
+           ((size_t)lc.bk * s.gamma + lc.i) * row_bytes;
+    const uint32_t is_lane0 = lane == 0 ? 1u : 0u;
+#define SGBV_ISSUE_NEXT()                                                                                              \
+    do {                                                                                                               \
+        if (lc.rows_left > 0 && !timed_out) { /* warp-uniform */                                                       \
+            const uint32_t bytes_ = (lc.j == tail_j) ? (uint32_t)(tail_valid * (int)sizeof(T)) : (uint32_t)kHalfBytes; \
+            issue_cell(ring_u32 + (uint32_t)(lc.slot * kSlotBytes), lc.q + (size_t)lc.j * kStrideBytes,                \
+                       lc.p + (size_t)lc.j * kStrideBytes, bytes_, full_u32 + 8u * (uint32_t)lc.slot, is_lane0,        \
+                       kHalfBytes);                                                                                    \
+            ++lc.in_flight;                                                                                            \
+            if (++lc.slot == NS) lc.slot = 0;                                                                          \
+            if (++lc.j == ncw) { /* on to the next row of the walk */                                                  \
+                lc.j = 0;                                                                                              \
+                --lc.rows_left;                                                                                        \
+                lc.bk += step_bk;                                                                                      \
+                lc.i += step_i;                                                                                        \
+                if (lc.i >= s.gamma) {                                                                                 \
+                    lc.i -= s.gamma;                                                                                   \
+                    lc.bk += wrap_bk;                                                                                  \
+                }                                                                                                      \
+                lc.q = reinterpret_cast<const unsigned char *>(p.zq) + (size_t)first_cell * kHalfBytes +               \
+                       ((size_t)lc.bk * (s.gamma + 1) + lc.i) * row_bytes;                                             \
+                lc.p = reinterpret_cast<const unsigned char *>(p.zp) + (size_t)first_cell * kHalfBytes +               \
+                       ((size_t)lc.bk * s.gamma + lc.i) * row_bytes;                                                   \
+            }                                                                                                          \
+        }                                                                                                              \
+    } while (0)
+    for (int k = 0; k < NS; ++k) SGBV_ISSUE_NEXT();
     int c_slot = 0;           // slot of the next cell to consume
     uint32_t c_phase = 0;     // parity of that slot's barrier
 
@@ -532,7 +549,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
     if (chain_thread && nrows > 0) tok_next = p.tok[row_mode ? (size_t)cid : (size_t)cid * s.gamma];
     if (chain_thread && nrows > 0 && !row_mode) {  // the first row of the walk starts a chain: c_0 = 1
         ctl->c[0] = 1.0;
-        mbar_expect_tx(&ctl->xbar[0], xbytes);
+        mbar_expect_tx(xbar_u32, xbytes);
     }
 
     size_t bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
@@ -541,11 +558,12 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
         const size_t r = bk * s.gamma + i;
         const int par = n & 1;
         const uint32_t xph = (uint32_t)(n >> 1) & 1u;
+        const uint32_t xbar = xbar_u32 + 8u * (uint32_t)par;
 
         // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
         float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
         if (chain_thread) {
-            if (row_mode) mbar_expect_tx(&ctl->xbar[par], xbytes);  // the exchange does not wait for c_i here
+            if (row_mode) mbar_expect_tx(xbar, xbytes);  // the exchange does not wait for c_i here
             int t = tok_next;
             if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
             zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
@@ -571,21 +589,19 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
 #pragma unroll
         for (int j = 0; j < kCellsPerWarp; ++j) {
             if (j < ncw) {  // warp-uniform
-                if (in_flight > 0) {
-                    mbar_wait(&full[c_slot], c_phase, timed_out);
-                    timed_out = __any_sync(0xffffffffu, timed_out);
-                    --in_flight;
+                if (lc.in_flight > 0) {
+                    mbar_wait(full_u32 + 8u * (uint32_t)c_slot, c_phase, timed_out);
+                    --lc.in_flight;
                 }
                 float2 eq[4], ep[4];
-                const unsigned char *base = ring + (size_t)c_slot * kSlotBytes;
+                const unsigned char *base = ring + c_slot * kSlotBytes;
                 read_cell<T>(base, lane, eq);
                 read_cell<T>(base + kHalfBytes, lane, ep);
-                const int cell_x = x_warp + j * kFWarps * kCell;
-                if (cell_x + kCell > s.V) {  // the row ends inside this cell
+                if (j == tail_j) {  // the row ends inside this cell
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        if (cell_x + cell_offset<T>(lane, 2 * e) >= s.V) eq[e].x = ep[e].x = -INFINITY;
-                        if (cell_x + cell_offset<T>(lane, 2 * e + 1) >= s.V) eq[e].y = ep[e].y = -INFINITY;
+                        if (cell_offset<T>(lane, 2 * e) >= tail_valid) eq[e].x = ep[e].x = -INFINITY;
+                        if (cell_offset<T>(lane, 2 * e + 1) >= tail_valid) eq[e].y = ep[e].y = -INFINITY;
                     }
                 }
                 float m1 = -INFINITY, m2 = -INFINITY;
@@ -596,7 +612,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
                 }
                 // every lane holds its share of the slot in registers now: refill it with the cell NS further on
                 __syncwarp();
-                issue_next();
+                SGBV_ISSUE_NEXT();
                 if (++c_slot == NS) {
                     c_slot = 0;
                     c_phase ^= 1u;
@@ -657,36 +673,44 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
         }
         if (__shfl_sync(0xffffffffu, last_warp, 0)) {
             __threadfence_block();
-            const float4 v = ctl->wslots[par][lane];  // one warp partial per lane
+            const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
             const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
             const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
             const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
             const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
-            if (lane < C)
-                push_f4(&ctl->slots[par][rank], &ctl->xbar[par], (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
+            if (lane < C) push_f4(&ctl->slots[par][rank], xbar, (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
         }
-        mbar_wait(&ctl->xbar[par], xph, timed_out);
+        mbar_wait(xbar, xph, timed_out);
         timed_out = __any_sync(0xffffffffu, timed_out);  // the warp gives up as one
 
         // ---- row statistics: every warp combines the CTA partials, in the same order -------------
-        const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-        const float bq_row = warp_max_redux(cv.x), bp_row = warp_max_redux(cv.z);
+        float bq_row, bp_row, Zq, Zp;
+        if (C == 1) {  // the CTA's partial is the row's
+            const float4 cv = ctl->slots[par][0];
+            bq_row = cv.x;
+            bp_row = cv.z;
+            Zq = cv.y;
+            Zp = cv.w;
+        } else {
+            const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+            bq_row = warp_max_redux(cv.x);
+            bp_row = warp_max_redux(cv.z);
+            const float rq0 = (bq_row > -INFINITY) ? bq_row : 0.0f, rp0 = (bp_row > -INFINITY) ? bp_row : 0.0f;
+            Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq0) * s.scale) : 0.0f);
+            Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp0) * s.scale) : 0.0f);
+        }
         const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
-        const float Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
-        const float Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
         // the ratio p_i(tok_i)/q_i(tok_i) of this row (chain thread)
-        auto token_ratio = [&]() {
-            const double lp = ((double)zp_tok - (double)rp_row) * (double)s.scale;
-            const double lq = ((double)zq_tok - (double)rq_row) * (double)s.scale;
-            return exp2_short(lp - lq) * (double)(Zq / Zp);
-        };
+#define SGBV_TOKEN_RATIO()                                                                                  \
+    (exp2_short(((double)zp_tok - (double)rp_row) * (double)s.scale - ((double)zq_tok - (double)rq_row) * (double)s.scale) * \
+     (double)(Zq / Zp))
         double cd;
         if (row_mode) {
             // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
             // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
             // NaN (a row that produces one is flagged invalid anyway).
             if (chain_thread && rank == 0 && i + 1 < s.gamma && !(p.withhold && i == 0)) {
-                double ratio = token_ratio();
+                double ratio = SGBV_TOKEN_RATIO();
                 if (ratio != ratio) ratio = 0.0;
                 *reinterpret_cast<volatile double *>(p.ws.ratio + r) = ratio;
             }
@@ -694,6 +718,7 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
             // butterfly over the lanes).  Those rows are walked by other clusters at about the same
             // time and publish right after their own statistics, which do not depend on c: no chain of
             // waits forms.  Every lane of the last warp polls one of them.  Bounded waits.
+            const uint32_t cbar = cbar_u32 + 8u * (uint32_t)par;
             if (warp == kFWarps - 1) {
                 double cprod = 1.0;
                 const size_t r0 = bk * s.gamma;
@@ -721,10 +746,10 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
                 }
                 if (lane == 0) {
                     ctl->c[par] = cprod;
-                    mbar_arrive(&ctl->cbar[par]);  // c_i is there
+                    mbar_arrive(cbar);  // c_i is there
                 }
             }
-            mbar_wait(&ctl->cbar[par], xph, timed_out);
+            mbar_wait(cbar, xph, timed_out);
             timed_out = __any_sync(0xffffffffu, timed_out);
             cd = ctl->c[par];
         } else {
@@ -732,8 +757,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
             if (chain_thread && n + 1 < nrows) {
                 // c of the next row of the walk: c_{i+1} = c_i ratio, or 1 at the start of the next
                 // chain; publishing it arms the next row's exchange
-                ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * token_ratio() : 1.0;
-                mbar_expect_tx(&ctl->xbar[par ^ 1], xbytes);
+                ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * SGBV_TOKEN_RATIO() : 1.0;
+                mbar_expect_tx(xbar_u32 + 8u * (uint32_t)(par ^ 1), xbytes);
             }
         }
         RowScalars rs;
@@ -764,9 +789,9 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
         float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
               *mpp = p.ws.mpart + r * s.ntiles + first_cell;
         if (rs.c < 1.0f)
-            sweep_two_dispatch<true>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+            sweep_two<W, KT, true>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
         else
-            sweep_two_dispatch<false>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+            sweep_two<W, KT, false>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
 
         // one step of the walk
         bk += step_bk;
@@ -782,6 +807,8 @@ __global__ void __launch_bounds__(kFThreads, 1) fused_chain_kernel(const FusedPa
     tmem_fence_before();
     __syncthreads();  // every warp of this CTA is done with the tensor memory
     if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+#undef SGBV_ISSUE_NEXT
+#undef SGBV_TOKEN_RATIO
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -796,20 +823,21 @@ int g_opt_max_clusters = 0;
 int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
 int g_opt_poll_us = 0;     // 0 = about a second
 int g_opt_withhold = 0;
+int g_opt_warps = 0;       // 0 = automatic, 16 or 32
 
 constexpr int kSmemPerCta = 227 * 1024;    // largest dynamic shared memory of one CTA
 constexpr int kDevices = 64;
-std::mutex g_plan_mu;      // guards the per-device caches below
+std::mutex g_plan_mu;      // guards the options and the per-device caches below
 
 size_t slot_bytes(int dtype) { return 2 * (size_t)kCell * (dtype == SGBV_DTYPE_BF16 ? 2 : 4); }
-size_t smem_bytes(int dtype, int slots) { return (size_t)kFWarps * slots * (slot_bytes(dtype) + 8) + sizeof(Control); }
+size_t smem_bytes(int dtype, int warps, int slots) { return (size_t)warps * slots * (slot_bytes(dtype) + 8) + sizeof(Control); }
 int slice_cells_of(int cells, int C) { return (cells + C - 1) / C; }
 
-template <typename T, bool kRow>
+template <typename T, bool kRow, int W, int KT>
 cudaError_t prepare(int dev) {
     static bool attr_done[kDevices];
     if (!attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
+        cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow, W, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
@@ -817,13 +845,13 @@ cudaError_t prepare(int dev) {
 }
 
 // Clusters of C CTAs of this kernel that the device runs side by side (queried once per configuration).
-template <typename T, bool kRow>
+template <typename T, bool kRow, int W, int KT>
 int resident_clusters(int dev, int C, int slots, size_t smem) {
     static int cached[kDevices][kMaxCluster + 1][kMaxSlots + 1];
     int &slot = cached[dev][C][slots];
     if (slot == 0) {
         cudaLaunchConfig_t cfg = {};
-        cfg.blockDim = dim3(kFThreads);
+        cfg.blockDim = dim3(W * 32);
         cfg.dynamicSmemBytes = smem;
         cfg.gridDim = dim3(C * (148 / C));
         cudaLaunchAttribute attr[1];
@@ -834,7 +862,7 @@ int resident_clusters(int dev, int C, int slots, size_t smem) {
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int nmax = 0;
-        if (cudaOccupancyMaxActiveClusters(&nmax, fused_chain_kernel<T, kRow>, &cfg) != cudaSuccess || nmax < 1) {
+        if (cudaOccupancyMaxActiveClusters(&nmax, fused_chain_kernel<T, kRow, W, KT>, &cfg) != cudaSuccess || nmax < 1) {
             cudaGetLastError();
             return 0;
         }
@@ -843,7 +871,7 @@ int resident_clusters(int dev, int C, int slots, size_t smem) {
     return slot;
 }
 
-template <typename T, bool kRow>
+template <typename T, bool kRow, int W, int KT>
 int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) {
     FusedParams fp;
     fp.zq = L.zq;
@@ -860,7 +888,7 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
     fp.withhold = g_opt_withhold;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(kFThreads);
+    cfg.blockDim = dim3(W * 32);
     cfg.dynamicSmemBytes = plan.smem;
     cfg.stream = L.stream;
     cudaLaunchAttribute attr[2];
@@ -879,7 +907,7 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
         cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
         return SGBV_ERR_CUDA;
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_chain_kernel<T, kRow>, fp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_chain_kernel<T, kRow, W, KT>, fp);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -889,41 +917,40 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
 }
 
 // Chooses the cluster size and the walk, then launches.  Returns launches, 0 if declined, or < 0.
-template <typename T>
+template <typename T, int W, int KT>
 int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const Shape &s = L.s;
     const int cells = s.ntiles;
     const long nchains = (long)s.B * s.K, units = nchains * s.gamma;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDevices) return SGBV_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(g_plan_mu);
-    if (prepare<T, false>(dev) != cudaSuccess || prepare<T, true>(dev) != cudaSuccess) {
+    if (prepare<T, false, W, KT>(dev) != cudaSuccess || prepare<T, true, W, KT>(dev) != cudaSuccess) {
         cudaGetLastError();
         return SGBV_ERR_CUDA;
     }
     Plan plan;
     // ring depth: what fits beside the control block, at most the default (deeper rings keep more bytes
     // in flight than the memory system rewards)
-    const int max_slots = (int)std::min<size_t>(kMaxSlots, (kSmemPerCta - sizeof(Control)) / ((size_t)kFWarps * (slot_bytes(L.dtype) + 8)));
-    int slots = g_opt_slots ? g_opt_slots : (L.dtype == SGBV_DTYPE_BF16 ? 6 : 3);
+    const int max_slots = (int)std::min<size_t>(kMaxSlots, (kSmemPerCta - sizeof(Control)) / ((size_t)W * (slot_bytes(L.dtype) + 8)));
+    int slots = g_opt_slots ? g_opt_slots : (W == 32 ? 3 : 6) * (L.dtype == SGBV_DTYPE_BF16 ? 2 : 1);
     if (slots > max_slots) {
         if (g_opt_slots) return SGBV_ERR_SHAPE;
         slots = max_slots;
     }
     plan.slots = slots;
-    plan.smem = smem_bytes(L.dtype, slots);
+    plan.smem = smem_bytes(L.dtype, W, slots);
     int Cmin = (cells + kCtaCells - 1) / kCtaCells;  // smallest cluster whose slices fit the tensor memory
     if (Cmin > kMaxCluster) return 0;
     auto fits = [&](int C) { return C >= Cmin && C <= kMaxCluster; };
     auto resident = [&](int C, bool row) {
-        return row ? resident_clusters<T, true>(dev, C, plan.slots, plan.smem)
-                   : resident_clusters<T, false>(dev, C, plan.slots, plan.smem);
+        return row ? resident_clusters<T, true, W, KT>(dev, C, plan.slots, plan.smem)
+                   : resident_clusters<T, false, W, KT>(dev, C, plan.slots, plan.smem);
     };
     // Few units of work: spread each over more CTAs (at least half the warps keep a cell) while all of them
     // still run side by side.
     auto widen = [&](long n_units, bool row) {
         int C = Cmin;
-        while (2 * C <= kMaxCluster && cells >= C * kFWarps && n_units <= resident(2 * C, row)) C *= 2;
+        while (2 * C <= kMaxCluster && cells >= C * W && n_units <= resident(2 * C, row)) C *= 2;
         return C;
     };
     int C = g_opt_cluster ? g_opt_cluster : widen(nchains, false);
@@ -946,12 +973,13 @@ int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const long share = plan.row_mode ? units : nchains;  // what the clusters share out
     if (clusters > share) clusters = (int)share;
     *walked_rows = plan.row_mode != 0;
-    return plan.row_mode ? launch_as<T, true>(L, plan, error_flag, clusters) : launch_as<T, false>(L, plan, error_flag, clusters);
+    return plan.row_mode ? launch_as<T, true, W, KT>(L, plan, error_flag, clusters)
+                         : launch_as<T, false, W, KT>(L, plan, error_flag, clusters);
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold) {
+void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold, int warps) {
     std::lock_guard<std::mutex> lock(g_plan_mu);
     g_opt_withhold = withhold;
     g_opt_walk = walk;
@@ -959,6 +987,7 @@ void fused_set_options(int cluster, int slots, int max_clusters, int walk, int p
     g_opt_slots = slots;
     g_opt_max_clusters = max_clusters;
     g_opt_poll_us = poll_us;
+    g_opt_warps = warps;
 }
 
 // Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and a
@@ -969,10 +998,26 @@ bool fused_supported(const Launch &L) {
     return L.s.ntiles <= kMaxCluster * kCtaCells;
 }
 
+template <typename T, int W>
+int dispatch_k(const Launch &L, int *error_flag, bool *walked_rows) {
+    switch (L.s.K) {
+        case 1: return plan_and_launch<T, W, 1>(L, error_flag, walked_rows);
+        case 2: return plan_and_launch<T, W, 2>(L, error_flag, walked_rows);
+        case 3: return plan_and_launch<T, W, 3>(L, error_flag, walked_rows);
+        case 4: return plan_and_launch<T, W, 4>(L, error_flag, walked_rows);
+        case 8: return plan_and_launch<T, W, 8>(L, error_flag, walked_rows);
+        default: return plan_and_launch<T, W, 0>(L, error_flag, walked_rows);
+    }
+}
+
 int launch_fused(const Launch &L, int *error_flag, bool *walked_rows) {
     *walked_rows = false;
-    return L.dtype == SGBV_DTYPE_BF16 ? plan_and_launch<uint16_t>(L, error_flag, walked_rows)
-                                      : plan_and_launch<float>(L, error_flag, walked_rows);
+    std::lock_guard<std::mutex> lock(g_plan_mu);
+    const int warps = g_opt_warps ? g_opt_warps : 32;
+    if (L.dtype == SGBV_DTYPE_BF16)
+        return warps == 16 ? dispatch_k<uint16_t, 16>(L, error_flag, walked_rows)
+                           : dispatch_k<uint16_t, 32>(L, error_flag, walked_rows);
+    return warps == 16 ? dispatch_k<float, 16>(L, error_flag, walked_rows) : dispatch_k<float, 32>(L, error_flag, walked_rows);
 }
 
 }  // namespace sgbv
