@@ -200,16 +200,22 @@ __device__ __forceinline__ void tmem_wait_ld(float2 (&a)[4], float2 (&b)[4]) {
 // ---- shared memory layout ------------------------------------------------------------------------
 // [rings: 32 warps x slots x (cell of zq, cell of zp)] [full barriers: 32 warps x slots] [Control]
 struct Control {
-    uint64_t xbar[2];                    // by row parity: "all partials of the row (chain walk: and c_i) are here"
-    uint64_t cbar[2];                    // by row parity, row walk only: "c_i is here"
-    // partials (maximum of zq, sum eq, maximum of zp, sum ep), double-buffered by row parity:
-    // of this CTA's warps, and of every CTA of the cluster (pushed by their owners)
-    float4 wslots[2][kMaxWarps];
+    uint64_t xbar[2];                    // by row parity: "the partials of all CTAs of the cluster are here"
+    // partials (maximum of zq, sum eq, maximum of zp, sum ep): of this CTA's warps, and, double-buffered by
+    // row parity, of every CTA of the cluster (pushed by their owners)
+    float4 wslots[kMaxWarps];
     float4 slots[2][kMaxCluster];
-    double c[2];                         // joint likelihood ratio c_i of the current row, by row parity
-    int arrivals;                        // partials left in wslots so far, over all rows (never reset)
+    float4 rs;                           // the row's scalars for the second sweep: rq, rp, kappa, c
     uint32_t tmem_base;                  // address of the allocated tensor memory
 };
+
+// Named hardware barriers of the CTA (0 is the one of __syncthreads).
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+    asm volatile("barrier.cta.sync.aligned %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int nthreads) {
+    asm volatile("barrier.cta.arrive.aligned %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 
 // Reads this lane's 8 elements of one cell of one tensor from the ring.
 template <typename T>
@@ -436,7 +442,7 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     const uint32_t ring_u32 = smem_u32(ring);
     const uint32_t full_u32 = smem_u32(smem) + (uint32_t)(kFWarps * NS * kSlotBytes + warp * NS * 8);
     Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * NS * (kSlotBytes + 8));
-    const uint32_t xbar_u32 = smem_u32(&ctl->xbar[0]), cbar_u32 = smem_u32(&ctl->cbar[0]);
+    const uint32_t xbar_u32 = smem_u32(&ctl->xbar[0]);
 
     // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 32, ...
     const int cell_begin = rank * p.slice_cells;
@@ -450,9 +456,6 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     if (tid == 0) {
         mbar_init(xbar_u32, 1);
         mbar_init(xbar_u32 + 8, 1);
-        mbar_init(cbar_u32, 1);
-        mbar_init(cbar_u32 + 8, 1);
-        ctl->arrivals = 0;
     }
     if (lane == 0)
         for (int k = 0; k < NS; ++k) mbar_init(full_u32 + 8 * k, 1);
@@ -542,40 +545,37 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     int c_slot = 0;           // slot of the next cell to consume
     uint32_t c_phase = 0;     // parity of that slot's barrier
 
-    // The chain thread of this CTA carries c_i and fetches the token logits one row
-    // ahead: tok_next is the token of the next row of the walk.
-    const bool chain_thread = tid == kFThreads - 32;  // lane 0 of the last warp; thread 0 writes the row records
+    // The last warp of this CTA combines the partials, carries c_i and fetches the token logits one row
+    // ahead (every lane the same words): tok_next is the token of the next row of the walk.
+    const bool combiner = warp == kFWarps - 1;
     int tok_next = 0;
-    if (chain_thread && nrows > 0) tok_next = p.tok[row_mode ? (size_t)cid : (size_t)cid * s.gamma];
-    if (chain_thread && nrows > 0 && !row_mode) {  // the first row of the walk starts a chain: c_0 = 1
-        ctl->c[0] = 1.0;
-        mbar_expect_tx(xbar_u32, xbytes);
-    }
+    if (combiner && nrows > 0) tok_next = p.tok[row_mode ? (size_t)cid : (size_t)cid * s.gamma];
+    double c_carry = 1.0;  // chain walk: c of the row at hand (the first row of the walk starts a chain)
 
-    size_t bk = row_mode ? (size_t)(cid / s.gamma) : (size_t)cid;
+    int bk = row_mode ? cid / s.gamma : cid;
     int i = row_mode ? cid % s.gamma : 0;
     for (int n = 0; n < nrows; ++n) {
-        const size_t r = bk * s.gamma + i;
+        const size_t r = (size_t)bk * s.gamma + i;
         const int par = n & 1;
         const uint32_t xph = (uint32_t)(n >> 1) & 1u;
         const uint32_t xbar = xbar_u32 + 8u * (uint32_t)par;
 
-        // ---- chain thread: the logits of this row's draft token, and the next row's token -----------
+        // ---- combining warp: the logits of this row's draft token, and the next row's token --------
         float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
-        if (chain_thread) {
-            if (row_mode) mbar_expect_tx(xbar, xbytes);  // the exchange does not wait for c_i here
+        if (combiner) {
+            if (C > 1 && lane == 0) mbar_expect_tx(xbar, xbytes);  // this row's partials of the cluster's CTAs
             int t = tok_next;
             if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
-            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + (bk * (s.gamma + 1) + i) * s.V, t);
-            zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + (bk * s.gamma + i) * s.V, t);
+            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk * (s.gamma + 1) + i) * s.V, t);
+            zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + ((size_t)bk * s.gamma + i) * s.V, t);
             if (n + 1 < nrows) {
-                size_t bk_n = bk + step_bk;
+                int bk_n = bk + step_bk;
                 int i_n = i + step_i;
                 if (i_n >= s.gamma) {
                     i_n -= s.gamma;
                     bk_n += wrap_bk;
                 }
-                tok_next = p.tok[bk_n * s.gamma + i_n];
+                tok_next = p.tok[(size_t)bk_n * s.gamma + i_n];
             }
         }
 
@@ -663,127 +663,112 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
         const float rqw = (bqw > -INFINITY) ? bqw : 0.0f, rpw = (bpw > -INFINITY) ? bpw : 0.0f;
         sqt = warp_sum(has_q ? sqt * ex2((bqt - rqw) * s.scale) : 0.0f);
         spt = warp_sum(has_p ? spt * ex2((bpt - rpw) * s.scale) : 0.0f);
-        // two-level exchange: the warp partials meet in this CTA's shared memory; the warp that
-        // arrives last combines them (fixed order) and pushes ONE partial per CTA to every CTA
-        bool last_warp = false;
-        if (lane == 0) {
-            ctl->wslots[par][warp] = make_float4(bqw, sqt, bpw, spt);
-            __threadfence_block();
-            last_warp = atomicAdd(&ctl->arrivals, 1) + 1 == kFWarps * (n + 1);
-        }
-        if (__shfl_sync(0xffffffffu, last_warp, 0)) {
-            __threadfence_block();
-            const float4 v = lane < kFWarps ? ctl->wslots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-            const float mqc = warp_max_redux(v.x), mpc = warp_max_redux(v.z);
-            const float rqc = (mqc > -INFINITY) ? mqc : 0.0f, rpc = (mpc > -INFINITY) ? mpc : 0.0f;
-            const float sqc = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rqc) * s.scale) : 0.0f);
-            const float spc = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rpc) * s.scale) : 0.0f);
-            if (lane < C) push_f4(&ctl->slots[par][rank], xbar, (uint32_t)lane, make_float4(mqc, sqc, mpc, spc));
-        }
-        mbar_wait(xbar, xph, timed_out);
-        timed_out = __any_sync(0xffffffffu, timed_out);  // the warp gives up as one
-
-        // ---- row statistics: every warp combines the CTA partials, in the same order -------------
-        float bq_row, bp_row, Zq, Zp;
-        if (C == 1) {  // the CTA's partial is the row's
-            const float4 cv = ctl->slots[par][0];
-            bq_row = cv.x;
-            bp_row = cv.z;
-            Zq = cv.y;
-            Zp = cv.w;
+        // Exchange.  Every warp leaves its partial in shared memory; the LAST warp of the CTA combines them,
+        // trades the CTA's partial with the other CTAs of the cluster (asynchronous distributed-shared-memory
+        // stores that complete on the receiver's mbarrier; it alone polls that barrier), works out the row's
+        // scalars and hands them to the others.  The others wait on hardware barriers, which costs them no
+        // issue slots: barrier 1 = "all partials are in", barrier 2 = "the row's scalars are in".
+        if (lane == 0) ctl->wslots[warp] = make_float4(bqw, sqt, bpw, spt);
+        __threadfence_block();
+        RowScalars rs;
+        if (warp != kFWarps - 1) {
+            bar_arrive(1, kFThreads);
+            bar_sync(2, kFThreads);
+            const float4 v = ctl->rs;  // (the barrier statement is a compiler barrier for memory)
+            rs.rq = v.x;
+            rs.rp = v.y;
+            rs.kappa = v.z;
+            rs.c = v.w;
         } else {
-            const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
-            bq_row = warp_max_redux(cv.x);
-            bp_row = warp_max_redux(cv.z);
-            const float rq0 = (bq_row > -INFINITY) ? bq_row : 0.0f, rp0 = (bp_row > -INFINITY) ? bp_row : 0.0f;
-            Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq0) * s.scale) : 0.0f);
-            Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp0) * s.scale) : 0.0f);
-        }
-        const float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
-        // the ratio p_i(tok_i)/q_i(tok_i) of this row (chain thread)
-#define SGBV_TOKEN_RATIO()                                                                                  \
-    (exp2_short(((double)zp_tok - (double)rp_row) * (double)s.scale - ((double)zq_tok - (double)rq_row) * (double)s.scale) * \
-     (double)(Zq / Zp))
-        double cd;
-        if (row_mode) {
-            // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
-            // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
-            // NaN (a row that produces one is flagged invalid anyway).
-            if (chain_thread && rank == 0 && i + 1 < s.gamma && !(p.withhold && i == 0)) {
-                double ratio = SGBV_TOKEN_RATIO();
-                if (ratio != ratio) ratio = 0.0;
-                *reinterpret_cast<volatile double *>(p.ws.ratio + r) = ratio;
+            bar_sync(1, kFThreads);
+            const float4 v = lane < kFWarps ? ctl->wslots[lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+            float bq_row = warp_max_redux(v.x), bp_row = warp_max_redux(v.z);
+            float rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f, rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
+            float Zq = warp_sum(v.x > -INFINITY ? v.y * ex2((v.x - rq_row) * s.scale) : 0.0f);
+            float Zp = warp_sum(v.z > -INFINITY ? v.w * ex2((v.z - rp_row) * s.scale) : 0.0f);
+            if (C > 1) {  // the same once more over the CTAs of the cluster
+                if (lane < C) push_f4(&ctl->slots[par][rank], xbar, (uint32_t)lane, make_float4(bq_row, Zq, bp_row, Zp));
+                mbar_wait(xbar, xph, timed_out);
+                timed_out = __any_sync(0xffffffffu, timed_out);  // the warp gives up as one
+                const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
+                bq_row = warp_max_redux(cv.x);
+                bp_row = warp_max_redux(cv.z);
+                rq_row = (bq_row > -INFINITY) ? bq_row : 0.0f;
+                rp_row = (bp_row > -INFINITY) ? bp_row : 0.0f;
+                Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
+                Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
             }
-            // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
-            // butterfly over the lanes).  Those rows are walked by other clusters at about the same
-            // time and publish right after their own statistics, which do not depend on c: no chain of
-            // waits forms.  Every lane of the last warp polls one of them.  Bounded waits.
-            const uint32_t cbar = cbar_u32 + 8u * (uint32_t)par;
-            if (warp == kFWarps - 1) {
-                double cprod = 1.0;
-                const size_t r0 = bk * s.gamma;
+            // the ratio p_i(tok_i)/q_i(tok_i) of this row
+            const double ratio = exp2_short(((double)zp_tok - (double)rp_row) * (double)s.scale -
+                                            ((double)zq_tok - (double)rq_row) * (double)s.scale) *
+                                 (double)(Zq / Zp);
+            double cd;
+            if (row_mode) {
+                // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
+                // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
+                // NaN (a row that produces one is flagged invalid anyway).
+                if (lane == 0 && rank == 0 && i + 1 < s.gamma && !(p.withhold && i == 0))
+                    *reinterpret_cast<volatile double *>(p.ws.ratio + r) = (ratio != ratio) ? 0.0 : ratio;
+                // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
+                // butterfly over the lanes).  Those rows are walked by other clusters at about the same
+                // time and publish right after their own statistics, which do not depend on c: no chain of
+                // waits forms.  Every lane polls one of them.  Bounded waits.
+                cd = 1.0;
+                const size_t r0 = (size_t)bk * s.gamma;
                 for (int j0 = 0; j0 < i; j0 += 32) {
-                    double v = 1.0;
+                    double w = 1.0;
                     if (j0 + lane < i) {
-                        const volatile double *word =
-                            reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
-                        v = *word;
-                        if (v != v && timed_out) v = 0.0;
-                        if (v != v) {
+                        const volatile double *word = reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
+                        w = *word;
+                        if (w != w && timed_out) w = 0.0;
+                        if (w != w) {
                             const long long t0 = clock64();
-                            while ((v = *word) != v) {
+                            while ((w = *word) != w) {
                                 if (clock64() - t0 > p.poll_limit) {
                                     timed_out = true;
-                                    v = 0.0;
+                                    w = 0.0;
                                     break;
                                 }
                             }
                         }
                     }
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) v *= __shfl_xor_sync(0xffffffffu, v, o);
-                    cprod *= v;
+                    for (int o = 16; o > 0; o >>= 1) w *= __shfl_xor_sync(0xffffffffu, w, o);
+                    cd *= w;
                 }
-                if (lane == 0) {
-                    ctl->c[par] = cprod;
-                    mbar_arrive(cbar);  // c_i is there
+                timed_out = __any_sync(0xffffffffu, timed_out);
+            } else {
+                // c is carried along the chain: c_{i+1} = c_i ratio, and 1 at the start of the next chain
+                cd = c_carry;
+                c_carry = (i + 1 < s.gamma) ? cd * ratio : 1.0;
+            }
+            rs.rq = rq_row;
+            rs.rp = rp_row;
+            rs.c = (float)cd;
+            rs.kappa = (float)(cd * (double)(Zq / Zp));
+            if (lane == 0) {
+                ctl->rs = make_float4(rs.rq, rs.rp, rs.kappa, rs.c);
+                if (rank == 0) {
+                    // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
+                    // -inf only has Z = 0
+                    const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
+                                     !(bq_row < INFINITY) || !(bp_row < INFINITY);
+                    RowInfo ri;
+                    ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
+                    ri.pad_ = 0;
+                    ri.Zq = (double)Zq;
+                    ri.Zp = (double)Zp;
+                    ri.mq = bq_row;
+                    ri.mp = bp_row;
+                    ri.kappa = rs.kappa;
+                    ri.c = rs.c;
+                    p.ws.rows[r] = ri;
                 }
             }
-            mbar_wait(cbar, xph, timed_out);
-            timed_out = __any_sync(0xffffffffu, timed_out);
-            cd = ctl->c[par];
-        } else {
-            cd = ctl->c[par];
-            if (chain_thread && n + 1 < nrows) {
-                // c of the next row of the walk: c_{i+1} = c_i ratio, or 1 at the start of the next
-                // chain; publishing it arms the next row's exchange
-                ctl->c[par ^ 1] = (i + 1 < s.gamma) ? cd * SGBV_TOKEN_RATIO() : 1.0;
-                mbar_expect_tx(xbar_u32 + 8u * (uint32_t)(par ^ 1), xbytes);
-            }
+            __threadfence_block();
+            bar_arrive(2, kFThreads);
         }
-        RowScalars rs;
-        rs.rq = rq_row;
-        rs.rp = rp_row;
-        rs.c = (float)cd;
-        rs.kappa = (float)(cd * (double)(Zq / Zp));
         rs.scale = s.scale;
-
-        if (tid == 0 && rank == 0) {
-            // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
-            // -inf only has Z = 0
-            const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
-                             !(bq_row < INFINITY) || !(bp_row < INFINITY);
-            RowInfo ri;
-            ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
-            ri.pad_ = 0;
-            ri.Zq = (double)Zq;
-            ri.Zp = (double)Zp;
-            ri.mq = bq_row;
-            ri.mp = bp_row;
-            ri.kappa = rs.kappa;
-            ri.c = rs.c;
-            p.ws.rows[r] = ri;
-        }
 
         // ---- second sweep from tensor memory ----------------------------------------------------------
         float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
@@ -808,7 +793,6 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     __syncthreads();  // every warp of this CTA is done with the tensor memory
     if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 #undef SGBV_ISSUE_NEXT
-#undef SGBV_TOKEN_RATIO
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
