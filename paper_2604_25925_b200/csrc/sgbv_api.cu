@@ -107,8 +107,7 @@ int grow(void **ptr, size_t *have, size_t need, size_t preset_head = 0) {
 
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
-int g_opt_path = 0, g_opt_cluster = 0, g_opt_stages = 0, g_opt_max_clusters = 0, g_opt_walk = 0, g_opt_poll_us = 0,
-    g_opt_withhold = 0, g_opt_warps = 0;
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_max_clusters = 0, g_opt_walk = 0, g_opt_poll_us = 0, g_opt_withhold = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -318,9 +317,6 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "cluster")) {
         if (value < 0 || value > 8) return SGBV_ERR_SHAPE;
         g_opt_cluster = value;
-    } else if (!strcmp(name, "stages")) {
-        if (value < 0 || value > 12) return SGBV_ERR_SHAPE;
-        g_opt_stages = value;
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;
         g_opt_max_clusters = value;
@@ -330,16 +326,13 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "poll_us")) {
         if (value < 0 || value > 1000000) return SGBV_ERR_SHAPE;
         g_opt_poll_us = value;
-    } else if (!strcmp(name, "warps")) {
-        if (value != 0 && value != 16 && value != 32) return SGBV_ERR_SHAPE;
-        g_opt_warps = value;
     } else if (!strcmp(name, "withhold")) {
         if (value < 0 || value > 1) return SGBV_ERR_SHAPE;
         g_opt_withhold = value;
     } else {
         return SGBV_ERR_SHAPE;
     }
-    fused_set_options(g_opt_cluster, g_opt_stages, g_opt_max_clusters, g_opt_walk, g_opt_poll_us, g_opt_withhold, g_opt_warps);
+    fused_set_options(g_opt_cluster, g_opt_max_clusters, g_opt_walk, g_opt_poll_us, g_opt_withhold);
     return SGBV_OK;
 }
 

@@ -179,6 +179,6 @@ bool fused_supported(const Launch &L);
 // anything (the caller then takes the two-sweep path), or < 0
 // *walked_rows: the kernel used (and consumed the preset of) ws.ratio
 int launch_fused(const Launch &L, int *error_flag, bool *walked_rows);
-void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold, int warps);
+void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold);
 
 }  // namespace sgbv

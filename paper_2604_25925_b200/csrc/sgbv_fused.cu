@@ -42,7 +42,6 @@ constexpr int kCell = kTile;               // 256 contiguous entries: the unit a
 constexpr int kCtaCells = 128;             // cells of a row per CTA: 512 tensor-memory columns / 16 per cell, x 4 lane quarters
                                            // = 32,768 entries; a CTA of W warps gives each warp 128 / W cells
 constexpr int kTmemCols = 512;             // all of the SM's tensor memory (one CTA per SM)
-constexpr int kMaxSlots = 12;              // ring depth per warp
 constexpr int kMaxCluster = 8;             // portable cluster size
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 constexpr uint32_t kPollNs = 100u;                    // sleep between two tests of a barrier that is not ready
@@ -56,7 +55,6 @@ struct FusedParams {
     Workspace ws;
     int cluster;      // CTAs per cluster
     int slice_cells;  // cells of a row per CTA (at most kCtaCells)
-    int slots;        // ring depth per warp
     int nchains;      // B*K
     int *error_flag;  // set to 1 if a bounded wait expired
     long long poll_limit;  // cycles a poll of a published ratio may take (row walk)
@@ -73,9 +71,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -91,7 +86,7 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 // warp sleeps, so that a waiting warp leaves the issue slots to the working ones; the clock is read only
 // every 64 tests.  A thread that has given up once only tests from then on, so that the time a failing
 // kernel takes stays bounded.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool &gave_up) {
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t &gave_up) {
     if (mbar_test(bar, parity) || gave_up) return;
     uint32_t tests = 0;
     long long t0 = 0;
@@ -102,7 +97,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, bool &g
             const long long t = clock64();
             if (t0 == 0) t0 = t;
             else if (t - t0 > kWaitLimitCycles) {
-                gave_up = true;
+                gave_up = 1u;
                 return;
             }
         }
@@ -303,26 +298,28 @@ __device__ __forceinline__ void warp_sum_multi(float (&v)[P], int lane) {
     for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
 }
 
-// What the second sweep needs of a row, the same for every cell.
+// What the second sweep needs of a row from this thread's point of view.
 struct RowScalars {
-    float rq, rp;   // row maxima (0 where the row has none)
-    float kappa;    // c_i Zq / Zp: makes c p(x)/q(x) = kappa ep/eq in row-max units
-    float c;        // c_i
-    float scale;    // log2(e) / T
+    float Fq;     // moves sums in units of this thread's row maximum of zq to row-max units (0: the thread saw no finite zq)
+    float KF;     // kappa * Fp / Fq: with the cell's factor ratio it makes c p(x)/q(x) = kt * ep/eq
+    float kFp;    // kappa * Fp (cells whose target share underflows)
+    float c;      // c_i
 };
 
 // Second sweep over the warp's cells, read back from tensor memory, two vocabulary entries per
-// instruction (f32x2).  eq/ep are exponentials relative to the THREAD's maxima of the cell (mq[j],
-// mp[j]); kt = kappa * (fp / fq) makes c p(x)/q(x) = kt * ep/eq, where fq, fp move the thread's
-// units to row-max units.  Per cell:
+// instruction (f32x2).  eq/ep are exponentials relative to the THREAD's maxima of the cell;
+// fmq[j] moves cell j's target units to the thread's row units, rt[j] is the ratio of the cell's draft and
+// target factors, so that fq = fmq[j] Fq and kt = KF rt[j].  Per cell:
 //   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
 //   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
 //   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
-// The output pointers address this warp's first cell; its cells are kFWarps apart.
+// The output pointers address this warp's first cell; its cells are W apart.  fmp_stash: this thread's
+// draft factors of the cells in shared memory (cells apart by `stash_stride` floats), read only by a cell
+// whose target share underflows in a row with c < 1.
 template <int W, int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCtaCells / W], const float (&mp)[kCtaCells / W],
-                                          const RowScalars &rs, int K, int lane, int ncw, float *wpart, float *dpart,
-                                          float *mpart) {
+__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&fmq)[kCtaCells / W], const float (&rt)[kCtaCells / W],
+                                          const RowScalars &rs, int K, int lane, int ncw, const float *fmp_stash,
+                                          int stash_stride, float *wpart, float *dpart, float *mpart) {
     constexpr int kCellsPerWarp = kCtaCells / W, kFWarps = W;
     const float v1 = 1.0f - rs.c;
     const float2 nv1 = splat(-v1);
@@ -345,23 +342,22 @@ __device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCta
         float2 eq[4], ep[4];
         tmem_ld_cell(taddr + 16u * (uint32_t)j, eq, ep);
         // thread units -> row units
-        const float fq = (mq[j] > -INFINITY) ? ex2((mq[j] - rs.rq) * rs.scale) : 0.0f;
-        const float fp = (mp[j] > -INFINITY) ? ex2((mp[j] - rs.rp) * rs.scale) : 0.0f;
-        // equal factors (identical rows above all) must give kappa itself: p = q everywhere then leaves an
-        // exactly zero residual
-        float kt = (fp == fq) ? rs.kappa : rs.kappa * fp * rcp(fq);
-        float scale_w = fq, scale_d = fq;
-        const bool tiny = !(fq > 1e-30f);
+        float scale_w = fmq[j] * rs.Fq, scale_d = scale_w;
+        float kt = rs.KF * rt[j];
         tmem_wait_ld(eq, ep);
-        if (__any_sync(0xffffffffu, tiny)) {
-            // a thread whose share of the target row underflows (or nearly so, which would
-            // overflow kt): its q is 0 in row units, its weights vanish, and max(c p - q, 0) = c p
-            if (tiny) {
+        if (kAux) {
+            // A thread whose share of the target row underflows (or nearly so, which would overflow kt): its q
+            // is 0 in row units, its weights vanish, and max(c p - q, 0) = c p.  Without the extra sums nothing
+            // needs doing: an infinite or NaN kt gives a zero weight through the clamps below.
+            const bool tiny = !(scale_w > 1e-30f);
+            if (__any_sync(0xffffffffu, tiny)) {
+                if (tiny) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) eq[e] = splat(0.0f);
-                kt = 1.0f;
-                scale_w = 0.0f;
-                scale_d = rs.kappa * fp;
+                    for (int e = 0; e < 4; ++e) eq[e] = splat(0.0f);
+                    kt = 1.0f;
+                    scale_w = 0.0f;
+                    scale_d = rs.kFp * fmp_stash[j * stash_stride];
+                }
             }
         }
         const float2 nkt = splat(-kt);
@@ -413,38 +409,34 @@ __device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&mq)[kCta
     if ((lane & kOwnerMask) == 0 && idx < ncw) wpart[idx * kFWarps] = wsum[0];
 }
 
-// A warp's place in its stream of cell loads: cells j = 0..ncw-1 of walk position 0, then of position 1, ...
-// Kept by every lane (the values are warp-uniform); lane 0 starts the copies.
-struct LoadCursor {
-    const unsigned char *q, *p;  // this warp's first cell of the row being requested, in both tensors
-    int rows_left;               // rows whose cells have not all been requested
-    int j, i, slot;              // next cell of the row, position of the row in its chain, next ring slot
-    int bk;                      // chain of the row
-    int in_flight;               // loads issued and not consumed yet
-};
-
-// KT: the number of drafts K when it has a specialised second sweep (1, 2, 3, 4, 8), else 0 (any K, loops).
-template <typename T, bool kRow, int W, int KT>
+// W warps per CTA; NS ring slots per warp (the cells per warp and row, kCtaCells / W, are a multiple of it, so
+// that cell j of a row always sits in slot j % NS); KT: the number of drafts K when it has a specialised
+// second sweep (1, 2, 3, 4, 8), else 0 (any K, loops).
+template <typename T, bool kRow, int W, int NS, int KT>
 __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParams p) {
     constexpr int kFWarps = W, kFThreads = W * 32, kCellsPerWarp = kCtaCells / W;
+    static_assert(kCellsPerWarp % NS == 0, "cell j of a row must always land in slot j % NS");
     extern __shared__ __align__(1024) unsigned char smem[];
     const Shape &s = p.s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);  // (tells the compiler that it is the same in all lanes)
     const int C = p.cluster;
     const int rank = (int)cluster_ctarank();
     const int cid = blockIdx.x / C;
     const int G = gridDim.x / C;
-    const int NS = p.slots;
     constexpr int kHalfBytes = kCell * (int)sizeof(T);  // one tensor's cell
     constexpr int kSlotBytes = 2 * kHalfBytes;          // the cell of zq, then the same cell of zp
     constexpr int kStrideBytes = kFWarps * kHalfBytes;  // from one cell of a warp to its next, in a row
+    constexpr int kRingBytes = kFWarps * NS * kSlotBytes;
+    // [rings][full barriers][draft factors of every thread's cells][Control]
     const unsigned char *ring = smem + (size_t)warp * NS * kSlotBytes;
     const uint32_t ring_u32 = smem_u32(ring);
-    const uint32_t full_u32 = smem_u32(smem) + (uint32_t)(kFWarps * NS * kSlotBytes + warp * NS * 8);
-    Control *ctl = reinterpret_cast<Control *>(smem + (size_t)kFWarps * NS * (kSlotBytes + 8));
+    const uint32_t full_u32 = smem_u32(smem) + (uint32_t)(kRingBytes + warp * NS * 8);
+    float *fmp_stash = reinterpret_cast<float *>(smem + kRingBytes + kFWarps * NS * 8) + tid;  // [cell][thread]
+    Control *ctl = reinterpret_cast<Control *>(smem + kRingBytes + kFWarps * NS * 8 + kCellsPerWarp * kFThreads * 4);
     const uint32_t xbar_u32 = smem_u32(&ctl->xbar[0]);
 
-    // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + 32, ...
+    // this CTA's slice of the vocabulary, and this warp's cells in it: warp, warp + W, ...
     const int cell_begin = rank * p.slice_cells;
     const int ncells_cta = max(0, min(s.ntiles, cell_begin + p.slice_cells) - cell_begin);
     const int ncw = ncells_cta > warp ? (ncells_cta - warp + kFWarps - 1) / kFWarps : 0;  // cells of this warp per row
@@ -465,9 +457,8 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     tmem_fence_before();
     __syncthreads();
     tmem_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
-    // lanes of this warp's quarter, and its 64 columns
-    const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(warp >> 2) * (16u * kCellsPerWarp);
+    // lanes of this warp's quarter, and its columns
+    const uint32_t taddr = ctl->tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(warp >> 2) * (16u * kCellsPerWarp);
     cluster_arrive();  // every CTA of the cluster is running before any remote shared-memory access
     cluster_wait();
 
@@ -496,69 +487,59 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     const int nrows = row_mode ? (int)((total_rows - cid + G - 1) / G)
                                : ((p.nchains - cid + G - 1) / G) * s.gamma;  // rows this cluster walks
     const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
-    bool timed_out = false;
+    uint32_t timed_out = 0;
 
     // ---- this warp's copy ring --------------------------------------------------------------------
-    // Cell loads go out in consumption order: cell j = 0..ncw-1 of walk position 0, then of position 1, ...;
-    // a load lands in the slot that the cell NS before it has just left.  The cursor below (kept by every
-    // lane, the copies are started by lane 0) names the next load.  A warp that has given up on a wait
-    // issues no further loads and waits for those in flight only.
+    // Cell j of a row lands in slot j % NS.  The warp that has moved a cell from its slot to registers refills
+    // the slot at once with the next cell that maps to it: cell j + NS of the same row, or, past the warp's
+    // last cell, the slot's first cell of the next row of the walk.  So the schedule is fixed at compile time
+    // apart from the number of cells this warp has (ncw); lane 0 starts the copies.  `pending` has bit k set
+    // while a copy into slot k is under way, `phases` bit k is the parity of slot k's barrier.  A warp that has
+    // given up on a wait issues no further loads and, before it leaves, waits for those in flight.
     const size_t row_bytes = (size_t)s.V * sizeof(T);
-    LoadCursor lc;
-    lc.rows_left = ncw > 0 ? nrows : 0;
-    lc.j = 0;
-    lc.i = row_mode ? cid % s.gamma : 0;
-    lc.slot = 0;
-    lc.bk = row_mode ? cid / s.gamma : cid;
-    lc.in_flight = 0;
-    lc.q = reinterpret_cast<const unsigned char *>(p.zq) + (size_t)first_cell * kHalfBytes +
-           ((size_t)lc.bk * (s.gamma + 1) + lc.i) * row_bytes;
-    lc.p = reinterpret_cast<const unsigned char *>(p.zp) + (size_t)first_cell * kHalfBytes +
-           ((size_t)lc.bk * s.gamma + lc.i) * row_bytes;
+    const unsigned char *const zq_warp = reinterpret_cast<const unsigned char *>(p.zq) + (size_t)first_cell * kHalfBytes;
+    const unsigned char *const zp_warp = reinterpret_cast<const unsigned char *>(p.zp) + (size_t)first_cell * kHalfBytes;
     const uint32_t is_lane0 = lane == 0 ? 1u : 0u;
-#define SGBV_ISSUE_NEXT()                                                                                              \
+    uint32_t pending = 0, phases = 0;
+#define SGBV_ISSUE(QROW, PROW, JJ, SLOT)                                                                                \
     do {                                                                                                               \
-        if (lc.rows_left > 0 && !timed_out) { /* warp-uniform */                                                       \
-            const uint32_t bytes_ = (lc.j == tail_j) ? (uint32_t)(tail_valid * (int)sizeof(T)) : (uint32_t)kHalfBytes; \
-            issue_cell(ring_u32 + (uint32_t)(lc.slot * kSlotBytes), lc.q + (size_t)lc.j * kStrideBytes,                \
-                       lc.p + (size_t)lc.j * kStrideBytes, bytes_, full_u32 + 8u * (uint32_t)lc.slot, is_lane0,        \
-                       kHalfBytes);                                                                                    \
-            ++lc.in_flight;                                                                                            \
-            if (++lc.slot == NS) lc.slot = 0;                                                                          \
-            if (++lc.j == ncw) { /* on to the next row of the walk */                                                  \
-                lc.j = 0;                                                                                              \
-                --lc.rows_left;                                                                                        \
-                lc.bk += step_bk;                                                                                      \
-                lc.i += step_i;                                                                                        \
-                if (lc.i >= s.gamma) {                                                                                 \
-                    lc.i -= s.gamma;                                                                                   \
-                    lc.bk += wrap_bk;                                                                                  \
-                }                                                                                                      \
-                lc.q = reinterpret_cast<const unsigned char *>(p.zq) + (size_t)first_cell * kHalfBytes +               \
-                       ((size_t)lc.bk * (s.gamma + 1) + lc.i) * row_bytes;                                             \
-                lc.p = reinterpret_cast<const unsigned char *>(p.zp) + (size_t)first_cell * kHalfBytes +               \
-                       ((size_t)lc.bk * s.gamma + lc.i) * row_bytes;                                                   \
-            }                                                                                                          \
-        }                                                                                                              \
+        const uint32_t bytes_ = ((JJ) == tail_j) ? (uint32_t)(tail_valid * (int)sizeof(T)) : (uint32_t)kHalfBytes;      \
+        issue_cell(ring_u32 + (uint32_t)((SLOT) * kSlotBytes), (QROW) + (size_t)(JJ) * kStrideBytes,                    \
+                   (PROW) + (size_t)(JJ) * kStrideBytes, bytes_, full_u32 + 8u * (uint32_t)(SLOT), is_lane0, kHalfBytes); \
+        pending |= 1u << (SLOT);                                                                                       \
     } while (0)
-    for (int k = 0; k < NS; ++k) SGBV_ISSUE_NEXT();
-    int c_slot = 0;           // slot of the next cell to consume
-    uint32_t c_phase = 0;     // parity of that slot's barrier
+
+    int bk = row_mode ? cid / s.gamma : cid;
+    int i = row_mode ? cid % s.gamma : 0;
+    const unsigned char *q_cur = zq_warp + ((size_t)bk * (s.gamma + 1) + i) * row_bytes;  // this warp's first cell of the row
+    const unsigned char *p_cur = zp_warp + ((size_t)bk * s.gamma + i) * row_bytes;
+    if (nrows > 0) {
+#pragma unroll
+        for (int k = 0; k < NS; ++k)
+            if (k < ncw) SGBV_ISSUE(q_cur, p_cur, k, k);
+    }
 
     // The last warp of this CTA combines the partials, carries c_i and fetches the token logits one row
     // ahead (every lane the same words): tok_next is the token of the next row of the walk.
     const bool combiner = warp == kFWarps - 1;
     int tok_next = 0;
-    if (combiner && nrows > 0) tok_next = p.tok[row_mode ? (size_t)cid : (size_t)cid * s.gamma];
+    if (combiner && nrows > 0) tok_next = p.tok[(size_t)bk * s.gamma + i];
     double c_carry = 1.0;  // chain walk: c of the row at hand (the first row of the walk starts a chain)
 
-    int bk = row_mode ? cid / s.gamma : cid;
-    int i = row_mode ? cid % s.gamma : 0;
     for (int n = 0; n < nrows; ++n) {
         const size_t r = (size_t)bk * s.gamma + i;
         const int par = n & 1;
         const uint32_t xph = (uint32_t)(n >> 1) & 1u;
         const uint32_t xbar = xbar_u32 + 8u * (uint32_t)par;
+        // the next row of the walk (its cells are requested while this row is worked on)
+        int bk_n = bk + step_bk, i_n = i + step_i;
+        if (i_n >= s.gamma) {
+            i_n -= s.gamma;
+            bk_n += wrap_bk;
+        }
+        const bool more = n + 1 < nrows && !timed_out;
+        const unsigned char *q_nxt = zq_warp + ((size_t)bk_n * (s.gamma + 1) + i_n) * row_bytes;
+        const unsigned char *p_nxt = zp_warp + ((size_t)bk_n * s.gamma + i_n) * row_bytes;
 
         // ---- combining warp: the logits of this row's draft token, and the next row's token --------
         float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
@@ -568,15 +549,7 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
             if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
             zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk * (s.gamma + 1) + i) * s.V, t);
             zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + ((size_t)bk * s.gamma + i) * s.V, t);
-            if (n + 1 < nrows) {
-                int bk_n = bk + step_bk;
-                int i_n = i + step_i;
-                if (i_n >= s.gamma) {
-                    i_n -= s.gamma;
-                    bk_n += wrap_bk;
-                }
-                tok_next = p.tok[(size_t)bk_n * s.gamma + i_n];
-            }
+            if (n + 1 < nrows) tok_next = p.tok[(size_t)bk_n * s.gamma + i_n];
         }
 
         // ---- first sweep: ring -> exponentials in tensor memory, maximum and sum of every cell --------
@@ -589,14 +562,15 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
 #pragma unroll
         for (int j = 0; j < kCellsPerWarp; ++j) {
             if (j < ncw) {  // warp-uniform
-                if (lc.in_flight > 0) {
-                    mbar_wait(full_u32 + 8u * (uint32_t)c_slot, c_phase, timed_out);
-                    --lc.in_flight;
+                const int slot = j % NS;  // (a constant once the loop is unrolled)
+                if (pending & (1u << slot)) {
+                    mbar_wait(full_u32 + 8u * slot, (phases >> slot) & 1u, timed_out);
+                    phases ^= 1u << slot;
+                    pending ^= 1u << slot;
                 }
                 float2 eq[4], ep[4];
-                const unsigned char *base = ring + c_slot * kSlotBytes;
-                read_cell<T>(base, lane, eq);
-                read_cell<T>(base + kHalfBytes, lane, ep);
+                read_cell<T>(ring + slot * kSlotBytes, lane, eq);
+                read_cell<T>(ring + slot * kSlotBytes + kHalfBytes, lane, ep);
                 if (j == tail_j) {  // the row ends inside this cell
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -610,12 +584,12 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                     m1 = max3(m1, eq[e].x, eq[e].y);
                     m2 = max3(m2, ep[e].x, ep[e].y);
                 }
-                // every lane holds its share of the slot in registers now: refill it with the cell NS further on
+                // every lane holds its share of the slot in registers now: refill it
                 __syncwarp();
-                SGBV_ISSUE_NEXT();
-                if (++c_slot == NS) {
-                    c_slot = 0;
-                    c_phase ^= 1u;
+                if (j + NS < ncw) {
+                    if (!timed_out) SGBV_ISSUE(q_cur, p_cur, j + NS, slot);
+                } else if (more) {
+                    SGBV_ISSUE(q_nxt, p_nxt, slot, slot);
                 }
                 // reference points of this thread's exponentials: its own maxima of the cell (0 if it saw
                 // only -inf); the maximum itself maps to exactly 1, so point-mass rows stay exact
@@ -639,9 +613,12 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                 sp[j] = sp2.x + sp2.y;
             }
         }
+        timed_out = __any_sync(0xffffffffu, timed_out != 0);  // the warp gives up as one
         tmem_wait_st();
 
-        // ---- this thread's partial of the row: cell sums moved to its maximum over the cells ---------
+        // ---- this thread's partial of the row: cell sums moved to its maximum over the cells; what the
+        //      second sweep will need of every cell: fmq[j] = cell's target units -> thread's row units,
+        //      rt[j] = ratio of the cell's draft and target factors ------------------------------------
         float mqt = mq[0], mpt = mp[0];
 #pragma unroll
         for (int j = 1; j < kCellsPerWarp; ++j) {
@@ -651,11 +628,18 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
         const bool has_q = mqt > -INFINITY, has_p = mpt > -INFINITY;
         const float bqt = has_q ? mqt : 0.0f, bpt = has_p ? mpt : 0.0f;
         float sqt = 0.0f, spt = 0.0f;
+        float fmq[kCellsPerWarp], rt[kCellsPerWarp];
 #pragma unroll
         for (int j = 0; j < kCellsPerWarp; ++j) {
+            fmq[j] = rt[j] = 0.0f;
             if (j < ncw) {  // a cell without a finite entry has sum 0 and factor 2^-inf = 0
-                sqt = fmaf(sq[j], ex2((mq[j] - bqt) * s.scale), sqt);
-                spt = fmaf(sp[j], ex2((mp[j] - bpt) * s.scale), spt);
+                const float dq = (mq[j] - bqt) * s.scale, dp = (mp[j] - bpt) * s.scale;
+                const float fmp = ex2(dp);
+                fmq[j] = ex2(dq);
+                rt[j] = ex2(dp - dq);  // (NaN or inf where a factor is 0: those cells weigh nothing)
+                sqt = fmaf(sq[j], fmq[j], sqt);
+                spt = fmaf(sp[j], fmp, spt);
+                fmp_stash[j * kFThreads] = fmp;
             }
         }
         // warp partials relative to the warp's maxima
@@ -670,15 +654,11 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
         // issue slots: barrier 1 = "all partials are in", barrier 2 = "the row's scalars are in".
         if (lane == 0) ctl->wslots[warp] = make_float4(bqw, sqt, bpw, spt);
         __threadfence_block();
-        RowScalars rs;
-        if (warp != kFWarps - 1) {
+        float4 rowv;  // rq, rp, kappa, c
+        if (!combiner) {
             bar_arrive(1, kFThreads);
             bar_sync(2, kFThreads);
-            const float4 v = ctl->rs;  // (the barrier statement is a compiler barrier for memory)
-            rs.rq = v.x;
-            rs.rp = v.y;
-            rs.kappa = v.z;
-            rs.c = v.w;
+            rowv = ctl->rs;  // (the barrier statement is a compiler barrier for memory)
         } else {
             bar_sync(1, kFThreads);
             const float4 v = lane < kFWarps ? ctl->wslots[lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
@@ -689,7 +669,7 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
             if (C > 1) {  // the same once more over the CTAs of the cluster
                 if (lane < C) push_f4(&ctl->slots[par][rank], xbar, (uint32_t)lane, make_float4(bq_row, Zq, bp_row, Zp));
                 mbar_wait(xbar, xph, timed_out);
-                timed_out = __any_sync(0xffffffffu, timed_out);  // the warp gives up as one
+                timed_out = __any_sync(0xffffffffu, timed_out != 0);
                 const float4 cv = lane < C ? ctl->slots[par][lane] : make_float4(-INFINITY, 0.0f, -INFINITY, 0.0f);
                 bq_row = warp_max_redux(cv.x);
                 bp_row = warp_max_redux(cv.z);
@@ -725,7 +705,7 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                             const long long t0 = clock64();
                             while ((w = *word) != w) {
                                 if (clock64() - t0 > p.poll_limit) {
-                                    timed_out = true;
+                                    timed_out = 1;
                                     w = 0.0;
                                     break;
                                 }
@@ -736,18 +716,15 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                     for (int o = 16; o > 0; o >>= 1) w *= __shfl_xor_sync(0xffffffffu, w, o);
                     cd *= w;
                 }
-                timed_out = __any_sync(0xffffffffu, timed_out);
+                timed_out = __any_sync(0xffffffffu, timed_out != 0);
             } else {
                 // c is carried along the chain: c_{i+1} = c_i ratio, and 1 at the start of the next chain
                 cd = c_carry;
                 c_carry = (i + 1 < s.gamma) ? cd * ratio : 1.0;
             }
-            rs.rq = rq_row;
-            rs.rp = rp_row;
-            rs.c = (float)cd;
-            rs.kappa = (float)(cd * (double)(Zq / Zp));
+            rowv = make_float4(rq_row, rp_row, (float)(cd * (double)(Zq / Zp)), (float)cd);
             if (lane == 0) {
-                ctl->rs = make_float4(rs.rq, rs.rp, rs.kappa, rs.c);
+                ctl->rs = rowv;
                 if (rank == 0) {
                     // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
                     // -inf only has Z = 0
@@ -760,68 +737,84 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                     ri.Zp = (double)Zp;
                     ri.mq = bq_row;
                     ri.mp = bp_row;
-                    ri.kappa = rs.kappa;
-                    ri.c = rs.c;
+                    ri.kappa = rowv.z;
+                    ri.c = rowv.w;
                     p.ws.rows[r] = ri;
                 }
             }
             __threadfence_block();
             bar_arrive(2, kFThreads);
         }
-        rs.scale = s.scale;
+        // this thread's row units -> row-max units
+        RowScalars rs;
+        const float Fp = has_p ? ex2((bpt - rowv.y) * s.scale) : 0.0f;
+        rs.Fq = has_q ? ex2((bqt - rowv.x) * s.scale) : 0.0f;
+        // equal factors (identical rows above all) must give kappa itself: p = q everywhere then leaves an
+        // exactly zero residual
+        rs.KF = (Fp == rs.Fq) ? rowv.z : rowv.z * Fp * rcp(rs.Fq);
+        rs.kFp = rowv.z * Fp;
+        rs.c = rowv.w;
 
         // ---- second sweep from tensor memory ----------------------------------------------------------
         float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
               *mpp = p.ws.mpart + r * s.ntiles + first_cell;
         if (rs.c < 1.0f)
-            sweep_two<W, KT, true>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+            sweep_two<W, KT, true>(taddr, fmq, rt, rs, s.K, lane, ncw, fmp_stash, kFThreads, wp, dp, mpp);
         else
-            sweep_two<W, KT, false>(taddr, mq, mp, rs, s.K, lane, ncw, wp, dp, mpp);
+            sweep_two<W, KT, false>(taddr, fmq, rt, rs, s.K, lane, ncw, fmp_stash, kFThreads, wp, dp, mpp);
 
         // one step of the walk
-        bk += step_bk;
-        i += step_i;
-        if (i >= s.gamma) {
-            i -= s.gamma;
-            bk += wrap_bk;
-        }
+        bk = bk_n;
+        i = i_n;
+        q_cur = q_nxt;
+        p_cur = p_nxt;
     }
-    if (__any_sync(0xffffffffu, timed_out) && lane == 0) atomicExch(p.error_flag, 1);
+    // a warp that gave up may still have copies under way: they must land before the shared memory goes
+    if (timed_out) {
+        uint32_t fresh = 0;
+#pragma unroll
+        for (int k = 0; k < NS; ++k)
+            if (pending & (1u << k)) mbar_wait(full_u32 + 8u * k, (phases >> k) & 1u, fresh);
+        if (lane == 0) atomicExch(p.error_flag, 1);
+    }
     cluster_arrive();  // no CTA leaves while a neighbour may still write into its slots
     cluster_wait();
     tmem_fence_before();
     __syncthreads();  // every warp of this CTA is done with the tensor memory
-    if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
-#undef SGBV_ISSUE_NEXT
+    if (warp == 0) tmem_dealloc(ctl->tmem_base, kTmemCols);
+#undef SGBV_ISSUE
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
 struct Plan {
-    int cluster, slice_cells, slots, grid_clusters, row_mode;
-    size_t smem;
+    int cluster, slice_cells, row_mode;
 };
 
 int g_opt_cluster = 0;     // 0 = automatic
-int g_opt_slots = 0;
 int g_opt_max_clusters = 0;
 int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
 int g_opt_poll_us = 0;     // 0 = about a second
 int g_opt_withhold = 0;
-int g_opt_warps = 0;       // 0 = automatic, 16 or 32
 
 constexpr int kSmemPerCta = 227 * 1024;    // largest dynamic shared memory of one CTA
 constexpr int kDevices = 64;
 std::mutex g_plan_mu;      // guards the options and the per-device caches below
 
-size_t slot_bytes(int dtype) { return 2 * (size_t)kCell * (dtype == SGBV_DTYPE_BF16 ? 2 : 4); }
-size_t smem_bytes(int dtype, int warps, int slots) { return (size_t)warps * slots * (slot_bytes(dtype) + 8) + sizeof(Control); }
+constexpr int kWarps = 32;  // warps per CTA
+// ring slots per warp: half a row's cells for float32 (128 KB of copies under way per SM), all of them for bfloat16
+template <typename T>
+constexpr int slots_for() { return sizeof(T) == 4 ? 2 : 4; }
+template <typename T>
+constexpr size_t smem_bytes() {
+    return (size_t)kWarps * slots_for<T>() * (2 * kCell * sizeof(T) + 8) + (size_t)(kCtaCells / kWarps) * kWarps * 32 * 4 + sizeof(Control);
+}
 int slice_cells_of(int cells, int C) { return (cells + C - 1) / C; }
 
-template <typename T, bool kRow, int W, int KT>
+template <typename T, bool kRow, int KT>
 cudaError_t prepare(int dev) {
     static bool attr_done[kDevices];
     if (!attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow, W, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
+        cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow, kWarps, slots_for<T>(), KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
         if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
@@ -829,14 +822,14 @@ cudaError_t prepare(int dev) {
 }
 
 // Clusters of C CTAs of this kernel that the device runs side by side (queried once per configuration).
-template <typename T, bool kRow, int W, int KT>
-int resident_clusters(int dev, int C, int slots, size_t smem) {
-    static int cached[kDevices][kMaxCluster + 1][kMaxSlots + 1];
-    int &slot = cached[dev][C][slots];
+template <typename T, bool kRow, int KT>
+int resident_clusters(int dev, int C) {
+    static int cached[kDevices][kMaxCluster + 1];
+    int &slot = cached[dev][C];
     if (slot == 0) {
         cudaLaunchConfig_t cfg = {};
-        cfg.blockDim = dim3(W * 32);
-        cfg.dynamicSmemBytes = smem;
+        cfg.blockDim = dim3(kWarps * 32);
+        cfg.dynamicSmemBytes = smem_bytes<T>();
         cfg.gridDim = dim3(C * (148 / C));
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -846,7 +839,7 @@ int resident_clusters(int dev, int C, int slots, size_t smem) {
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int nmax = 0;
-        if (cudaOccupancyMaxActiveClusters(&nmax, fused_chain_kernel<T, kRow, W, KT>, &cfg) != cudaSuccess || nmax < 1) {
+        if (cudaOccupancyMaxActiveClusters(&nmax, fused_chain_kernel<T, kRow, kWarps, slots_for<T>(), KT>, &cfg) != cudaSuccess || nmax < 1) {
             cudaGetLastError();
             return 0;
         }
@@ -855,7 +848,7 @@ int resident_clusters(int dev, int C, int slots, size_t smem) {
     return slot;
 }
 
-template <typename T, bool kRow, int W, int KT>
+template <typename T, bool kRow, int KT>
 int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) {
     FusedParams fp;
     fp.zq = L.zq;
@@ -865,15 +858,14 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
     fp.ws = L.ws;
     fp.cluster = plan.cluster;
     fp.slice_cells = plan.slice_cells;
-    fp.slots = plan.slots;
     fp.nchains = L.s.B * L.s.K;
     fp.error_flag = error_flag;
     fp.poll_limit = g_opt_poll_us > 0 ? (long long)g_opt_poll_us * 2000ll : kWaitLimitCycles;
     fp.withhold = g_opt_withhold;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(W * 32);
-    cfg.dynamicSmemBytes = plan.smem;
+    cfg.blockDim = dim3(kWarps * 32);
+    cfg.dynamicSmemBytes = smem_bytes<T>();
     cfg.stream = L.stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -891,7 +883,7 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
         cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
         return SGBV_ERR_CUDA;
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_chain_kernel<T, kRow, W, KT>, fp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, fused_chain_kernel<T, kRow, kWarps, slots_for<T>(), KT>, fp);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -901,40 +893,29 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
 }
 
 // Chooses the cluster size and the walk, then launches.  Returns launches, 0 if declined, or < 0.
-template <typename T, int W, int KT>
+template <typename T, int KT>
 int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const Shape &s = L.s;
     const int cells = s.ntiles;
     const long nchains = (long)s.B * s.K, units = nchains * s.gamma;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDevices) return SGBV_ERR_CUDA;
-    if (prepare<T, false, W, KT>(dev) != cudaSuccess || prepare<T, true, W, KT>(dev) != cudaSuccess) {
+    if (prepare<T, false, KT>(dev) != cudaSuccess || prepare<T, true, KT>(dev) != cudaSuccess) {
         cudaGetLastError();
         return SGBV_ERR_CUDA;
     }
     Plan plan;
-    // ring depth: what fits beside the control block, at most the default (deeper rings keep more bytes
-    // in flight than the memory system rewards)
-    const int max_slots = (int)std::min<size_t>(kMaxSlots, (kSmemPerCta - sizeof(Control)) / ((size_t)W * (slot_bytes(L.dtype) + 8)));
-    int slots = g_opt_slots ? g_opt_slots : (W == 32 ? 3 : 6) * (L.dtype == SGBV_DTYPE_BF16 ? 2 : 1);
-    if (slots > max_slots) {
-        if (g_opt_slots) return SGBV_ERR_SHAPE;
-        slots = max_slots;
-    }
-    plan.slots = slots;
-    plan.smem = smem_bytes(L.dtype, W, slots);
     int Cmin = (cells + kCtaCells - 1) / kCtaCells;  // smallest cluster whose slices fit the tensor memory
     if (Cmin > kMaxCluster) return 0;
     auto fits = [&](int C) { return C >= Cmin && C <= kMaxCluster; };
     auto resident = [&](int C, bool row) {
-        return row ? resident_clusters<T, true, W, KT>(dev, C, plan.slots, plan.smem)
-                   : resident_clusters<T, false, W, KT>(dev, C, plan.slots, plan.smem);
+        return row ? resident_clusters<T, true, KT>(dev, C) : resident_clusters<T, false, KT>(dev, C);
     };
     // Few units of work: spread each over more CTAs (at least half the warps keep a cell) while all of them
     // still run side by side.
     auto widen = [&](long n_units, bool row) {
         int C = Cmin;
-        while (2 * C <= kMaxCluster && cells >= C * W && n_units <= resident(2 * C, row)) C *= 2;
+        while (2 * C <= kMaxCluster && cells >= C * kWarps && n_units <= resident(2 * C, row)) C *= 2;
         return C;
     };
     int C = g_opt_cluster ? g_opt_cluster : widen(nchains, false);
@@ -957,21 +938,19 @@ int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const long share = plan.row_mode ? units : nchains;  // what the clusters share out
     if (clusters > share) clusters = (int)share;
     *walked_rows = plan.row_mode != 0;
-    return plan.row_mode ? launch_as<T, true, W, KT>(L, plan, error_flag, clusters)
-                         : launch_as<T, false, W, KT>(L, plan, error_flag, clusters);
+    return plan.row_mode ? launch_as<T, true, KT>(L, plan, error_flag, clusters)
+                         : launch_as<T, false, KT>(L, plan, error_flag, clusters);
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int slots, int max_clusters, int walk, int poll_us, int withhold, int warps) {
+void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold) {
     std::lock_guard<std::mutex> lock(g_plan_mu);
     g_opt_withhold = withhold;
     g_opt_walk = walk;
     g_opt_cluster = cluster;
-    g_opt_slots = slots;
     g_opt_max_clusters = max_clusters;
     g_opt_poll_us = poll_us;
-    g_opt_warps = warps;
 }
 
 // Whether the fused path can take this call: rows must be 16-byte aligned for the bulk copies and a
@@ -982,26 +961,23 @@ bool fused_supported(const Launch &L) {
     return L.s.ntiles <= kMaxCluster * kCtaCells;
 }
 
-template <typename T, int W>
+template <typename T>
 int dispatch_k(const Launch &L, int *error_flag, bool *walked_rows) {
     switch (L.s.K) {
-        case 1: return plan_and_launch<T, W, 1>(L, error_flag, walked_rows);
-        case 2: return plan_and_launch<T, W, 2>(L, error_flag, walked_rows);
-        case 3: return plan_and_launch<T, W, 3>(L, error_flag, walked_rows);
-        case 4: return plan_and_launch<T, W, 4>(L, error_flag, walked_rows);
-        case 8: return plan_and_launch<T, W, 8>(L, error_flag, walked_rows);
-        default: return plan_and_launch<T, W, 0>(L, error_flag, walked_rows);
+        case 1: return plan_and_launch<T, 1>(L, error_flag, walked_rows);
+        case 2: return plan_and_launch<T, 2>(L, error_flag, walked_rows);
+        case 3: return plan_and_launch<T, 3>(L, error_flag, walked_rows);
+        case 4: return plan_and_launch<T, 4>(L, error_flag, walked_rows);
+        case 8: return plan_and_launch<T, 8>(L, error_flag, walked_rows);
+        default: return plan_and_launch<T, 0>(L, error_flag, walked_rows);
     }
 }
 
 int launch_fused(const Launch &L, int *error_flag, bool *walked_rows) {
     *walked_rows = false;
     std::lock_guard<std::mutex> lock(g_plan_mu);
-    const int warps = g_opt_warps ? g_opt_warps : 32;
-    if (L.dtype == SGBV_DTYPE_BF16)
-        return warps == 16 ? dispatch_k<uint16_t, 16>(L, error_flag, walked_rows)
-                           : dispatch_k<uint16_t, 32>(L, error_flag, walked_rows);
-    return warps == 16 ? dispatch_k<float, 16>(L, error_flag, walked_rows) : dispatch_k<float, 32>(L, error_flag, walked_rows);
+    return L.dtype == SGBV_DTYPE_BF16 ? dispatch_k<uint16_t>(L, error_flag, walked_rows)
+                                      : dispatch_k<float>(L, error_flag, walked_rows);
 }
 
 }  // namespace sgbv
