@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 
 L2_BYTES = 126e6
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0        # the nominal peak the fractions are also quoted against
 
 
 def describe(cfg) -> str:
@@ -151,6 +152,20 @@ def time_oracle(cfg, inp_cpu, budget_s: float = 12.0):
             f"first {rows} of {cfg.B} batch rows of one {cfg.name} step, scaled to whole steps", res, rows)
 
 
+def config_dict(cfg, nsets=None, set_bytes=None) -> dict:
+    """The `config` object of the JSON line; the same from both arms."""
+    d = {"workload": describe(cfg), "per_rank_batch": cfg.B}
+    if nsets is not None:
+        d["l2"] = (f"{nsets} rotating input sets of {set_bytes / 1e6:.1f} MB ({nsets * set_bytes / 1e6:.0f} MB total, "
+                   "L2 is 126 MB)" + ("" if nsets * set_bytes >= 2 * L2_BYTES else ": NOT larger than L2, no flush"))
+    return d
+
+
+def rotating_sets(cfg) -> int:
+    """Enough input sets to exceed twice the L2; capped for toy shapes, whose line then says that they stay in L2."""
+    return int(min(512, max(2, math.ceil(2.2 * L2_BYTES / cfg.logit_bytes()))))
+
+
 def run_reference(args):
     """The oracle as the reference arm: rank 0 only, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -182,12 +197,128 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "verify_steps_per_s", "value": value, "unit": "verify-steps/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": describe(cfg)},
+            "config": config_dict(cfg, rotating_sets(cfg), cfg.logit_bytes()),
             "cpu_baseline": {"value": value, "unit": "verify-steps/s", "cores": int(res.threads), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": "verify-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+class Workload:
+    """One configuration resident on the device: rotating input sets, output buffers, prepared C-ABI calls."""
+
+    def __init__(self, cfg, dev, rank):
+        import torch
+        from paper_2604_25925_b200 import binding, workloads
+        self.cfg, self.dev = cfg, dev
+        self.nsets = rotating_sets(cfg)
+        self.sets = [workloads.make_inputs(cfg, device=dev, set_index=rank * 1000 + i) for i in range(self.nsets)]
+        self.outs = [binding.VerifyOutput(torch.empty(cfg.B, dtype=torch.int32, device=dev),
+                                          torch.empty(cfg.B, dtype=torch.int32, device=dev),
+                                          torch.empty((cfg.B, cfg.gamma + 1), dtype=torch.int32, device=dev))
+                     for _ in range(self.nsets)]
+        lib = binding.load()
+        self.fn = lib.sgbv_verify_bf16 if cfg.dtype == "bf16" else lib.sgbv_verify
+        self.stream = torch.cuda.current_stream(dev)
+        self.calls = [(i.target_logits.data_ptr(), i.draft_logits.data_ptr(), i.draft_tokens.data_ptr(),
+                       i.uniforms.data_ptr(), cfg.B, cfg.K, cfg.gamma, cfg.V, float(cfg.temperature),
+                       o.accept_len.data_ptr(), o.draft_idx.data_ptr(), o.tokens.data_ptr(), self.stream.cuda_stream)
+                      for i, o in zip(self.sets, self.outs)]
+        self.count = 0
+
+    def step(self):
+        from paper_2604_25925_b200 import binding
+        rc = self.fn(*self.calls[self.count % self.nsets])
+        self.count += 1
+        if rc != 0:
+            raise binding.SgbvError(rc)
+
+
+def timed_blocks(wl, steps, warmup, world, min_seconds=1.0, max_repeats=400):
+    """Blocks of exactly `steps` steps, each bracketed by a barrier and a synchronisation on both sides and timed
+    with CUDA events on the launching stream, repeated until `min_seconds` have been timed.  Returns the per-block
+    milliseconds (max over ranks), the wall-clock interval, and the kernel launches per step."""
+    import torch
+    import torch.distributed as dist
+    from paper_2604_25925_b200 import binding, sharding
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    launches_per_step = binding.last_launch_count()
+    blocks, total = [], 0.0
+    t0 = time.time()
+    while True:
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(wl.stream)
+        for _ in range(steps):
+            wl.step()
+        ev1.record(wl.stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), device=wl.dev)   # a block takes as long as its slowest rank
+        blocks.append(ms)
+        total += ms
+        if total >= 1e3 * min_seconds or len(blocks) >= max_repeats:   # (the same decision on every rank: ms is the max)
+            break
+    return blocks, (t0, time.time()), launches_per_step
+
+
+def kernel_pass(wl, n):
+    """A separate pass of n steps with an event pair around the streaming kernel of every step (the pairs sit between
+    the kernels of a step, so this pass is not the one `value` comes from).  -> (mean kernel ms, launches timed)"""
+    import torch
+    from paper_2604_25925_b200 import binding
+    binding.profile_begin(n)
+    for _ in range(n):
+        wl.step()
+    torch.cuda.synchronize()
+    ms, cnt = binding.profile_end()
+    return ms / max(cnt, 1), cnt
+
+
+def parity_report(wl, budget_s):
+    """Oracle on the host cores against the CUDA path on the first input set (whole batch or its first rows)."""
+    import torch
+    from oracle.compare import compare
+    from paper_2604_25925_b200 import binding
+    cfg = wl.cfg
+    host = wl.sets[0].to("cpu")
+    v, cores, sample, ref, rows = time_oracle(cfg, host, budget_s)
+    s0 = wl.sets[0]
+    dx = binding.sgbv_verify_ex(s0.target_logits, s0.draft_logits, s0.draft_tokens, s0.uniforms, cfg.temperature)
+    torch.cuda.synchronize()
+    sl = slice(None) if rows is None else slice(0, rows)
+    rep = compare(ref, dx.accept_len[sl].cpu().numpy(), dx.draft_idx[sl].cpu().numpy(), dx.tokens[sl].cpu().numpy(),
+                  dx.h[sl].cpu().numpy(), dx.resmass[sl].cpu().numpy(), dx.status[sl].cpu().numpy())
+    return rep.summary(), {"value": v, "unit": "verify-steps/s", "cores": int(cores), "kind": "oracle", "sample": sample}
+
+
+def roofline_of(wl, ab, kern_ms, kern_n):
+    from paper_2604_25925_b200 import binding
+    peak, which = hbm_peak()
+    achieved = ab["sweep"] / (kern_ms * 1e-3) / 1e9 if kern_n else None
+    return {"bound": "hbm", "kernel": binding.last_main_kernel(), "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": (achieved / peak) if achieved else None, "peak_source": f"of {which}",
+            "frac_of_nominal_8000": (achieved / NOMINAL_HBM_GBS) if achieved else None,
+            "kernel_ms": kern_ms, "launches_timed": kern_n, "algorithmic_bytes_per_launch": ab["sweep"],
+            "traffic": kernel_traffic(wl.cfg.name)}
+
+
+def block_facts(wl):
+    """Mean number of fully accepted batch rows (they cost one more vocabulary row each) and block efficiency."""
+    g = wl.cfg.gamma
+    used = wl.outs[:min(wl.nsets, max(1, wl.count))]
+    n_bonus = float(sum(int((o.accept_len == g).sum().item()) for o in used)) / len(used)
+    be = float(sum(float((o.accept_len.float() + 1).mean().item()) for o in used)) / len(used)
+    return n_bonus, be
+
+
+PER_CONFIG = ("c2", "c3", "c5_K1_a0.8_T1.0", "c5_K8_a0.8_T1.0")
 
 
 def main():
@@ -196,9 +327,10 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 3
@@ -208,7 +340,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2604_25925_b200 import binding, sharding, workloads
+    from paper_2604_25925_b200 import binding, workloads
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -221,34 +353,11 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = workloads.get_config(args.workload)
-    set_bytes = cfg.logit_bytes()
-    # enough input sets to exceed twice the L2; capped for toy shapes, whose line then says that they stay in L2
-    nsets = int(min(512, max(2, math.ceil(2.2 * L2_BYTES / set_bytes))))
-    est_ms = max(0.02, set_bytes / 2.5e9)                  # rough step time for choosing defaults
-    steps = args.steps if args.steps is not None else int(max(20, min(50000, 4000.0 / est_ms)))
-    warmup = args.warmup if args.warmup is not None else max(3, min(50, steps // 10))
-    warmup = max(3, warmup)
+    est_ms = max(0.02, cfg.logit_bytes() / 4.0e9)             # rough step time for choosing defaults
+    steps = args.steps if args.steps is not None else int(max(20, min(2000, 50.0 / est_ms)))
+    warmup = max(3, args.warmup if args.warmup is not None else min(50, steps // 4))
 
-    sets = [workloads.make_inputs(cfg, device=dev, set_index=rank * 1000 + i) for i in range(nsets)]
-    outs = [binding.VerifyOutput(torch.empty(cfg.B, dtype=torch.int32, device=dev),
-                                 torch.empty(cfg.B, dtype=torch.int32, device=dev),
-                                 torch.empty((cfg.B, cfg.gamma + 1), dtype=torch.int32, device=dev))
-            for _ in range(nsets)]
-    lib = binding.load()
-    fn = lib.sgbv_verify_bf16 if cfg.dtype == "bf16" else lib.sgbv_verify
-    stream = torch.cuda.current_stream(dev)
-    calls = []
-    for inp, out in zip(sets, outs):
-        calls.append((inp.target_logits.data_ptr(), inp.draft_logits.data_ptr(), inp.draft_tokens.data_ptr(),
-                      inp.uniforms.data_ptr(), cfg.B, cfg.K, cfg.gamma, cfg.V, float(cfg.temperature),
-                      out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(),
-                      stream.cuda_stream))
-
-    def step(i):
-        rc = fn(*calls[i % nsets])
-        if rc != 0:
-            raise binding.SgbvError(rc)
-
+    wl = Workload(cfg, dev, rank)
     uuid = None
     try:
         uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
@@ -257,70 +366,36 @@ def main():
     sampler = ClockSampler(uuid) if rank == 0 else None
     time.sleep(0.25)
     # the warm-up steps run right before the timed ones (the sampler's start-up pause would let the GPU idle)
-    for i in range(warmup):
-        step(i)
-    torch.cuda.synchronize()
-    launches_per_step = binding.last_launch_count()
-    # event pairs around the streaming kernel on a tenth of the timed steps at most: the records sit between
-    # the two kernels of a step and between steps, where they cost the overlap that the launches otherwise have
-    nrec = max(1, min(steps // 10, 4000))
-    binding.profile_begin(nrec)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
-    ev0.record(stream)
-    for i in range(steps):
-        step(i)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    t1 = time.time()
-    if world > 1:
-        dist.barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    kern_ms, kern_n = binding.profile_end()
-    ms_total = sharding.max_over_ranks(ms_total, device=dev)   # a step takes as long as its slowest rank
+    blocks, (t0, t1), launches_per_step = timed_blocks(wl, steps, warmup, world)
     clocks = sampler.stop(t0, t1) if sampler else None
+    kern_ms, kern_n = kernel_pass(wl, max(20, min(steps, 200)))
+    n_bonus, be = block_facts(wl)
 
-    # parity-relevant facts of the timed outputs, and the end-to-end / CPU legs (rank 0)
-    n_bonus = float(sum(int((o.accept_len == cfg.gamma).sum().item()) for o in outs)) / nsets
-    be = float(sum(float((o.accept_len.float() + 1).mean().item()) for o in outs)) / nsets
     if rank == 0:
         ab = algorithmic_bytes(cfg, n_bonus)
-        ms_step = ms_total / steps
-        value = world * steps / (ms_total * 1e-3)
-        peak, which = hbm_peak()
-        kern_avg_ms = kern_ms / max(kern_n, 1)
-        achieved = ab["sweep"] / (kern_avg_ms * 1e-3) / 1e9 if kern_n else None
+        ms_block = sorted(blocks)[len(blocks) // 2]           # the median block
+        ms_step = ms_block / steps
         line = {
-            "metric": "verify_steps_per_s", "value": value, "unit": "verify-steps/s", "n_gpus": world,
-            "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": describe(cfg),
-                       "l2": f"{nsets} rotating input sets of {set_bytes / 1e6:.1f} MB "
-                             f"({nsets * set_bytes / 1e6:.0f} MB total, L2 is 126 MB)"
-                             + ("" if nsets * set_bytes >= 2 * L2_BYTES else ": NOT larger than L2, no flush"),
-                       "per_rank_batch": cfg.B},
+            "metric": "verify_steps_per_s", "value": world * steps / (ms_block * 1e-3), "unit": "verify-steps/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "repeats": len(blocks), "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": config_dict(cfg, wl.nsets, cfg.logit_bytes()),
             "hbm_gbs_step": ab["step"] / (ms_step * 1e-3) / 1e9,
             "algorithmic_bytes_per_step": ab["step"],
             "block_efficiency": be,
-            "roofline": {"bound": "hbm", "kernel": binding.last_main_kernel(), "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-                         "peak_source": f"of {which}", "kernel_ms": kern_avg_ms, "launches_timed": kern_n,
-                         "algorithmic_bytes_per_launch": ab["sweep"], "traffic": kernel_traffic(cfg.name)},
+            "roofline": roofline_of(wl, ab, kern_ms, kern_n),
             "gpu_launches": launches_per_step * steps,
             "clocks": clocks,
         }
         if not args.no_e2e:
-            host = sets[0].to("cpu")
+            host = wl.sets[0].to("cpu")
             pinned = [t.pin_memory() for t in (host.target_logits, host.draft_logits, host.draft_tokens,
                                                host.uniforms)]
             hout = binding.VerifyOutput(torch.empty(cfg.B, dtype=torch.int32).pin_memory(),
                                         torch.empty(cfg.B, dtype=torch.int32).pin_memory(),
                                         torch.empty((cfg.B, cfg.gamma + 1), dtype=torch.int32).pin_memory(),
                                         status=torch.empty(cfg.B, dtype=torch.int32).pin_memory())
-            e_steps = int(max(3, min(steps, 2.0 / max(set_bytes / 20e9, 1e-4))))
+            e_steps = int(max(3, min(steps, 2.0 / max(cfg.logit_bytes() / 20e9, 1e-4))))
             for _ in range(2):
                 binding.sgbv_verify_host(*pinned, cfg.temperature, out=hout, device=local)
             t = time.perf_counter()
@@ -333,20 +408,34 @@ def main():
             line["e2e"] = {"value": world * e_steps / dt, "unit": "verify-steps/s", "h2d_bytes_per_step": h2d,
                            "d2h_bytes_per_step": d2h, "steps": e_steps,
                            "note": "sgbv_verify_host: pinned host buffers, copies and sync inside the timed region"}
+            del pinned, host
         if not args.no_cpu_baseline:
-            from oracle.compare import compare
-            host = sets[0].to("cpu")
-            v, cores, sample, ref, rows = time_oracle(cfg, host)
-            line["cpu_baseline"] = {"value": v, "unit": "verify-steps/s", "cores": int(cores), "kind": "oracle",
-                                    "sample": sample}
-            dx = binding.sgbv_verify_ex(sets[0].target_logits, sets[0].draft_logits, sets[0].draft_tokens,
-                                        sets[0].uniforms, cfg.temperature)
-            torch.cuda.synchronize()
-            sl = slice(None) if rows is None else slice(0, rows)
-            rep = compare(ref, dx.accept_len[sl].cpu().numpy(), dx.draft_idx[sl].cpu().numpy(),
-                          dx.tokens[sl].cpu().numpy(), dx.h[sl].cpu().numpy(), dx.resmass[sl].cpu().numpy(),
-                          dx.status[sl].cpu().numpy())
-            line["parity"] = rep.summary()
+            line["parity"], line["cpu_baseline"] = parity_report(wl, 12.0)
+        del wl
+        torch.cuda.empty_cache()
+        # the other configurations the metric is quoted on, measured the same way (one GPU, shorter)
+        if world == 1 and not args.no_per_config:
+            per = []
+            for name in PER_CONFIG:
+                if name == cfg.name:
+                    continue
+                c = workloads.get_config(name)
+                w = Workload(c, dev, rank)
+                c_steps = int(max(20, min(2000, 50.0 / max(0.02, c.logit_bytes() / 4.0e9))))
+                bl, _, _ = timed_blocks(w, c_steps, max(3, c_steps // 4), 1, min_seconds=0.5)
+                k_ms, k_n = kernel_pass(w, max(20, min(c_steps, 200)))
+                nb, c_be = block_facts(w)
+                c_ab = algorithmic_bytes(c, nb)
+                msb = sorted(bl)[len(bl) // 2]
+                entry = {"workload": describe(c), "value": c_steps / (msb * 1e-3), "ms_per_step": msb / c_steps,
+                         "steps": c_steps, "repeats": len(bl), "block_efficiency": c_be,
+                         "roofline": roofline_of(w, c_ab, k_ms, k_n)}
+                if not args.no_cpu_baseline:
+                    entry["parity"], _ = parity_report(w, 2.0)
+                per.append(entry)
+                del w
+                torch.cuda.empty_cache()
+            line["per_config"] = per
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

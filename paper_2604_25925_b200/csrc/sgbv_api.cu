@@ -315,7 +315,7 @@ int sgbv_set_option(const char *name, int value) {
         if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
         g_opt_path = value;
     } else if (!strcmp(name, "cluster")) {
-        if (value < 0 || value > 8) return SGBV_ERR_SHAPE;
+        if (value < 0 || value > 16) return SGBV_ERR_SHAPE;
         g_opt_cluster = value;
     } else if (!strcmp(name, "max_clusters")) {
         if (value < 0) return SGBV_ERR_SHAPE;

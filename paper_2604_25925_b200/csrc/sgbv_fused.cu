@@ -39,10 +39,13 @@ namespace {
 
 constexpr int kMaxWarps = 32;              // warps per CTA: 32 (64 registers each) or 16 (128 registers each)
 constexpr int kCell = kTile;               // 256 contiguous entries: the unit a warp works on
-constexpr int kCtaCells = 128;             // cells of a row per CTA: 512 tensor-memory columns / 16 per cell, x 4 lane quarters
-                                           // = 32,768 entries; a CTA of W warps gives each warp 128 / W cells
-constexpr int kTmemCols = 512;             // all of the SM's tensor memory (one CTA per SM)
-constexpr int kMaxCluster = 8;             // portable cluster size
+constexpr int kCtasPerSm = 1;              // CTAs that share an SM (1 or 2): two are in different phases of their rows
+                                           // most of the time, so that one's exponentials overlap the other's sums
+constexpr int kWarps = 32 / kCtasPerSm;    // warps per CTA
+constexpr int kCtaCells = 4 * kWarps;      // cells of a row per CTA (four per warp); 16 tensor-memory columns per cell in
+                                           // each of the 4 lane quarters: 128 cells = 32,768 entries per SM
+constexpr int kTmemCols = 512 / kCtasPerSm;  // this CTA's share of the SM's tensor memory
+constexpr int kMaxCluster = 8 * kCtasPerSm;  // CTAs per cluster (beyond 8 the size is not portable, which sm_100 allows)
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
 constexpr uint32_t kPollNs = 100u;                    // sleep between two tests of a barrier that is not ready
 static_assert(kTile == 256, "the fused path writes one partial sum per 256-element cell");
@@ -306,114 +309,131 @@ struct RowScalars {
     float c;      // c_i
 };
 
-// Second sweep over the warp's cells, read back from tensor memory, two vocabulary entries per
-// instruction (f32x2).  eq/ep are exponentials relative to the THREAD's maxima of the cell;
-// fmq[j] moves cell j's target units to the thread's row units, rt[j] is the ratio of the cell's draft and
-// target factors, so that fq = fmq[j] Fq and kt = KF rt[j].  Per cell:
-//   wpart = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
-//   dpart = sum max(kt ep - eq, 0)                             (c < 1 only)
-//   mpart = sum eq (c - t)^2 Q(t)                              (c < 1 only)
-// The output pointers address this warp's first cell; its cells are W apart.  fmp_stash: this thread's
-// draft factors of the cells in shared memory (cells apart by `stash_stride` floats), read only by a cell
-// whose target share underflows in a row with c < 1.
-template <int W, int KT, bool kAux>
-__device__ __forceinline__ void sweep_two(uint32_t taddr, const float (&fmq)[kCtaCells / W], const float (&rt)[kCtaCells / W],
-                                          const RowScalars &rs, int K, int lane, int ncw, const float *fmp_stash,
-                                          int stash_stride, float *wpart, float *dpart, float *mpart) {
-    constexpr int kCellsPerWarp = kCtaCells / W, kFWarps = W;
-    const float v1 = 1.0f - rs.c;
-    const float2 nv1 = splat(-v1);
-    // Horner coefficients of Q: (t+1) (1-c)^t, t = 1..K-2 (uniform over the row)
-    float2 coef[KT > 2 ? KT - 2 : 1];
-    if (kAux && KT > 2) {
-        float vj = 1.0f;
-#pragma unroll
-        for (int t = 1; t <= KT - 2; ++t) {
-            vj *= v1;
-            coef[t - 1] = splat((float)(t + 1) * vj);
-        }
-    }
-    float wsum[kCellsPerWarp];
-#pragma unroll
-    for (int j = 0; j < kCellsPerWarp; ++j) wsum[j] = 0.0f;
-#pragma unroll
-    for (int j = 0; j < kCellsPerWarp; ++j) {
-        if (j >= ncw) break;  // warp-uniform
-        float2 eq[4], ep[4];
-        tmem_ld_cell(taddr + 16u * (uint32_t)j, eq, ep);
-        // thread units -> row units
-        float scale_w = fmq[j] * rs.Fq, scale_d = scale_w;
-        float kt = rs.KF * rt[j];
-        tmem_wait_ld(eq, ep);
-        if (kAux) {
-            // A thread whose share of the target row underflows (or nearly so, which would overflow kt): its q
-            // is 0 in row units, its weights vanish, and max(c p - q, 0) = c p.  Without the extra sums nothing
-            // needs doing: an infinite or NaN kt gives a zero weight through the clamps below.
-            const bool tiny = !(scale_w > 1e-30f);
-            if (__any_sync(0xffffffffu, tiny)) {
-                if (tiny) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) eq[e] = splat(0.0f);
-                    kt = 1.0f;
-                    scale_w = 0.0f;
-                    scale_d = rs.kFp * fmp_stash[j * stash_stride];
-                }
-            }
-        }
-        const float2 nkt = splat(-kt);
-        float2 sw = splat(0.0f), sd = splat(0.0f), sm = splat(0.0f);
+// First sweep of one cell, first half: the lane's 8 target and 8 draft logits from the ring slot (entries past the
+// end of the row read as -inf), and their maxima.
+template <typename T>
+__device__ __forceinline__ void first_sweep_fetch(const unsigned char *slot, int lane, bool is_tail, int tail_valid,
+                                                  float2 (&eq)[4], float2 (&ep)[4], float &m1, float &m2) {
+    read_cell<T>(slot, lane, eq);
+    read_cell<T>(slot + kCell * (int)sizeof(T), lane, ep);
+    if (is_tail) {  // the row ends inside this cell
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const float2 q = eq[e];
-            const float2 diff = __ffma2_rn(nkt, ep[e], q);  // q - c p, thread units
-            const float2 pos = make_float2(fmaxf(diff.x, 0.0f), fmaxf(diff.y, 0.0f));
-            if (KT == 1) sw = __fadd2_rn(sw, pos);
-            if (KT == 1 && !kAux) continue;
-            // r = 1 - min{c p/q, 1}; q = 0 gives -inf or NaN before the clamp, 0 after it
-            const float2 t = __fmul2_rn(diff, make_float2(rcp(q.x), rcp(q.y)));
-            const float2 r = make_float2(fmaxf(t.x, 0.0f), fmaxf(t.y, 0.0f));
-            if (KT != 1) sw = __ffma2_rn(q, ipow2<KT>(r, K), sw);
-            if (kAux) {
-                sd = __fadd2_rn(sd, make_float2(fmaxf(-diff.x, 0.0f), fmaxf(-diff.y, 0.0f)));
-                float2 acc = splat(0.0f);
-                if (KT > 0) {
-                    if (KT >= 2) {
-                        acc = splat(1.0f);
-#pragma unroll
-                        for (int u = 0; u < KT - 2; ++u) acc = __ffma2_rn(acc, r, coef[u]);
-                    }
-                } else if (K >= 2) {
-                    acc = splat(1.0f);
-                    float vj = 1.0f;
-                    for (int u = 1; u <= K - 2; ++u) {
-                        vj *= v1;
-                        acc = __ffma2_rn(acc, r, splat((float)(u + 1) * vj));
-                    }
-                }
-                const float2 ct = __fadd2_rn(r, nv1);  // c - t with t = 1 - r
-                sm = __ffma2_rn(__fmul2_rn(q, __fmul2_rn(ct, ct)), acc, sm);
-            }
-        }
-        wsum[j] = (sw.x + sw.y) * scale_w;
-        if (kAux) {
-            // the two extra sums of the cell leave right away (they are rare: rows with c < 1)
-            float aux[2] = {(sd.x + sd.y) * scale_d, (sm.x + sm.y) * scale_w};
-            warp_sum_multi<2>(aux, lane);
-            if ((lane & 15) == 0) ((lane & 16) ? mpart : dpart)[j * kFWarps] = aux[0];
+            if (cell_offset<T>(lane, 2 * e) >= tail_valid) eq[e].x = ep[e].x = -INFINITY;
+            if (cell_offset<T>(lane, 2 * e + 1) >= tail_valid) eq[e].y = ep[e].y = -INFINITY;
         }
     }
-    warp_sum_multi<kCellsPerWarp>(wsum, lane);
-    // the lane that owns value number idx (and has the low lane bits clear) stores it
-    const int idx = owner_index<kCellsPerWarp>(lane);
-    constexpr int kOwnerMask = 32 / kCellsPerWarp - 1;  // lanes that hold the same total
-    if ((lane & kOwnerMask) == 0 && idx < ncw) wpart[idx * kFWarps] = wsum[0];
+    m1 = m2 = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        m1 = max3(m1, eq[e].x, eq[e].y);
+        m2 = max3(m2, ep[e].x, ep[e].y);
+    }
+}
+// Second half: exponentials relative to the thread's own maxima of the cell (0 if it saw only -inf; the maximum
+// itself maps to exactly 1, so point-mass rows stay exact) into tensor memory, and their sums.
+__device__ __forceinline__ void first_sweep_store(uint32_t taddr_cell, float scale, float2 (&eq)[4], float2 (&ep)[4], float m1,
+                                                  float m2, float &s1, float &s2) {
+    const float bq = (m1 > -INFINITY) ? m1 : 0.0f;
+    const float bp = (m2 > -INFINITY) ? m2 : 0.0f;
+    const float2 nbq = splat(-bq), nbp = splat(-bp), sc2 = splat(scale);
+    float2 sq2 = splat(0.0f), sp2 = splat(0.0f);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 aq = __fmul2_rn(__fadd2_rn(eq[e], nbq), sc2);
+        const float2 ap = __fmul2_rn(__fadd2_rn(ep[e], nbp), sc2);
+        eq[e] = make_float2(ex2(aq.x), ex2(aq.y));
+        ep[e] = make_float2(ex2(ap.x), ex2(ap.y));
+        sq2 = __fadd2_rn(sq2, eq[e]);
+        sp2 = __fadd2_rn(sp2, ep[e]);
+    }
+    tmem_st_cell(taddr_cell, eq, ep);
+    s1 = sq2.x + sq2.y;
+    s2 = sp2.x + sp2.y;
+}
+
+// Second sweep of one cell, read back from tensor memory, two vocabulary entries per instruction (f32x2).
+// eq/ep are exponentials relative to the THREAD's maxima of the cell; fmq moves the cell's target units to the
+// thread's row units, rt is the ratio of the cell's draft and target factors, so that fq = fmq Fq and
+// kt = KF rt.  Returns in row-max units
+//   w  = sum eq (1 - min{kt ep/eq, 1})^K                    (Eq. 4's weights, Eq. 2's sum)
+//   sd = sum max(kt ep - eq, 0)                             (c < 1 only)
+//   sm = sum eq (c - t)^2 Q(t)                              (c < 1 only)
+// coef: Horner coefficients of Q, (t+1) (1-c)^t, t = 1..K-2.  fmp_stash: this thread's draft factor of the cell
+// in shared memory, read only when its target share underflows in a row with c < 1.
+template <int KT, bool kAux>
+__device__ __forceinline__ void second_sweep_cell(uint32_t taddr_cell, float fmq, float rt, const RowScalars &rs, int K,
+                                                  const float2 *coef, const float *fmp_stash, float &w, float &sd_out,
+                                                  float &sm_out) {
+    float2 eq[4], ep[4];
+    tmem_ld_cell(taddr_cell, eq, ep);
+    // thread units -> row units
+    float scale_w = fmq * rs.Fq, scale_d = scale_w;
+    float kt = rs.KF * rt;
+    const float v1 = 1.0f - rs.c;
+    const float2 nv1 = splat(-v1);
+    tmem_wait_ld(eq, ep);
+    if (kAux) {
+        // A thread whose share of the target row underflows (or nearly so, which would overflow kt): its q
+        // is 0 in row units, its weights vanish, and max(c p - q, 0) = c p.  Without the extra sums nothing
+        // needs doing: an infinite or NaN kt gives a zero weight through the clamps below.
+        const bool tiny = !(scale_w > 1e-30f);
+        if (__any_sync(0xffffffffu, tiny)) {
+            if (tiny) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) eq[e] = splat(0.0f);
+                kt = 1.0f;
+                scale_w = 0.0f;
+                scale_d = rs.kFp * *fmp_stash;
+            }
+        }
+    }
+    const float2 nkt = splat(-kt);
+    float2 sw = splat(0.0f), sd = splat(0.0f), sm = splat(0.0f);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float2 q = eq[e];
+        const float2 diff = __ffma2_rn(nkt, ep[e], q);  // q - c p, thread units
+        const float2 pos = make_float2(fmaxf(diff.x, 0.0f), fmaxf(diff.y, 0.0f));
+        if (KT == 1) sw = __fadd2_rn(sw, pos);
+        if (KT == 1 && !kAux) continue;
+        // r = 1 - min{c p/q, 1}; q = 0 gives -inf or NaN before the clamp, 0 after it
+        const float2 t = __fmul2_rn(diff, make_float2(rcp(q.x), rcp(q.y)));
+        const float2 r = make_float2(fmaxf(t.x, 0.0f), fmaxf(t.y, 0.0f));
+        if (KT != 1) sw = __ffma2_rn(q, ipow2<KT>(r, K), sw);
+        if (kAux) {
+            sd = __fadd2_rn(sd, make_float2(fmaxf(-diff.x, 0.0f), fmaxf(-diff.y, 0.0f)));
+            float2 acc = splat(0.0f);
+            if (KT > 0) {
+                if (KT >= 2) {
+                    acc = splat(1.0f);
+#pragma unroll
+                    for (int u = 0; u < KT - 2; ++u) acc = __ffma2_rn(acc, r, coef[u]);
+                }
+            } else if (K >= 2) {
+                acc = splat(1.0f);
+                float vj = 1.0f;
+                for (int u = 1; u <= K - 2; ++u) {
+                    vj *= v1;
+                    acc = __ffma2_rn(acc, r, splat((float)(u + 1) * vj));
+                }
+            }
+            const float2 ct = __fadd2_rn(r, nv1);  // c - t with t = 1 - r
+            sm = __ffma2_rn(__fmul2_rn(q, __fmul2_rn(ct, ct)), acc, sm);
+        }
+    }
+    w = (sw.x + sw.y) * scale_w;
+    if (kAux) {
+        sd_out = (sd.x + sd.y) * scale_d;
+        sm_out = (sm.x + sm.y) * scale_w;
+    }
 }
 
 // W warps per CTA; NS ring slots per warp (the cells per warp and row, kCtaCells / W, are a multiple of it, so
 // that cell j of a row always sits in slot j % NS); KT: the number of drafts K when it has a specialised
 // second sweep (1, 2, 3, 4, 8), else 0 (any K, loops).
 template <typename T, bool kRow, int W, int NS, int KT>
-__global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParams p) {
+__global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const FusedParams p) {
     constexpr int kFWarps = W, kFThreads = W * 32, kCellsPerWarp = kCtaCells / W;
     static_assert(kCellsPerWarp % NS == 0, "cell j of a row must always land in slot j % NS");
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -508,115 +528,139 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                    (PROW) + (size_t)(JJ) * kStrideBytes, bytes_, full_u32 + 8u * (uint32_t)(SLOT), is_lane0, kHalfBytes); \
         pending |= 1u << (SLOT);                                                                                       \
     } while (0)
+    // First sweep of cell J of the row whose cells start at (QROW, PROW); the slot is refilled from the same row
+    // or, past this warp's last cell, from the row that follows (QNXT, PNXT; only if MORE).
+#define SGBV_FIRST_SWEEP_CELL(J, QROW, PROW, QNXT, PNXT, MORE)                                                          \
+    do {                                                                                                               \
+        const int slot_ = (J) % NS; /* (a constant once the loop is unrolled) */                                       \
+        if (pending & (1u << slot_)) {                                                                                 \
+            mbar_wait(full_u32 + 8u * slot_, (phases >> slot_) & 1u, timed_out);                                       \
+            phases ^= 1u << slot_;                                                                                     \
+            pending ^= 1u << slot_;                                                                                    \
+        }                                                                                                              \
+        float2 eq_[4], ep_[4];                                                                                         \
+        first_sweep_fetch<T>(ring + slot_ * kSlotBytes, lane, (J) == tail_j, tail_valid, eq_, ep_, mq[J], mp[J]);      \
+        /* every lane holds its share of the slot in registers now: refill it */                                       \
+        __syncwarp();                                                                                                  \
+        if ((J) + NS < ncw) {                                                                                          \
+            if (!timed_out) SGBV_ISSUE(QROW, PROW, (J) + NS, slot_);                                                   \
+        } else if (MORE) {                                                                                             \
+            SGBV_ISSUE(QNXT, PNXT, slot_, slot_);                                                                      \
+        }                                                                                                              \
+        first_sweep_store(taddr + 16u * (uint32_t)(J), s.scale, eq_, ep_, mq[J], mp[J], sq[J], sp[J]);                 \
+    } while (0)
 
-    int bk = row_mode ? cid / s.gamma : cid;
-    int i = row_mode ? cid % s.gamma : 0;
-    const unsigned char *q_cur = zq_warp + ((size_t)bk * (s.gamma + 1) + i) * row_bytes;  // this warp's first cell of the row
-    const unsigned char *p_cur = zp_warp + ((size_t)bk * s.gamma + i) * row_bytes;
+    // rows of the walk: A = the row whose second sweep runs, B = the one after it, whose first sweep runs in the
+    // same loop, D = the one after B, whose cells are requested meanwhile
+    int bk_a = 0, i_a = 0;  // (set when B becomes A)
+    int bk_b = row_mode ? cid / s.gamma : cid;
+    int i_b = row_mode ? cid % s.gamma : 0;
+    const unsigned char *q_b = zq_warp + ((size_t)bk_b * (s.gamma + 1) + i_b) * row_bytes;  // this warp's first cell of row B
+    const unsigned char *p_b = zp_warp + ((size_t)bk_b * s.gamma + i_b) * row_bytes;
     if (nrows > 0) {
 #pragma unroll
         for (int k = 0; k < NS; ++k)
-            if (k < ncw) SGBV_ISSUE(q_cur, p_cur, k, k);
+            if (k < ncw) SGBV_ISSUE(q_b, p_b, k, k);
     }
 
-    // The last warp of this CTA combines the partials, carries c_i and fetches the token logits one row
-    // ahead (every lane the same words): tok_next is the token of the next row of the walk.
+    // The last warp of this CTA combines the partials, carries c_i and fetches the token logits of a row while its
+    // first sweep runs (every lane the same words).
     const bool combiner = warp == kFWarps - 1;
-    int tok_next = 0;
-    if (combiner && nrows > 0) tok_next = p.tok[(size_t)bk * s.gamma + i];
-    double c_carry = 1.0;  // chain walk: c of the row at hand (the first row of the walk starts a chain)
+    double c_carry = 1.0;  // chain walk: c of the row whose exchange comes next (the first row of the walk starts a chain)
 
-    for (int n = 0; n < nrows; ++n) {
-        const size_t r = (size_t)bk * s.gamma + i;
-        const int par = n & 1;
-        const uint32_t xph = (uint32_t)(n >> 1) & 1u;
+    float fmq[kCellsPerWarp], rt[kCellsPerWarp];  // row A: what the second sweep needs of every cell
+    RowScalars rs;                                 // row A
+    rs.Fq = rs.KF = rs.kFp = 0.0f;
+    rs.c = 1.0f;
+#pragma unroll
+    for (int j = 0; j < kCellsPerWarp; ++j) fmq[j] = rt[j] = 0.0f;
+
+    // n = -1: only the first sweep of row 0; n = nrows - 1: only the second sweep of the last row
+    for (int n = -1; n < nrows; ++n) {
+        const bool has_a = n >= 0, has_b = n + 1 < nrows;
+        // row D, the one after B
+        int bk_d = bk_b + step_bk, i_d = i_b + step_i;
+        if (i_d >= s.gamma) {
+            i_d -= s.gamma;
+            bk_d += wrap_bk;
+        }
+        const bool more = n + 2 < nrows && !timed_out;
+        const unsigned char *q_d = zq_warp + ((size_t)bk_d * (s.gamma + 1) + i_d) * row_bytes;
+        const unsigned char *p_d = zp_warp + ((size_t)bk_d * s.gamma + i_d) * row_bytes;
+        const size_t r_a = (size_t)bk_a * s.gamma + i_a, r_b = (size_t)bk_b * s.gamma + i_b;
+
+        // ---- combining warp: the logits of row B's draft token ------------------------------------------
+        float zq_tok = 0.0f, zp_tok = 0.0f;
+        const int par = (n + 1) & 1;  // of row B's exchange
+        const uint32_t xph = (uint32_t)((n + 1) >> 1) & 1u;
         const uint32_t xbar = xbar_u32 + 8u * (uint32_t)par;
-        // the next row of the walk (its cells are requested while this row is worked on)
-        int bk_n = bk + step_bk, i_n = i + step_i;
-        if (i_n >= s.gamma) {
-            i_n -= s.gamma;
-            bk_n += wrap_bk;
-        }
-        const bool more = n + 1 < nrows && !timed_out;
-        const unsigned char *q_nxt = zq_warp + ((size_t)bk_n * (s.gamma + 1) + i_n) * row_bytes;
-        const unsigned char *p_nxt = zp_warp + ((size_t)bk_n * s.gamma + i_n) * row_bytes;
-
-        // ---- combining warp: the logits of this row's draft token, and the next row's token --------
-        float zq_tok = 0.0f, zp_tok = 0.0f;  // logits of this row's draft token
-        if (combiner) {
-            if (C > 1 && lane == 0) mbar_expect_tx(xbar, xbytes);  // this row's partials of the cluster's CTAs
-            int t = tok_next;
+        if (combiner && has_b) {
+            if (C > 1 && lane == 0) mbar_expect_tx(xbar, xbytes);  // row B's partials of the cluster's CTAs
+            int t = p.tok[r_b];
             if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
-            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk * (s.gamma + 1) + i) * s.V, t);
-            zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + ((size_t)bk * s.gamma + i) * s.V, t);
-            if (n + 1 < nrows) tok_next = p.tok[(size_t)bk_n * s.gamma + i_n];
+            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk_b * (s.gamma + 1) + i_b) * s.V, t);
+            zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + r_b * s.V, t);
         }
 
-        // ---- first sweep: ring -> exponentials in tensor memory, maximum and sum of every cell --------
-        float mq[kCellsPerWarp], mp[kCellsPerWarp], sq[kCellsPerWarp], sp[kCellsPerWarp];
+        // ---- second sweep of row A from tensor memory, cell by cell, each followed by the first sweep of the
+        //      same cell of row B into the columns just read: the exponentials of the one and the sums of the
+        //      other keep different pipes busy --------------------------------------------------------------
+        float mq[kCellsPerWarp], mp[kCellsPerWarp], sq[kCellsPerWarp], sp[kCellsPerWarp];  // row B
+        float wsum[kCellsPerWarp];                                                         // row A
 #pragma unroll
         for (int j = 0; j < kCellsPerWarp; ++j) {
             mq[j] = mp[j] = -INFINITY;
-            sq[j] = sp[j] = 0.0f;
+            sq[j] = sp[j] = wsum[j] = 0.0f;
         }
+        float *wp = p.ws.wpart + r_a * s.ntiles + first_cell;
+        if (has_a && rs.c < 1.0f) {  // the rare kind of row: two more sums per cell
+            float *dp = p.ws.dpart + r_a * s.ntiles + first_cell, *mpp = p.ws.mpart + r_a * s.ntiles + first_cell;
+            float2 coef[KT > 2 ? KT - 2 : 1];
+            if (KT > 2) {
+                float vj = 1.0f;
 #pragma unroll
-        for (int j = 0; j < kCellsPerWarp; ++j) {
-            if (j < ncw) {  // warp-uniform
-                const int slot = j % NS;  // (a constant once the loop is unrolled)
-                if (pending & (1u << slot)) {
-                    mbar_wait(full_u32 + 8u * slot, (phases >> slot) & 1u, timed_out);
-                    phases ^= 1u << slot;
-                    pending ^= 1u << slot;
+                for (int t = 1; t <= KT - 2; ++t) {
+                    vj *= 1.0f - rs.c;
+                    coef[t - 1] = splat((float)(t + 1) * vj);
                 }
-                float2 eq[4], ep[4];
-                read_cell<T>(ring + slot * kSlotBytes, lane, eq);
-                read_cell<T>(ring + slot * kSlotBytes + kHalfBytes, lane, ep);
-                if (j == tail_j) {  // the row ends inside this cell
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (cell_offset<T>(lane, 2 * e) >= tail_valid) eq[e].x = ep[e].x = -INFINITY;
-                        if (cell_offset<T>(lane, 2 * e + 1) >= tail_valid) eq[e].y = ep[e].y = -INFINITY;
-                    }
-                }
-                float m1 = -INFINITY, m2 = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    m1 = max3(m1, eq[e].x, eq[e].y);
-                    m2 = max3(m2, ep[e].x, ep[e].y);
-                }
-                // every lane holds its share of the slot in registers now: refill it
-                __syncwarp();
-                if (j + NS < ncw) {
-                    if (!timed_out) SGBV_ISSUE(q_cur, p_cur, j + NS, slot);
-                } else if (more) {
-                    SGBV_ISSUE(q_nxt, p_nxt, slot, slot);
-                }
-                // reference points of this thread's exponentials: its own maxima of the cell (0 if it saw
-                // only -inf); the maximum itself maps to exactly 1, so point-mass rows stay exact
-                const float bq = (m1 > -INFINITY) ? m1 : 0.0f;
-                const float bp = (m2 > -INFINITY) ? m2 : 0.0f;
-                const float2 nbq = splat(-bq), nbp = splat(-bp), sc2 = splat(s.scale);
-                float2 sq2 = splat(0.0f), sp2 = splat(0.0f);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 aq = __fmul2_rn(__fadd2_rn(eq[e], nbq), sc2);
-                    const float2 ap = __fmul2_rn(__fadd2_rn(ep[e], nbp), sc2);
-                    eq[e] = make_float2(ex2(aq.x), ex2(aq.y));
-                    ep[e] = make_float2(ex2(ap.x), ex2(ap.y));
-                    sq2 = __fadd2_rn(sq2, eq[e]);
-                    sp2 = __fadd2_rn(sp2, ep[e]);
-                }
-                tmem_st_cell(taddr + 16u * (uint32_t)j, eq, ep);
-                mq[j] = m1;
-                mp[j] = m2;
-                sq[j] = sq2.x + sq2.y;
-                sp[j] = sp2.x + sp2.y;
             }
+#pragma unroll
+            for (int j = 0; j < kCellsPerWarp; ++j) {
+                if (j < ncw) {  // warp-uniform
+                    float aux[2];
+                    second_sweep_cell<KT, true>(taddr + 16u * (uint32_t)j, fmq[j], rt[j], rs, s.K, coef,
+                                                fmp_stash + j * kFThreads, wsum[j], aux[0], aux[1]);
+                    warp_sum_multi<2>(aux, lane);  // the two extra sums of the cell leave right away
+                    if ((lane & 15) == 0) ((lane & 16) ? mpp : dp)[j * kFWarps] = aux[0];
+                    if (has_b) SGBV_FIRST_SWEEP_CELL(j, q_b, p_b, q_d, p_d, more);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kCellsPerWarp; ++j) {
+                if (j < ncw) {  // warp-uniform
+                    float unused0, unused1;
+                    if (has_a)
+                        second_sweep_cell<KT, false>(taddr + 16u * (uint32_t)j, fmq[j], rt[j], rs, s.K, nullptr, nullptr, wsum[j],
+                                                     unused0, unused1);
+                    if (has_b) SGBV_FIRST_SWEEP_CELL(j, q_b, p_b, q_d, p_d, more);
+                }
+            }
+        }
+        // row A's cell sums: summed over the warp now, stored after the exchange below (a store that is still
+        // under way would hold up the memory fence of the exchange)
+        const int idx = owner_index<kCellsPerWarp>(lane);  // the lane that owns value number idx stores it
+        constexpr int kOwnerMask = 32 / kCellsPerWarp - 1;  // lanes that hold the same total
+        const bool store_w = has_a && (lane & kOwnerMask) == 0 && idx < ncw;
+        if (has_a) warp_sum_multi<kCellsPerWarp>(wsum, lane);
+        if (!has_b) {
+            if (store_w) wp[idx * kFWarps] = wsum[0];
+            break;
         }
         timed_out = __any_sync(0xffffffffu, timed_out != 0);  // the warp gives up as one
         tmem_wait_st();
 
-        // ---- this thread's partial of the row: cell sums moved to its maximum over the cells; what the
+        // ---- this thread's partial of row B: cell sums moved to its maximum over the cells; what the
         //      second sweep will need of every cell: fmq[j] = cell's target units -> thread's row units,
         //      rt[j] = ratio of the cell's draft and target factors ------------------------------------
         float mqt = mq[0], mpt = mp[0];
@@ -628,7 +672,6 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
         const bool has_q = mqt > -INFINITY, has_p = mpt > -INFINITY;
         const float bqt = has_q ? mqt : 0.0f, bpt = has_p ? mpt : 0.0f;
         float sqt = 0.0f, spt = 0.0f;
-        float fmq[kCellsPerWarp], rt[kCellsPerWarp];
 #pragma unroll
         for (int j = 0; j < kCellsPerWarp; ++j) {
             fmq[j] = rt[j] = 0.0f;
@@ -678,26 +721,28 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                 Zq = warp_sum(cv.x > -INFINITY ? cv.y * ex2((cv.x - rq_row) * s.scale) : 0.0f);
                 Zp = warp_sum(cv.z > -INFINITY ? cv.w * ex2((cv.z - rp_row) * s.scale) : 0.0f);
             }
-            // the ratio p_i(tok_i)/q_i(tok_i) of this row
-            const double ratio = exp2_short(((double)zp_tok - (double)rp_row) * (double)s.scale -
-                                            ((double)zq_tok - (double)rq_row) * (double)s.scale) *
-                                 (double)(Zq / Zp);
+            // The ratio p_i(tok_i)/q_i(tok_i) of this row: a chain of float64 operations.  In the chain walk only the
+            // NEXT row needs it, so it is worked out after the other warps have been released.
+#define SGBV_RATIO()                                                                                                     \
+    (exp2_short(((double)zp_tok - (double)rp_row) * (double)s.scale - ((double)zq_tok - (double)rq_row) * (double)s.scale) * \
+     (double)(Zq / Zp))
             double cd;
             if (row_mode) {
+                const double ratio = SGBV_RATIO();
                 // Publish this row's ratio for the clusters that walk the later rows of this chain.  The
                 // word itself says "ready": it is preset to a NaN pattern, and a ratio is never stored as
                 // NaN (a row that produces one is flagged invalid anyway).
-                if (lane == 0 && rank == 0 && i + 1 < s.gamma && !(p.withhold && i == 0))
-                    *reinterpret_cast<volatile double *>(p.ws.ratio + r) = (ratio != ratio) ? 0.0 : ratio;
+                if (lane == 0 && rank == 0 && i_b + 1 < s.gamma && !(p.withhold && i_b == 0))
+                    *reinterpret_cast<volatile double *>(p.ws.ratio + r_b) = (ratio != ratio) ? 0.0 : ratio;
                 // c_i = product of the published ratios of rows 0..i-1 of this chain (fixed order: a
                 // butterfly over the lanes).  Those rows are walked by other clusters at about the same
                 // time and publish right after their own statistics, which do not depend on c: no chain of
                 // waits forms.  Every lane polls one of them.  Bounded waits.
                 cd = 1.0;
-                const size_t r0 = (size_t)bk * s.gamma;
-                for (int j0 = 0; j0 < i; j0 += 32) {
+                const size_t r0 = (size_t)bk_b * s.gamma;
+                for (int j0 = 0; j0 < i_b; j0 += 32) {
                     double w = 1.0;
-                    if (j0 + lane < i) {
+                    if (j0 + lane < i_b) {
                         const volatile double *word = reinterpret_cast<const volatile double *>(p.ws.ratio + r0 + j0 + lane);
                         w = *word;
                         if (w != w && timed_out) w = 0.0;
@@ -718,35 +763,35 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
                 }
                 timed_out = __any_sync(0xffffffffu, timed_out != 0);
             } else {
-                // c is carried along the chain: c_{i+1} = c_i ratio, and 1 at the start of the next chain
-                cd = c_carry;
-                c_carry = (i + 1 < s.gamma) ? cd * ratio : 1.0;
+                cd = c_carry;  // carried along the chain
             }
             rowv = make_float4(rq_row, rp_row, (float)(cd * (double)(Zq / Zp)), (float)cd);
-            if (lane == 0) {
-                ctl->rs = rowv;
-                if (rank == 0) {
-                    // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
-                    // -inf only has Z = 0
-                    const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
-                                     !(bq_row < INFINITY) || !(bp_row < INFINITY);
-                    RowInfo ri;
-                    ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
-                    ri.pad_ = 0;
-                    ri.Zq = (double)Zq;
-                    ri.Zp = (double)Zp;
-                    ri.mq = bq_row;
-                    ri.mp = bp_row;
-                    ri.kappa = rowv.z;
-                    ri.c = rowv.w;
-                    p.ws.rows[r] = ri;
-                }
-            }
+            if (lane == 0) ctl->rs = rowv;
             __threadfence_block();
             bar_arrive(2, kFThreads);
+            // off the critical path: c of the next row of the chain walk (c_{i+1} = c_i ratio, and 1 at the start of
+            // the next chain), and the row's record for the finishing kernel
+            if (!row_mode) c_carry = (i_b + 1 < s.gamma) ? cd * SGBV_RATIO() : 1.0;
+            if (lane == 0 && rank == 0) {
+                // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
+                // -inf only has Z = 0
+                const bool bad = !(Zq > 0.0f) || !(Zp > 0.0f) || !(Zq < INFINITY) || !(Zp < INFINITY) ||
+                                 !(bq_row < INFINITY) || !(bp_row < INFINITY);
+                RowInfo ri;
+                ri.flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
+                ri.pad_ = 0;
+                ri.Zq = (double)Zq;
+                ri.Zp = (double)Zp;
+                ri.mq = bq_row;
+                ri.mp = bp_row;
+                ri.kappa = rowv.z;
+                ri.c = rowv.w;
+                p.ws.rows[r_b] = ri;
+            }
+#undef SGBV_RATIO
         }
-        // this thread's row units -> row-max units
-        RowScalars rs;
+        if (store_w) wp[idx * kFWarps] = wsum[0];
+        // this thread's row units -> row-max units; row B becomes row A
         const float Fp = has_p ? ex2((bpt - rowv.y) * s.scale) : 0.0f;
         rs.Fq = has_q ? ex2((bqt - rowv.x) * s.scale) : 0.0f;
         // equal factors (identical rows above all) must give kappa itself: p = q everywhere then leaves an
@@ -754,20 +799,12 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
         rs.KF = (Fp == rs.Fq) ? rowv.z : rowv.z * Fp * rcp(rs.Fq);
         rs.kFp = rowv.z * Fp;
         rs.c = rowv.w;
-
-        // ---- second sweep from tensor memory ----------------------------------------------------------
-        float *wp = p.ws.wpart + r * s.ntiles + first_cell, *dp = p.ws.dpart + r * s.ntiles + first_cell,
-              *mpp = p.ws.mpart + r * s.ntiles + first_cell;
-        if (rs.c < 1.0f)
-            sweep_two<W, KT, true>(taddr, fmq, rt, rs, s.K, lane, ncw, fmp_stash, kFThreads, wp, dp, mpp);
-        else
-            sweep_two<W, KT, false>(taddr, fmq, rt, rs, s.K, lane, ncw, fmp_stash, kFThreads, wp, dp, mpp);
-
-        // one step of the walk
-        bk = bk_n;
-        i = i_n;
-        q_cur = q_nxt;
-        p_cur = p_nxt;
+        bk_a = bk_b;
+        i_a = i_b;
+        bk_b = bk_d;
+        i_b = i_d;
+        q_b = q_d;
+        p_b = p_d;
     }
     // a warp that gave up may still have copies under way: they must land before the shared memory goes
     if (timed_out) {
@@ -783,6 +820,7 @@ __global__ void __launch_bounds__(W * 32, 1) fused_chain_kernel(const FusedParam
     __syncthreads();  // every warp of this CTA is done with the tensor memory
     if (warp == 0) tmem_dealloc(ctl->tmem_base, kTmemCols);
 #undef SGBV_ISSUE
+#undef SGBV_FIRST_SWEEP_CELL
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -796,11 +834,11 @@ int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
 int g_opt_poll_us = 0;     // 0 = about a second
 int g_opt_withhold = 0;
 
-constexpr int kSmemPerCta = 227 * 1024;    // largest dynamic shared memory of one CTA
+constexpr int kSmemPerCta = (228 * 1024) / kCtasPerSm - 1024;  // largest dynamic shared memory of one CTA
 constexpr int kDevices = 64;
 std::mutex g_plan_mu;      // guards the options and the per-device caches below
 
-constexpr int kWarps = 32;  // warps per CTA
+constexpr int kCtaSlots = 148 * kCtasPerSm;  // CTAs the device holds
 // ring slots per warp: half a row's cells for float32 (128 KB of copies under way per SM), all of them for bfloat16
 template <typename T>
 constexpr int slots_for() { return sizeof(T) == 4 ? 2 : 4; }
@@ -816,6 +854,8 @@ cudaError_t prepare(int dev) {
     if (!attr_done[dev]) {
         cudaError_t e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow, kWarps, slots_for<T>(), KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(fused_chain_kernel<T, kRow, kWarps, slots_for<T>(), KT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
         attr_done[dev] = true;
     }
     return cudaSuccess;
@@ -830,7 +870,7 @@ int resident_clusters(int dev, int C) {
         cudaLaunchConfig_t cfg = {};
         cfg.blockDim = dim3(kWarps * 32);
         cfg.dynamicSmemBytes = smem_bytes<T>();
-        cfg.gridDim = dim3(C * (148 / C));
+        cfg.gridDim = dim3(C * (kCtaSlots / C));
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = C;

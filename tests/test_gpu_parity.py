@@ -223,8 +223,8 @@ def _slice_fits(V, cluster):
 
 
 @pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 3),
-                                    ("cluster", 4), ("cluster", 5), ("cluster", 8), ("max_clusters", 3), ("walk", 1),
-                                    ("walk", 2)])
+                                    ("cluster", 4), ("cluster", 5), ("cluster", 7), ("cluster", 8),
+                                    ("max_clusters", 3), ("walk", 1), ("walk", 2)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / walk /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
