@@ -695,8 +695,10 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
         // stores that complete on the receiver's mbarrier; it alone polls that barrier), works out the row's
         // scalars and hands them to the others.  The others wait on hardware barriers, which costs them no
         // issue slots: barrier 1 = "all partials are in", barrier 2 = "the row's scalars are in".
+        // (a store to shared memory followed by an arrival on the barrier is the producer half of the hardware
+        // barrier's producer/consumer pattern: the consumer that syncs on it sees the store)
         if (lane == 0) ctl->wslots[warp] = make_float4(bqw, sqt, bpw, spt);
-        __threadfence_block();
+        __syncwarp();
         float4 rowv;  // rq, rp, kappa, c
         if (!combiner) {
             bar_arrive(1, kFThreads);
@@ -767,7 +769,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
             }
             rowv = make_float4(rq_row, rp_row, (float)(cd * (double)(Zq / Zp)), (float)cd);
             if (lane == 0) ctl->rs = rowv;
-            __threadfence_block();
+            __syncwarp();
             bar_arrive(2, kFThreads);
             // off the critical path: c of the next row of the chain walk (c_{i+1} = c_i ratio, and 1 at the start of
             // the next chain), and the row's record for the finishing kernel
