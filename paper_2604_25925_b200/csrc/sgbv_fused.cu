@@ -613,7 +613,32 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
             sq[j] = sp[j] = wsum[j] = 0.0f;
         }
         float *wp = p.ws.wpart + r_a * s.ntiles + first_cell;
-        if (has_a && rs.c < 1.0f) {  // the rare kind of row: two more sums per cell
+        // The common case by far has nothing to decide per cell: a warp with all its cells, rows before and after,
+        // no partial cell, the plain kind of row.  Its loop body is straight-line code.
+        const bool steady = ncw == kCellsPerWarp && has_a && more && tail_j < 0 && !(rs.c < 1.0f);
+        if (steady) {
+#pragma unroll
+            for (int j = 0; j < kCellsPerWarp; ++j) {
+                float unused0, unused1;
+                second_sweep_cell<KT, false>(taddr + 16u * (uint32_t)j, fmq[j], rt[j], rs, s.K, nullptr, nullptr, wsum[j],
+                                             unused0, unused1);
+                const int slot = j % NS;  // (a constant once the loop is unrolled)
+                mbar_wait(full_u32 + 8u * slot, (phases >> slot) & 1u, timed_out);
+                phases ^= 1u << slot;
+                float2 eq_[4], ep_[4];
+                first_sweep_fetch<T>(ring + slot * kSlotBytes, lane, false, tail_valid, eq_, ep_, mq[j], mp[j]);
+                __syncwarp();  // every lane holds its share of the slot in registers now: refill it
+                if (j + NS < kCellsPerWarp)
+                    issue_cell(ring_u32 + (uint32_t)(slot * kSlotBytes), q_b + (size_t)(j + NS) * kStrideBytes,
+                               p_b + (size_t)(j + NS) * kStrideBytes, kHalfBytes, full_u32 + 8u * (uint32_t)slot, is_lane0,
+                               kHalfBytes);
+                else
+                    issue_cell(ring_u32 + (uint32_t)(slot * kSlotBytes), q_d + (size_t)slot * kStrideBytes,
+                               p_d + (size_t)slot * kStrideBytes, kHalfBytes, full_u32 + 8u * (uint32_t)slot, is_lane0,
+                               kHalfBytes);
+                first_sweep_store(taddr + 16u * (uint32_t)j, s.scale, eq_, ep_, mq[j], mp[j], sq[j], sp[j]);
+            }
+        } else if (has_a && rs.c < 1.0f) {  // the rare kind of row: two more sums per cell
             float *dp = p.ws.dpart + r_a * s.ntiles + first_cell, *mpp = p.ws.mpart + r_a * s.ntiles + first_cell;
             float2 coef[KT > 2 ? KT - 2 : 1];
             if (KT > 2) {
