@@ -64,6 +64,14 @@ def _load():
         lib.sgbv_oracle_verify.argtypes = [fp, fp, ip, fp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                            ctypes.c_int, ctypes.c_double, ip, ip, ip, dp, dp, dp,
                                            dp, ip, dp, dp, ctypes.c_int]
+        lib.sgbv_oracle_modify.restype = ctypes.c_int
+        lib.sgbv_oracle_modify.argtypes = [fp, fp, dp, dp, fp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                           ctypes.c_double, ip, dp, dp, dp, dp, ip, dp]
+        lib.sgbv_oracle_kseq_rho.restype = ctypes.c_double
+        lib.sgbv_oracle_kseq_rho.argtypes = [dp, dp, ctypes.c_int, ctypes.c_int]
+        lib.sgbv_oracle_kseq_verify.restype = ctypes.c_int
+        lib.sgbv_oracle_kseq_verify.argtypes = [fp, fp, ip, fp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_double, ip, ip, dp, dp, ip, dp, dp]
         _lib = lib
     return _lib
 
@@ -182,3 +190,74 @@ def verify(zq, zp, tok, uniforms, temperature: float = 1.0, nthreads: int = 0) -
     if used < 0:
         raise ValueError("oracle: bad argument")
     return VerifyResult(tau, f, tokens, h, S, la, lb, status, ma, ms, used)
+
+
+@dataclass
+class ModifyResult:
+    token: np.ndarray     # [B] int32 token drawn from q_new
+    loga: np.ndarray      # [B] carried log q(s, token)
+    logb: np.ndarray      # [B] carried log p(s, token)
+    R: np.ndarray         # [B] normaliser over a: sum_x q(x|s)(1 - min{(b/a) p(x|s)/q(x|s), 1})^K
+    qnew: np.ndarray      # [B, V] the modified distribution (None unless asked for)
+    status: np.ndarray    # [B] int32 flags
+    margin: np.ndarray    # [B] distance of u to the nearer CDF edge of the drawn cell
+
+
+def modify(zq, zp, loga, logb, u, K: int, temperature: float = 1.0, want_qnew: bool = False) -> ModifyResult:
+    """One position of Algorithm 2 for every batch row. zq, zp [B,V]; loga, logb, u [B]."""
+    zq, zp, u = _f32(zq), _f32(zp), _f32(u)
+    loga, logb = _f64(loga), _f64(logb)
+    B, V = zq.shape
+    assert zp.shape == (B, V) and loga.shape == (B,) and logb.shape == (B,) and u.shape == (B,)
+    tok = np.empty(B, np.int32)
+    la, lb, R, mg = (np.empty(B, np.float64) for _ in range(4))
+    st = np.empty(B, np.int32)
+    qn = np.empty((B, V), np.float64) if want_qnew else None
+    rc = _load().sgbv_oracle_modify(_p(zq, ctypes.c_float), _p(zp, ctypes.c_float), _p(loga, ctypes.c_double),
+                                    _p(logb, ctypes.c_double), _p(u, ctypes.c_float), B, V, int(K),
+                                    float(temperature), _p(tok, ctypes.c_int32), _p(la, ctypes.c_double),
+                                    _p(lb, ctypes.c_double), _p(R, ctypes.c_double),
+                                    _p(qn, ctypes.c_double) if want_qnew else None, _p(st, ctypes.c_int32),
+                                    _p(mg, ctypes.c_double))
+    if rc < 0:
+        raise ValueError("oracle: bad argument")
+    return ModifyResult(tok, la, lb, R, qn, st, mg)
+
+
+def kseq_rho(q, p, n: int) -> float:
+    """K-SEQ's rho for n candidate drafts: the root of 1 - (1 - beta(rho))^n = rho beta(rho) in [1, n]."""
+    q, p = _f64(q), _f64(p)
+    return _load().sgbv_oracle_kseq_rho(_p(q, ctypes.c_double), _p(p, ctypes.c_double), q.shape[0], int(n))
+
+
+@dataclass
+class KseqResult:
+    tau: np.ndarray            # [B] accepted length
+    tokens: np.ndarray         # [B, gamma+1]
+    rho: np.ndarray            # [B, gamma] rho of every position reached (NaN elsewhere)
+    acc: np.ndarray            # [B, K, gamma] acceptance probability of every token tried (NaN elsewhere)
+    status: np.ndarray         # [B]
+    margin_accept: np.ndarray  # [B]
+    margin_sample: np.ndarray  # [B]
+
+
+def kseq_verify(zq, zp, tok, uniforms, temperature: float = 1.0) -> KseqResult:
+    """Position-wise K-SEQ verification (token-level speculative sampling at K = 1)."""
+    zq, zp, tok, uniforms = _f32(zq), _f32(zp), _i32(tok), _f32(uniforms)
+    B, K, g1, V = zq.shape
+    gamma = g1 - 1
+    assert zp.shape == (B, K, gamma, V) and tok.shape == (B, K, gamma) and uniforms.shape == (B, K * gamma + 1)
+    tau = np.empty(B, np.int32)
+    tokens = np.empty((B, gamma + 1), np.int32)
+    rho = np.empty((B, gamma), np.float64)
+    acc = np.empty((B, K, gamma), np.float64)
+    st = np.empty(B, np.int32)
+    ma, ms = np.empty(B, np.float64), np.empty(B, np.float64)
+    rc = _load().sgbv_oracle_kseq_verify(_p(zq, ctypes.c_float), _p(zp, ctypes.c_float), _p(tok, ctypes.c_int32),
+                                         _p(uniforms, ctypes.c_float), B, K, gamma, V, float(temperature),
+                                         _p(tau, ctypes.c_int32), _p(tokens, ctypes.c_int32),
+                                         _p(rho, ctypes.c_double), _p(acc, ctypes.c_double),
+                                         _p(st, ctypes.c_int32), _p(ma, ctypes.c_double), _p(ms, ctypes.c_double))
+    if rc < 0:
+        raise ValueError("oracle: bad argument")
+    return KseqResult(tau, tokens, rho, acc, st, ma, ms)

@@ -29,6 +29,9 @@
  *     if rounding leaves none, the last x with positive mass;
  *   - one temperature T > 0 divides the logits of both models.
  *
+ * Also here, with their own pins: one position of Algorithm 2 (sgbv_oracle_modify) and the comparison
+ * verifiers of Section 3, token-level speculative sampling and SpecTr's K-SEQ (sgbv_oracle_kseq_verify).
+ *
  * Pins (tests, CPU only): the K=1 case against an independent single-draft GBV; K=1,gamma=1
  * against token-level speculative sampling; exactness of the output law at K=1 by exhaustive
  * enumeration on tree models; the hand-derived two-token example (19/27); closed forms of S on
@@ -370,4 +373,212 @@ int sgbv_oracle_verify(const float *zq, const float *zp, const int32_t *tok, con
                    out_margin_sample ? out_margin_sample + b : NULL);
     }
     return used;
+}
+
+/* ============================================================================================== */
+/* Algorithm 2 (Distribution Modification), one position.                                          */
+/*                                                                                                 */
+/* After an iteration that stopped short (tau < L), the next L - tau - 1 tokens are drawn from    */
+/*   q_new(x) = q(s,x) (1 - min{p(s,x)/q(s,x), 1})^K / sum_x' q(s,x') (1 - min{p(s,x')/q(s,x'),1})^K */
+/* where s = (t^tau, y, x^{i-1}) is everything emitted so far and q(s,x) = a q(x|s), p(s,x) =      */
+/* b p(x|s) are JOINT probabilities, a = q(s), b = p(s) carried along as logarithms.  The common   */
+/* factor a cancels between numerator and denominator, so the sums are formed with (1, b/a) in     */
+/* place of (a, b): same distribution, and a long s cannot underflow it.                           */
+/*   zq, zp [B,V] logits of the position; loga, logb [B]; u [B] uniforms for the inverse CDF       */
+/*   out_token [B]; out_loga/out_logb [B] = carried logs with the drawn token appended;            */
+/*   out_R [B] = sum_x q(x|s)(1 - min{(b/a) p(x|s)/q(x|s), 1})^K; out_qnew [B,V] or NULL;          */
+/*   out_status [B]; out_margin [B] (distance of u to the nearer CDF edge of the drawn cell).      */
+/* Zero total mass: the token is drawn from q(.|s) itself (flagged), as for Eq. 4.                 */
+int sgbv_oracle_modify(const float *zq, const float *zp, const double *loga, const double *logb,
+                       const float *u, int B, int V, int K, double T, int32_t *out_token,
+                       double *out_loga, double *out_logb, double *out_R, double *out_qnew,
+                       int32_t *out_status, double *out_margin) {
+    if (B < 0 || V < 1 || K < 1 || !(T > 0.0) || !isfinite(T)) return -1;
+    for (int b = 0; b < B; ++b) {
+        const float *rq = zq + (size_t)b * V, *rp = zp + (size_t)b * V;
+        int status = 0, anyq = 0, anyp = 0;
+        for (int x = 0; x < V; ++x) {
+            if (isnan(rq[x]) || rq[x] == INFINITY || isnan(rp[x]) || rp[x] == INFINITY)
+                status |= ORACLE_STATUS_NONFINITE;
+            anyq |= isfinite(rq[x]);
+            anyp |= isfinite(rp[x]);
+        }
+        if (!anyq || !anyp) status |= ORACLE_STATUS_NONFINITE;
+        int32_t y = -1;
+        double R = NAN, la = NAN, lb = NAN, margin = 0.0;
+        if (status == 0) {
+            double *q = (double *)malloc((size_t)V * sizeof(double));
+            double *p = (double *)malloc((size_t)V * sizeof(double));
+            double *w = (double *)malloc((size_t)V * sizeof(double));
+            double lse_q = sgbv_oracle_softmax(rq, V, T, q);
+            double lse_p = sgbv_oracle_softmax(rp, V, T, p);
+            R = sgbv_oracle_resmass(q, p, V, 1.0, exp(logb[b] - loga[b]), K, w);
+            y = sgbv_oracle_sample(w, V, (double)u[b], &margin);
+            if (y < 0) {
+                status |= ORACLE_STATUS_DEGENERATE_RESIDUAL;
+                y = sgbv_oracle_sample(q, V, (double)u[b], &margin);
+                if (out_qnew) memcpy(out_qnew + (size_t)b * V, q, (size_t)V * sizeof(double));
+            } else if (out_qnew) {
+                for (int x = 0; x < V; ++x) out_qnew[(size_t)b * V + x] = w[x] / R;
+            }
+            la = loga[b] + ((double)rq[y] / T - lse_q);
+            lb = logb[b] + ((double)rp[y] / T - lse_p);
+            free(q); free(p); free(w);
+        } else if (out_qnew) {
+            for (int x = 0; x < V; ++x) out_qnew[(size_t)b * V + x] = NAN;
+        }
+        out_token[b] = y;
+        if (out_loga) out_loga[b] = la;
+        if (out_logb) out_logb[b] = lb;
+        if (out_R) out_R[b] = R;
+        if (out_status) out_status[b] = status;
+        if (out_margin) out_margin[b] = margin;
+    }
+    return 1;
+}
+
+/* ============================================================================================== */
+/* Comparison verifiers of Section 3: token-level speculative sampling (3.1) and SpecTr's K-SEQ   */
+/* (3.2), position by position.  K = 1 of K-SEQ is token-level speculative sampling (rho = 1).     */
+/*                                                                                                 */
+/* Per position i, with the drafts that still match the accepted prefix ("retained", n of them;    */
+/* they share the rows of that prefix, the rows of the first retained draft are read):             */
+/*   beta(rho) = sum_x min{p(x), q(x)/rho};  rho in [1, n] solves 1 - (1 - beta(rho))^n = rho beta(rho) */
+/*   (bisection; the left side minus the right is >= 0 at rho = 1 and <= 0 at rho = n);            */
+/*   the retained drafts are tried in order: draft k's token x is accepted if eta_{k,i} <          */
+/*   min{1, q(x)/(rho p(x))}; the first accepted token extends the prefix and the drafts with that */
+/*   token stay retained; if none is accepted, y is drawn from norm(q - rho min{p, q/rho}) =       */
+/*   norm(max{q - rho p, 0}) and the step ends; after L accepted positions y ~ q(.|x^L).           */
+/* Reading: n is the number of retained drafts at that position (the candidates that are actually  */
+/* i.i.d. draws from p(.|prefix)), n = K at the first position.                                    */
+/* Layouts as in sgbv_oracle_verify; uniforms[b, k*gamma + i] is eta of draft k at position i      */
+/* (0-based), the last entry draws y.  out_rho [B,gamma] (NaN where not reached); out_acc          */
+/* [B,K,gamma] acceptance probabilities of the tokens that were tried (NaN elsewhere).             */
+static double kseq_beta(const double *q, const double *p, int V, double rho) {
+    double s = 0.0;
+    for (int x = 0; x < V; ++x) {
+        double t = q[x] / rho;
+        s += p[x] < t ? p[x] : t;
+    }
+    return s;
+}
+
+double sgbv_oracle_kseq_rho(const double *q, const double *p, int V, int n) {
+    if (n <= 1) return 1.0;
+    double lo = 1.0, hi = (double)n;
+    for (int it = 0; it < 200 && hi - lo > 1e-15 * hi; ++it) {
+        double mid = 0.5 * (lo + hi);
+        double beta = kseq_beta(q, p, V, mid);
+        double f = sgbv_oracle_g(beta, n) - mid * beta;
+        if (f > 0.0) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+int sgbv_oracle_kseq_verify(const float *zq, const float *zp, const int32_t *tok, const float *uniforms,
+                            int B, int K, int gamma, int V, double T, int32_t *out_tau,
+                            int32_t *out_tokens, double *out_rho, double *out_acc, int32_t *out_status,
+                            double *out_margin_accept, double *out_margin_sample) {
+    if (B < 0 || K < 1 || gamma < 1 || V < 1 || !(T > 0.0) || !isfinite(T)) return -1;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int b = 0; b < B; ++b) {
+        const float *zq_b = zq + (size_t)b * K * (gamma + 1) * V, *zp_b = zp + (size_t)b * K * gamma * V;
+        const int32_t *tok_b = tok + (size_t)b * K * gamma;
+        const float *u = uniforms + (size_t)b * (K * gamma + 1);
+        double *q = (double *)malloc((size_t)V * sizeof(double));
+        double *p = (double *)malloc((size_t)V * sizeof(double));
+        double *w = (double *)malloc((size_t)V * sizeof(double));
+        int *kept = (int *)malloc((size_t)K * sizeof(int));
+        int status = 0;
+        for (int n = 0; n < K * gamma; ++n)
+            if (tok_b[n] < 0 || tok_b[n] >= V) status |= ORACLE_STATUS_TOKEN_RANGE;
+        for (int i = 0; i <= gamma; ++i) out_tokens[(size_t)b * (gamma + 1) + i] = -1;
+        for (int i = 0; i < gamma; ++i) out_rho[(size_t)b * gamma + i] = NAN;
+        for (int n = 0; n < K * gamma; ++n) out_acc[(size_t)b * K * gamma + n] = NAN;
+        int tau = 0;
+        int32_t y = -1;
+        double margin_a = INFINITY, margin_s = 0.0;
+        int nk = K;
+        for (int k = 0; k < K; ++k) kept[k] = k;
+        int stopped = 0;
+        for (int i = 0; i < gamma && status == 0 && !stopped; ++i) {
+            const float *rq = zq_b + ((size_t)kept[0] * (gamma + 1) + i) * V;
+            const float *rp = zp_b + ((size_t)kept[0] * gamma + i) * V;
+            int anyq = 0, anyp = 0;
+            for (int x = 0; x < V; ++x) {
+                if (isnan(rq[x]) || rq[x] == INFINITY || isnan(rp[x]) || rp[x] == INFINITY)
+                    status |= ORACLE_STATUS_NONFINITE;
+                anyq |= isfinite(rq[x]);
+                anyp |= isfinite(rp[x]);
+            }
+            if (!anyq || !anyp) status |= ORACLE_STATUS_NONFINITE;
+            if (status) break;
+            sgbv_oracle_softmax(rq, V, T, q);
+            sgbv_oracle_softmax(rp, V, T, p);
+            double rho = sgbv_oracle_kseq_rho(q, p, V, nk);
+            out_rho[(size_t)b * gamma + i] = rho;
+            int accepted = -1;
+            for (int j = 0; j < nk && accepted < 0; ++j) {
+                int k = kept[j];
+                int32_t x = tok_b[k * gamma + i];
+                double acc = (p[x] > 0.0) ? q[x] / (rho * p[x]) : 1.0;
+                if (acc > 1.0) acc = 1.0;
+                out_acc[((size_t)b * K + k) * gamma + i] = acc;
+                double eta = (double)u[k * gamma + i];
+                double d = fabs(eta - acc);
+                if (d < margin_a) margin_a = d;
+                if (eta < acc) accepted = k;
+            }
+            if (accepted >= 0) {
+                int32_t x = tok_b[accepted * gamma + i];
+                out_tokens[(size_t)b * (gamma + 1) + i] = x;
+                tau = i + 1;
+                int m = 0;
+                for (int j = 0; j < nk; ++j)
+                    if (tok_b[kept[j] * gamma + i] == x) kept[m++] = kept[j];
+                nk = m;
+            } else {
+                for (int x = 0; x < V; ++x) {
+                    double d = q[x] - rho * p[x];
+                    w[x] = d > 0.0 ? d : 0.0;
+                }
+                y = sgbv_oracle_sample(w, V, (double)u[K * gamma], &margin_s);
+                if (y < 0) {
+                    status |= ORACLE_STATUS_DEGENERATE_RESIDUAL;
+                    y = sgbv_oracle_sample(q, V, (double)u[K * gamma], &margin_s);
+                }
+                stopped = 1;
+            }
+        }
+        if (status == 0 || status == ORACLE_STATUS_DEGENERATE_RESIDUAL) {
+            if (!stopped) { /* every position accepted: bonus token from the target row after the block */
+                const float *rq = zq_b + ((size_t)kept[0] * (gamma + 1) + gamma) * V;
+                int any = 0, badrow = 0;
+                for (int x = 0; x < V; ++x) {
+                    badrow |= isnan(rq[x]) || rq[x] == INFINITY;
+                    any |= isfinite(rq[x]);
+                }
+                if (badrow || !any) {
+                    status |= ORACLE_STATUS_NONFINITE;
+                } else {
+                    sgbv_oracle_softmax(rq, V, T, q);
+                    y = sgbv_oracle_sample(q, V, (double)u[K * gamma], &margin_s);
+                }
+            }
+        }
+        if (status & (ORACLE_STATUS_NONFINITE | ORACLE_STATUS_TOKEN_RANGE)) {
+            tau = -1;
+            for (int i = 0; i <= gamma; ++i) out_tokens[(size_t)b * (gamma + 1) + i] = -1;
+        } else {
+            out_tokens[(size_t)b * (gamma + 1) + tau] = y;
+        }
+        out_tau[b] = tau;
+        if (out_status) out_status[b] = status;
+        if (out_margin_accept) out_margin_accept[b] = margin_a;
+        if (out_margin_sample) out_margin_sample[b] = margin_s;
+        free(q); free(p); free(w); free(kept);
+    }
+    return 1;
 }

@@ -115,15 +115,13 @@ def test_k1_equals_single_draft_gbv(seed):
 # modification of Algorithm 2 for the tokens after y.
 # --------------------------------------------------------------------------------------------
 def _modified_next(tm, seq, K):
-    """Algorithm 2: law of the token after `seq` when it lies in the modified region."""
+    """Algorithm 2: law of the token after `seq` when it lies in the modified region -- taken from the oracle's
+    own Algorithm 2 (sgbv_oracle_modify) with the carried joint log-probabilities of `seq`, so that the
+    enumeration below pins that function too."""
     a, b = tm.joint(seq)
-    q, p = tm.q(seq), tm.p(seq)
-    w = np.zeros(tm.V)
-    for x in range(tm.V):
-        qj, pj = a * q[x], b * p[x]
-        if qj > 0:
-            w[x] = qj * (1 - min(pj / qj, 1.0)) ** K
-    return w / w.sum() if w.sum() > 0 else q
+    res = oracle.modify(tm.zq[tuple(seq)][None], tm.zp[tuple(seq)][None], np.array([np.log(a)]),
+                        np.array([np.log(b)]), np.array([0.5], np.float32), K, tm.T, want_qnew=True)
+    return res.qnew[0]
 
 
 @pytest.mark.parametrize("V,g,seed", [(3, 2, 0), (3, 3, 1), (4, 2, 2), (2, 3, 3)])
