@@ -114,6 +114,33 @@ int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dt
                      int32_t *out_tokens, int32_t *out_status, void *stream);
 
 /*
+ * One position of the distribution modification that follows a verify step which stopped short
+ * (Algorithm 2; Theorem 4.2 needs it for the law of a whole decode).  With s = everything emitted so
+ * far in the modified region (the accepted block, the extra token, the tokens drawn here before),
+ * the next token comes from
+ *   q_new(x) = q(s,x) (1 - min{p(s,x)/q(s,x), 1})^K / sum_x' q(s,x') (1 - min{p(s,x')/q(s,x'), 1})^K
+ * with JOINT probabilities q(s,x) = q(s) q(x|s), p(s,x) = p(s) p(x|s): Eq. 4's weights with the ratio
+ * p(s)/q(s) carried in instead of built from a draft.  Per batch row the call draws that token by
+ * inverse CDF and appends it to the carried logs.  All pointers are device pointers.
+ *   target_logits [B,V], draft_logits [B,V]   logits of this position given s (dtype as in sgbv_verify_ex)
+ *   log_a, log_b  [B] float64                 log q(s), log p(s); 0 for an empty s
+ *   uniforms      [B] float32 in [0,1)        one per row, for the inverse CDF
+ *   K                                          the number of drafts of the decode (the exponent above)
+ *   out_token     [B] int32                   the drawn token, -1 if the row was flagged invalid
+ *   out_log_a, out_log_b [B] float64          log q(s,token), log p(s,token) (may alias log_a, log_b)
+ *   out_resmass   [B] float64 or NULL         sum_x q(x|s)(1 - min{(p(s)/q(s)) p(x|s)/q(x|s), 1})^K, the normaliser over q(s)
+ *   out_status    [B] int32 or NULL           SGBV_STATUS_* bits; zero total mass draws from q(.|s), flagged
+ *                                             DEGENERATE_RESIDUAL
+ *   workspace                                  >= sgbv_workspace_bytes(B, 1, 1, V, dtype) bytes, 256-byte aligned,
+ *                                              or NULL for the library's per-device buffer (see sgbv_verify)
+ * Errors as for sgbv_verify_ex.
+ */
+int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, const double *log_a,
+                const double *log_b, const float *uniforms, int B, int K, int V, float temperature,
+                int32_t *out_token, double *out_log_a, double *out_log_b, double *out_resmass,
+                int32_t *out_status, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Allocation-free form of sgbv_verify_ex (the paper has no counterpart: this entry point exists
  * for deployment, not for the method).
  *

@@ -26,7 +26,7 @@ DTYPE_BF16 = 1
 EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_verify_ex",
            "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_last_main_kernel", "sgbv_status_string",
            "sgbv_profile_begin",
-           "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option")
+           "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option", "sgbv_modify")
 
 _lib = None
 
@@ -65,6 +65,8 @@ def load() -> ctypes.CDLL:
         lib.sgbv_verify_static.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, vp]
         lib.sgbv_verify_host.restype = i32
         lib.sgbv_verify_host.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+        lib.sgbv_modify.restype = i32
+        lib.sgbv_modify.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.sgbv_last_launch_count.restype = i32
         lib.sgbv_last_launch_count.argtypes = []
         lib.sgbv_last_main_kernel.restype = ctypes.c_char_p
@@ -268,6 +270,44 @@ def sgbv_verify_host(target_logits, draft_logits, draft_tokens, uniforms, temper
             out.accept_len.data_ptr(), out.draft_idx.data_ptr(), out.tokens.data_ptr(),
             out.status.data_ptr() if out.status is not None else None,
             torch.cuda.current_stream(device).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+@dataclass
+class ModifyOutput:
+    token: torch.Tensor      # [B] int32
+    log_a: torch.Tensor      # [B] float64 log q(s, token)
+    log_b: torch.Tensor      # [B] float64 log p(s, token)
+    resmass: torch.Tensor    # [B] float64 normaliser over q(s)
+    status: torch.Tensor     # [B] int32
+
+
+def sgbv_modify(target_logits, draft_logits, log_a, log_b, uniforms, K: int, temperature: float = 1.0,
+                workspace: Optional[torch.Tensor] = None) -> ModifyOutput:
+    """One position of Algorithm 2 per batch row: target/draft logits [B,V], carried joint logs [B] (float64),
+    uniforms [B]; returns the drawn tokens and the carried logs with them appended."""
+    B, V = target_logits.shape
+    if tuple(draft_logits.shape) != (B, V) or draft_logits.dtype != target_logits.dtype:
+        raise ValueError("draft_logits must match target_logits")
+    for t, dt in ((log_a, torch.float64), (log_b, torch.float64), (uniforms, torch.float32)):
+        if tuple(t.shape) != (B,) or t.dtype != dt or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("log_a, log_b must be float64 [B], uniforms float32 [B], CUDA, contiguous")
+    if not (target_logits.is_cuda and target_logits.is_contiguous() and draft_logits.is_contiguous()):
+        raise ValueError("logits must be contiguous CUDA tensors")
+    dev = target_logits.device
+    out = ModifyOutput(torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.float64, device=dev),
+                       torch.empty(B, dtype=torch.float64, device=dev), torch.empty(B, dtype=torch.float64, device=dev),
+                       torch.empty(B, dtype=torch.int32, device=dev))
+    ws_ptr, ws_bytes = (workspace.data_ptr(), workspace.numel() * workspace.element_size()) \
+        if workspace is not None else (None, 0)
+    with torch.cuda.device(dev):
+        rc = load().sgbv_modify(target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+                                log_a.data_ptr(), log_b.data_ptr(), uniforms.data_ptr(), B, int(K), V,
+                                float(temperature), out.token.data_ptr(), out.log_a.data_ptr(), out.log_b.data_ptr(),
+                                out.resmass.data_ptr(), out.status.data_ptr(), ws_ptr, ws_bytes,
+                                torch.cuda.current_stream(dev).cuda_stream)
     if rc != OK:
         raise SgbvError(rc)
     return out

@@ -23,6 +23,8 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
     s.K = K;
     s.gamma = gamma;
     s.V = V;
+    s.cpr = K;
+    s.zq_rows = gamma + 1;
     s.ntiles = (V + kTile - 1) / kTile;
     const long rows = (long)B * K * gamma;
     long want = (4L * 148 + rows - 1) / rows;  // enough slices to fill the machine a few times over
@@ -40,7 +42,7 @@ struct Carve {
 };
 
 Carve carve(const Shape &s) {
-    const size_t NR = (size_t)s.B * s.K * s.gamma;
+    const size_t NR = (size_t)s.B * s.cpr * s.gamma;
     Carve c;
     size_t off = 0;
     // the ratio words sit at the head, at the same place for every shape: on the library's own scratch
@@ -303,6 +305,83 @@ int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dt
         ok &= cudaMemcpyAsync(out_status, st + o_status, n_tau, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok &= cudaStreamSynchronize(stream) == cudaSuccess;
     return ok ? SGBV_OK : SGBV_ERR_CUDA;
+}
+
+int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, const double *log_a, const double *log_b,
+                const float *uniforms, int B, int K, int V, float temperature, int32_t *out_token, double *out_log_a,
+                double *out_log_b, double *out_resmass, int32_t *out_status, void *workspace, size_t workspace_bytes,
+                void *stream_) {
+    if (!target_logits || !draft_logits || !log_a || !log_b || !uniforms || !out_token || !out_log_a || !out_log_b)
+        return SGBV_ERR_NULL;
+    int rc = check_shape(B, K, 1, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return SGBV_ERR_TEMPERATURE;
+    const size_t esz = dtype == SGBV_DTYPE_BF16 ? 2 : 4;
+    if (((uintptr_t)target_logits % esz) || ((uintptr_t)draft_logits % esz) || ((uintptr_t)log_a % 8) ||
+        ((uintptr_t)log_b % 8) || ((uintptr_t)uniforms % 4) || ((uintptr_t)out_token % 4) || ((uintptr_t)out_log_a % 8) ||
+        ((uintptr_t)out_log_b % 8) || ((uintptr_t)out_resmass % 8) || ((uintptr_t)out_status % 4))
+        return SGBV_ERR_ALIGN;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    Launch L;
+    L.s = make_shape(B, K, 1, V, temperature);
+    L.s.cpr = 1;      // one chain per batch row: K is only the exponent of Eq. 4's weights here
+    L.s.zq_rows = 1;  // and the target tensor holds just the row of this position
+    const Carve c = carve(L.s);
+    unsigned char *base = nullptr;
+    if (workspace) {
+        if (workspace_bytes < c.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
+        base = (unsigned char *)workspace;
+    } else {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total, kRatioWords * sizeof(double));
+        if (rc != SGBV_OK) return rc;
+        base = (unsigned char *)g_buf[dev].scratch;
+    }
+    L.ws.rows = (RowInfo *)(base + c.rows);
+    L.ws.part = (float *)(base + c.part);
+    L.ws.wpart = (float *)(base + c.wpart);
+    L.ws.dpart = (float *)(base + c.dpart);
+    L.ws.mpart = (float *)(base + c.mpart);
+    L.ws.ratio = (double *)(base + c.ratio);
+    L.ws.ratio_used = 0;  // (a single position per chain never takes the row walk)
+    L.ws.bonus = (float *)(base + c.bonus);
+    L.ws.bonus_in_smem = 0;
+    L.ws.h = (double *)(base + c.h);
+    L.ws.resmass = (double *)(base + c.resmass);
+    L.ws.status = (int32_t *)(base + c.status);
+    L.ws.prestatus = nullptr;
+    L.ws.error = (int32_t *)(base + c.error);
+    L.zq = target_logits;
+    L.zp = draft_logits;
+    L.dtype = dtype;
+    L.tok = nullptr;
+    L.u = uniforms;
+    L.out_tau = nullptr;
+    L.out_f = nullptr;
+    L.out_tokens = nullptr;
+    L.stream = stream;
+    L.carry_loga = log_a;
+    L.carry_logb = log_b;
+    bool fused = g_opt_path != 1 && fused_supported(L);
+    bool walked_rows = false;
+    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows) : 0;
+    if (n1 < 0) return n1;
+    if (n1 == 0) {
+        if (g_opt_path == 2) return SGBV_ERR_SHAPE;
+        fused = false;
+        L.ws.prestatus = L.ws.status;
+        if (cudaMemsetAsync(L.ws.status, 0, (size_t)B * sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+        if (cudaMemsetAsync(L.ws.error, 0, sizeof(int32_t), stream) != cudaSuccess) return SGBV_ERR_CUDA;
+        n1 = launch_twopass(L);
+        if (n1 < 0) return n1;
+    }
+    const int n2 = launch_modify_finish(L, uniforms, out_token, out_log_a, out_log_b, out_resmass, out_status);
+    if (n2 < 0) return n2;
+    t_last_launches = n1 + n2;
+    t_last_kernel = fused ? "fused_chain_kernel" : "otreduce_kernel";
+    return SGBV_OK;
 }
 
 int sgbv_last_launch_count(void) { return t_last_launches; }

@@ -57,6 +57,8 @@ struct Workspace {
 
 struct Shape {
     int B, K, gamma, V;
+    int cpr;      // draft chains per batch row: K for the verify step, 1 for Algorithm 2 (K is then only the exponent)
+    int zq_rows;  // rows of the target tensor per chain: gamma + 1 for the verify step, 1 for Algorithm 2
     int ntiles;   // ceil(V / kTile)
     int nsplit;   // slices per row in the two-pass path
     int tiles_per_slice;
@@ -170,10 +172,17 @@ struct Launch {
     cudaEvent_t ev_begin = nullptr;  // optional: recorded around the dominant kernel
     cudaEvent_t ev_end = nullptr;
     bool ratio_preset = false;       // ws.ratio is known to hold the NaN pattern (the library's own scratch)
+    // Algorithm 2: joint log-probabilities log q(s), log p(s) of what has been emitted so far, per chain (device
+    // pointers); c starts at exp(log p(s) - log q(s)) instead of 1.  NULL for the verify step.
+    const double *carry_loga = nullptr;
+    const double *carry_logb = nullptr;
 };
 
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
 int launch_finish(const Launch &L);   // weights, scan, extra token
+// Algorithm 2's draw per batch row from the cell sums of a gamma = 1 launch with carried logs
+int launch_modify_finish(const Launch &L, const float *u, int32_t *out_token, double *out_loga, double *out_logb,
+                         double *out_resmass, int32_t *out_status);
 bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0

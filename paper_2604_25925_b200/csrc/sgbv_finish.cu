@@ -6,9 +6,7 @@
 //   2. the scan of Algorithm 1 over drafts and positions with the pre-drawn uniforms;
 //   3. the extra token: inverse CDF of Eq. 4's residual (located through the cached tile sums,
 //      only one tile is recomputed) or of the target row after a full accept.
-#include <limits.h>
-
-#include "sgbv_common.cuh"
+#include "sgbv_sample.cuh"
 
 namespace sgbv {
 
@@ -18,7 +16,6 @@ constexpr int kMaxThreads = 1024;  // CTA size when few batch rows leave most SM
 constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps per row help); else 512 or 256
 constexpr int kMaxWarps = kMaxThreads / 32;
 constexpr int kTilesInSmem = 4096;  // rows up to 2^20 entries keep the bonus row's tile sums in shared memory
-constexpr int kEpt = 1;  // elements per thread inside one tile (threads beyond the tile hold none)
 static_assert(kMinThreads >= kTile, "one thread per element of a tile");
 
 // 1 - (1-u)^K as the geometric sum u (1 + (1-u) + ... + (1-u)^(K-1)): all terms are positive, so
@@ -72,158 +69,6 @@ __device__ double weight_full(double la, double lb, int K) {
     return clamp01(a * gfun(c, K) / den);
 }
 
-struct Pick {
-    int first;  // smallest index whose cumulative weight exceeds the target, INT_MAX if none
-    int last;   // largest index with positive weight, -1 if none
-};
-
-// Inverse CDF inside one tile: element x0 + kEpt*tid + j has weight wfun(x). base = cumulative
-// weight before the tile. All threads must call.
-template <typename F>
-__device__ Pick pick_in_tile(int x0, int x1, double base, double target, F wfun, double *sh_warp, int *sh_pick) {
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    float w[kEpt];
-    double local = 0.0;
-#pragma unroll
-    for (int j = 0; j < kEpt; ++j) {
-        const int x = x0 + kEpt * tid + j;
-        w[j] = (x < x1) ? wfun(x) : 0.0f;
-        local += (double)w[j];
-    }
-    double incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        double v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (tid == 0) {
-        sh_pick[0] = INT_MAX;
-        sh_pick[1] = -1;
-    }
-    if (lane == 31) sh_warp[wid] = incl;
-    __syncthreads();
-    // mass of the warps before this one: a butterfly over the lanes instead of a loop over the warps
-    const double wv = lane < (int)(blockDim.x >> 5) ? sh_warp[lane] : 0.0;
-    const double off = base + warp_sum(lane < wid ? wv : 0.0);
-    double cum = off + incl - local;
-#pragma unroll
-    for (int j = 0; j < kEpt; ++j) {
-        cum += (double)w[j];
-        const int x = x0 + kEpt * tid + j;
-        if (w[j] > 0.0f) {
-            atomicMax(&sh_pick[1], x);
-            if (cum > target) atomicMin(&sh_pick[0], x);
-        }
-    }
-    __syncthreads();
-    Pick p{sh_pick[0], sh_pick[1]};
-    __syncthreads();
-    return p;
-}
-
-// First tile whose inclusive prefix of the tile sums exceeds the target (float64, ascending
-// vocabulary order), found by the whole block: every thread owns a contiguous run of tiles, the
-// runs' totals are scanned across the block, and each thread searches its own run.  If rounding
-// leaves no such tile, the last tile with positive mass is taken, with a base that makes the
-// in-tile search fall back to its last positive element.  scale[t] (may be NULL) multiplies tile
-// t's sum.  relative: `target` is a fraction of the total of all tile sums (computed here on the
-// way) instead of a mass.  All threads must call.  Results: sh_i[2] = tile, sh_d[0] = mass before it,
-// sh_d[1] = target.
-__device__ void locate_tile(const float *partials, const float *scale, int ntiles, double target, bool relative,
-                            int *sh_i, double *sh_d, double *sh_warp) {
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const int nthreads = blockDim.x;
-    const int per = (ntiles + nthreads - 1) / nthreads;
-    const int t0 = min(ntiles, tid * per), t1 = min(ntiles, t0 + per);
-    // the thread's tile sums: the first four stay in registers for the search below
-    constexpr int kKeep = 4;
-    double kept[kKeep];
-    double local = 0.0;
-#pragma unroll
-    for (int e = 0; e < kKeep; ++e) {
-        const int t = t0 + e;
-        kept[e] = (t < t1) ? (double)partials[t] * (scale ? (double)scale[t] : 1.0) : 0.0;
-        local += kept[e];
-    }
-    for (int t = t0 + kKeep; t < t1; ++t) local += (double)partials[t] * (scale ? (double)scale[t] : 1.0);
-    double incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (tid == 0) {
-        sh_i[2] = INT_MAX;  // first tile that crosses the target
-        sh_i[3] = -1;       // last tile with positive mass
-    }
-    if (lane == 31) sh_warp[wid] = incl;
-    __syncthreads();
-    // the warps' totals: every warp adds up those of the warps before it (and all of them) with a butterfly
-    // over its lanes instead of one after the other
-    const double wv = lane < (nthreads >> 5) ? sh_warp[lane] : 0.0;
-    const double cum0 = incl - local + warp_sum(lane < wid ? wv : 0.0);
-    if (relative) target *= warp_sum(wv);  // the target is given as a fraction of the total of all tiles
-    double cum = cum0;
-    int first = INT_MAX, lastpos = -1;
-    double base = 0.0;
-    for (int t = t0; t < t1; ++t) {
-        double v;
-        if (t - t0 < kKeep) {
-            v = kept[0];
-#pragma unroll
-            for (int e = 1; e < kKeep; ++e)
-                if (t - t0 == e) v = kept[e];
-        } else {
-            v = (double)partials[t] * (scale ? (double)scale[t] : 1.0);
-        }
-        if (v > 0.0) lastpos = t;
-        if (first == INT_MAX && cum + v > target) {
-            first = t;
-            base = cum;
-        }
-        cum += v;
-    }
-    if (first != INT_MAX) atomicMin(&sh_i[2], first);
-    if (lastpos >= 0) atomicMax(&sh_i[3], lastpos);
-    __syncthreads();
-    if (first != INT_MAX && sh_i[2] == first) sh_d[0] = base;  // exactly one thread owns that tile
-    __syncthreads();
-    if (tid == 0) {
-        if (sh_i[2] == INT_MAX) {
-            sh_i[2] = max(sh_i[3], 0);
-            sh_d[0] = -INFINITY;
-        }
-        sh_d[1] = target;
-    }
-    __syncthreads();
-}
-
-// The 8 entries of a 256-entry tile that one lane takes when the row can be read in 16-byte pieces (the row starts
-// on a 16-byte boundary and V is a multiple of the entries per piece, so a piece lies inside the row or past it).
-template <typename T>
-__device__ __forceinline__ void load_tile_pieces(const T *zq, int tile, bool in, int V, int lane, float (&z)[kTile / 32]);
-template <>
-__device__ __forceinline__ void load_tile_pieces<float>(const float *zq, int tile, bool in, int V, int lane,
-                                                        float (&z)[kTile / 32]) {
-    const float ninf = -INFINITY;
-    const int xa = tile * kTile + lane * 4, xb = xa + kTile / 2;
-    const float4 a = (in && xa < V) ? __ldg(reinterpret_cast<const float4 *>(zq + xa)) : make_float4(ninf, ninf, ninf, ninf);
-    const float4 b = (in && xb < V) ? __ldg(reinterpret_cast<const float4 *>(zq + xb)) : make_float4(ninf, ninf, ninf, ninf);
-    z[0] = a.x; z[1] = a.y; z[2] = a.z; z[3] = a.w;
-    z[4] = b.x; z[5] = b.y; z[6] = b.z; z[7] = b.w;
-}
-template <>
-__device__ __forceinline__ void load_tile_pieces<uint16_t>(const uint16_t *zq, int tile, bool in, int V, int lane,
-                                                           float (&z)[kTile / 32]) {
-    const uint32_t ninf2 = 0xff80ff80u;  // two bf16 -inf
-    const int xa = tile * kTile + lane * 8;
-    const uint4 a = (in && xa < V) ? __ldg(reinterpret_cast<const uint4 *>(zq + xa)) : make_uint4(ninf2, ninf2, ninf2, ninf2);
-    z[0] = __uint_as_float(a.x << 16); z[1] = __uint_as_float(a.x & 0xffff0000u);
-    z[2] = __uint_as_float(a.y << 16); z[3] = __uint_as_float(a.y & 0xffff0000u);
-    z[4] = __uint_as_float(a.z << 16); z[5] = __uint_as_float(a.z & 0xffff0000u);
-    z[6] = __uint_as_float(a.w << 16); z[7] = __uint_as_float(a.w & 0xffff0000u);
-}
-
 template <typename T>
 __global__ void __launch_bounds__(kMaxThreads)
 finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const int32_t *__restrict__ tok_all,
@@ -245,13 +90,12 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     float *tile_s = ws.bonus_in_smem ? reinterpret_cast<float *>(lcp_s + ((K * K + 15) / 16) * 16)
                                                : ws.bonus + (size_t)blockIdx.x * 2 * s.ntiles;  // [ntiles]
     float *tile_m = tile_s + s.ntiles;                                        // [ntiles]
-    __shared__ double sh_warp[kMaxWarps];
-    __shared__ float sh_redf[kMaxWarps];
-    __shared__ int sh_pick[2];
-    __shared__ int sh_i[4];
+    __shared__ SampleScratch sc;
     __shared__ unsigned sh_or[2];
     __shared__ int sh_flags;
-    __shared__ double sh_d[2];
+    double *sh_warp = sc.warp;
+    int *sh_pick = sc.pick, *sh_i = sc.i;
+    double *sh_d = sc.d;
 
     // A kernel launched behind this one with programmatic stream serialisation (the next call's streaming
     // kernel) may be scheduled from now on; it waits for this grid to complete before it touches memory.
@@ -482,81 +326,9 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         }
     }
     if (from_q) {
-        // softmax(zq/T) of one row in a single pass over memory: every tile's maximum and its
-        // sum of exponentials relative to that maximum, then the row maximum, the factors that move
-        // the tile sums to it, the tile search and the pick inside the tile
         bool bad = false;
-        float m = -INFINITY;
-        constexpr int kNT = 4;  // tiles a warp has in flight
-        static_assert(kTile == 256, "a lane takes 8 entries of a tile");
-        const bool pieces = (reinterpret_cast<uintptr_t>(zq) % 16 == 0) && (s.V % (16 / (int)sizeof(T)) == 0);
-        for (int tb = wid * kNT; tb < s.ntiles; tb += nwarps * kNT) {
-            float z[kNT][kTile / 32];
-            if (pieces) {  // 16-byte loads
-#pragma unroll
-                for (int q = 0; q < kNT; ++q) load_tile_pieces<T>(zq, tb + q, tb + q < s.ntiles, s.V, lane, z[q]);
-            } else {
-#pragma unroll
-                for (int q = 0; q < kNT; ++q)
-#pragma unroll
-                    for (int e = 0; e < kTile / 32; ++e) {
-                        const int x = (tb + q) * kTile + lane + 32 * e;
-                        z[q][e] = (tb + q < s.ntiles && x < s.V) ? ld_logit(zq, x) : -INFINITY;
-                    }
-            }
-            // the four tiles are reduced side by side (independent shuffle chains)
-            float mt[kNT], acc[kNT];
-#pragma unroll
-            for (int q = 0; q < kNT; ++q) {
-                mt[q] = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < kTile / 32; ++e) {
-                    bad |= (z[q][e] != z[q][e]) | (z[q][e] == INFINITY);
-                    mt[q] = fmaxf(mt[q], z[q][e]);
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-                for (int q = 0; q < kNT; ++q) mt[q] = fmaxf(mt[q], __shfl_xor_sync(0xffffffffu, mt[q], o));
-#pragma unroll
-            for (int q = 0; q < kNT; ++q) {
-                acc[q] = 0.0f;
-                if (mt[q] > -INFINITY) {
-#pragma unroll
-                    for (int e = 0; e < kTile / 32; ++e) acc[q] += expo(z[q][e], mt[q], s.scale);
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-                for (int q = 0; q < kNT; ++q) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], o);
-#pragma unroll
-            for (int q = 0; q < kNT; ++q) {
-                if (lane == 0 && tb + q < s.ntiles) {
-                    tile_s[tb + q] = acc[q];
-                    tile_m[tb + q] = mt[q];
-                }
-                m = fmaxf(m, mt[q]);
-            }
-        }
-        if (lane == 0) sh_redf[wid] = m;
-        bad = __syncthreads_or(bad);
-        m = warp_max(lane < nwarps ? sh_redf[lane] : -INFINITY);
-        if (bad || !(m > -INFINITY)) {
-            flags |= SGBV_STATUS_NONFINITE_LOGIT;
-        } else {
-            // tile_m becomes the factor exp((m_t - m)/T) of its tile
-            for (int t = tid; t < s.ntiles; t += nthreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
-            __syncthreads();
-            // the target is us times the row's total, which the tile search computes on its way
-            locate_tile(tile_s, tile_m, s.ntiles, us, true, sh_i, sh_d, sh_warp);
-            const int sel = sh_i[2];
-            const int x0 = sel * kTile, x1 = min(s.V, x0 + kTile);
-            auto wfun = [&](int x) { return expo(ld_logit(zq, x), m, s.scale); };
-            Pick p = pick_in_tile(x0, x1, sh_d[0], sh_d[1], wfun, sh_warp, sh_pick);
-            y = (p.first != INT_MAX) ? p.first : p.last;
-        }
+        y = draw_from_row<T>(zq, s, us, tile_s, tile_m, &sc, bad);
+        if (bad) flags |= SGBV_STATUS_NONFINITE_LOGIT;
     }
 
     // ---- 4. outputs ------------------------------------------------------------------------------
@@ -574,6 +346,96 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         }
         out_tokens[(size_t)b * (g + 1) + j] = v;
     }
+}
+
+// Algorithm 2, one position: per batch row the token drawn from q_new by inverse CDF over the cached cell sums
+// (one cell recomputed), the carried joint logs with that token appended, and the normaliser.  The streaming
+// kernels ran with one chain per batch row, gamma = 1 and c = exp(log p(s) - log q(s)) carried in.
+template <typename T>
+__global__ void __launch_bounds__(kMaxThreads)
+modify_finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const float *__restrict__ u_all, Shape s,
+                     Workspace ws, const double *carry_loga, const double *carry_logb, int32_t *__restrict__ out_token,
+                     double *out_loga, double *out_logb, double *__restrict__ out_resmass, int32_t *__restrict__ out_status) {
+    __shared__ SampleScratch sc;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int nthreads = blockDim.x, nwarps = nthreads / 32;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // (launched behind the streaming kernel)
+    const bool lost = *ws.error != 0;
+    const RowInfo ri = ws.rows[b];
+    const int status_in = (ri.flags | (ws.prestatus ? ws.prestatus[b] : 0)) & SGBV_STATUS_NONFINITE_LOGIT;
+    const float *wp = ws.wpart + (size_t)b * s.ntiles;
+    double local = 0.0;
+    for (int t = tid; t < s.ntiles; t += nthreads) local += (double)wp[t];
+    local = warp_sum(local);
+    if (lane == 0) sc.warp[wid] = local;
+    __syncthreads();
+    const double W = warp_sum(lane < nwarps ? sc.warp[lane] : 0.0);
+    __syncthreads();
+    const double la = carry_loga[b], lb = carry_logb[b];
+    if (lost || status_in) {
+        if (tid == 0) {
+            out_token[b] = -1;
+            out_loga[b] = NAN;
+            out_logb[b] = NAN;
+            if (out_resmass) out_resmass[b] = NAN;
+            if (out_status) out_status[b] = status_in | (lost ? SGBV_STATUS_TIMEOUT : 0);
+        }
+        return;
+    }
+    const T *zq = zq_all + (size_t)b * s.V, *zp = zp_all + (size_t)b * s.V;
+    const double us = (double)u_all[b];
+    int y = -1, flags = 0;
+    if (W > 0.0) {
+        locate_tile(wp, nullptr, s.ntiles, us * W, false, sc.i, sc.d, sc.warp);
+        const int sel = sc.i[2];
+        const int x0 = sel * kTile, x1 = min(s.V, x0 + kTile);
+        auto wfun = [&](int x) {
+            float eq = expo(ld_logit(zq, x), ri.mq, s.scale);
+            float ep = expo(ld_logit(zp, x), ri.mp, s.scale);
+            float w, d0, d1;
+            element_terms<false>(eq, ep, ri.kappa, ri.c, s.K, w, d0, d1);
+            return w;
+        };
+        Pick pk = pick_in_tile(x0, x1, sc.d[0], sc.d[1], wfun, sc.warp, sc.pick);
+        y = (pk.first != INT_MAX) ? pk.first : pk.last;
+    } else {  // no residual mass at all: the draw comes from q(.|s) itself
+        flags |= SGBV_STATUS_DEGENERATE_RESIDUAL;
+        bool bad = false;
+        float *tile_s = ws.bonus + (size_t)b * 2 * s.ntiles;
+        y = draw_from_row<T>(zq, s, us, tile_s, tile_s + s.ntiles, &sc, bad);
+        if (bad) flags |= SGBV_STATUS_NONFINITE_LOGIT;
+    }
+    if (tid == 0) {
+        const bool failed = y < 0;
+        out_token[b] = y;
+        const double lq = failed ? NAN : ((double)ld_logit(zq, y) - (double)ri.mq) * s.inv_T - log(ri.Zq);
+        const double lp = failed ? NAN : ((double)ld_logit(zp, y) - (double)ri.mp) * s.inv_T - log(ri.Zp);
+        out_loga[b] = la + lq;
+        out_logb[b] = lb + lp;
+        if (out_resmass) out_resmass[b] = W / ri.Zq;
+        if (out_status) out_status[b] = flags;
+    }
+}
+
+template <typename T>
+int run_modify(const Launch &L, const float *u, int32_t *out_token, double *out_loga, double *out_logb,
+               double *out_resmass, int32_t *out_status) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(L.s.B);
+    cfg.blockDim = dim3(L.s.B <= 148 ? kMaxThreads : L.s.B <= 296 ? 512 : kMinThreads);
+    cfg.stream = L.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, modify_finish_kernel<T>, (const T *)L.zq, (const T *)L.zp, u, L.s, L.ws,
+                                       L.carry_loga, L.carry_logb, out_token, out_loga, out_logb, out_resmass, out_status);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return SGBV_ERR_CUDA;
+    }
+    return 1;
 }
 
 template <typename T>
@@ -618,6 +480,12 @@ int run(const Launch &L) {
 
 int launch_finish(const Launch &L) {
     return L.dtype == SGBV_DTYPE_BF16 ? run<uint16_t>(L) : run<float>(L);
+}
+
+int launch_modify_finish(const Launch &L, const float *u, int32_t *out_token, double *out_loga, double *out_logb,
+                         double *out_resmass, int32_t *out_status) {
+    return L.dtype == SGBV_DTYPE_BF16 ? run_modify<uint16_t>(L, u, out_token, out_loga, out_logb, out_resmass, out_status)
+                                      : run_modify<float>(L, u, out_token, out_loga, out_logb, out_resmass, out_status);
 }
 
 }  // namespace sgbv

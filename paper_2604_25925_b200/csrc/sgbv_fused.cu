@@ -59,6 +59,7 @@ struct FusedParams {
     int cluster;      // CTAs per cluster
     int slice_cells;  // cells of a row per CTA (at most kCtaCells)
     int nchains;      // B*K
+    const double *carry_loga, *carry_logb;  // Algorithm 2: per-chain joint logs carried in (else NULL)
     int *error_flag;  // set to 1 if a bounded wait expired
     long long poll_limit;  // cycles a poll of a published ratio may take (row walk)
     int withhold;     // failure-detection test: the first row of every chain does not publish its ratio
@@ -555,7 +556,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     int bk_a = 0, i_a = 0;  // (set when B becomes A)
     int bk_b = row_mode ? cid / s.gamma : cid;
     int i_b = row_mode ? cid % s.gamma : 0;
-    const unsigned char *q_b = zq_warp + ((size_t)bk_b * (s.gamma + 1) + i_b) * row_bytes;  // this warp's first cell of row B
+    const unsigned char *q_b = zq_warp + ((size_t)bk_b * s.zq_rows + i_b) * row_bytes;  // this warp's first cell of row B
     const unsigned char *p_b = zp_warp + ((size_t)bk_b * s.gamma + i_b) * row_bytes;
     if (nrows > 0) {
 #pragma unroll
@@ -566,7 +567,10 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     // The last warp of this CTA combines the partials, carries c_i and fetches the token logits of a row while its
     // first sweep runs (every lane the same words).
     const bool combiner = warp == kFWarps - 1;
+    // c at the start of chain bk: 1, or exp(log p(s) - log q(s)) of what Algorithm 2 carries in
+#define SGBV_C0(BK) (p.carry_loga ? exp_short(p.carry_logb[BK] - p.carry_loga[BK]) : 1.0)
     double c_carry = 1.0;  // chain walk: c of the row whose exchange comes next (the first row of the walk starts a chain)
+    if (combiner && nrows > 0) c_carry = SGBV_C0(bk_b);
 
     float fmq[kCellsPerWarp], rt[kCellsPerWarp];  // row A: what the second sweep needs of every cell
     RowScalars rs;                                 // row A
@@ -584,8 +588,9 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
             i_d -= s.gamma;
             bk_d += wrap_bk;
         }
-        const bool more = n + 2 < nrows && !timed_out;
-        const unsigned char *q_d = zq_warp + ((size_t)bk_d * (s.gamma + 1) + i_d) * row_bytes;
+        const bool has_d = n + 2 < nrows;
+        const bool more = has_d && !timed_out;
+        const unsigned char *q_d = zq_warp + ((size_t)bk_d * s.zq_rows + i_d) * row_bytes;
         const unsigned char *p_d = zp_warp + ((size_t)bk_d * s.gamma + i_d) * row_bytes;
         const size_t r_a = (size_t)bk_a * s.gamma + i_a, r_b = (size_t)bk_b * s.gamma + i_b;
 
@@ -596,9 +601,9 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
         const uint32_t xbar = xbar_u32 + 8u * (uint32_t)par;
         if (combiner && has_b) {
             if (C > 1 && lane == 0) mbar_expect_tx(xbar, xbytes);  // row B's partials of the cluster's CTAs
-            int t = p.tok[r_b];
+            int t = p.tok ? p.tok[r_b] : 0;
             if (t < 0 || t >= s.V) t = 0;  // the finishing kernel flags the batch row
-            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk_b * (s.gamma + 1) + i_b) * s.V, t);
+            zq_tok = ld_logit(reinterpret_cast<const T *>(p.zq) + ((size_t)bk_b * s.zq_rows + i_b) * s.V, t);
             zp_tok = ld_logit(reinterpret_cast<const T *>(p.zp) + r_b * s.V, t);
         }
 
@@ -765,7 +770,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
                 // butterfly over the lanes).  Those rows are walked by other clusters at about the same
                 // time and publish right after their own statistics, which do not depend on c: no chain of
                 // waits forms.  Every lane polls one of them.  Bounded waits.
-                cd = 1.0;
+                cd = SGBV_C0(bk_b);
                 const size_t r0 = (size_t)bk_b * s.gamma;
                 for (int j0 = 0; j0 < i_b; j0 += 32) {
                     double w = 1.0;
@@ -798,7 +803,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
             bar_arrive(2, kFThreads);
             // off the critical path: c of the next row of the chain walk (c_{i+1} = c_i ratio, and 1 at the start of
             // the next chain), and the row's record for the finishing kernel
-            if (!row_mode) c_carry = (i_b + 1 < s.gamma) ? cd * SGBV_RATIO() : 1.0;
+            if (!row_mode) c_carry = (i_b + 1 < s.gamma) ? cd * SGBV_RATIO() : (has_d ? SGBV_C0(bk_d) : 1.0);
             if (lane == 0 && rank == 0) {
                 // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
                 // -inf only has Z = 0
@@ -848,6 +853,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     if (warp == 0) tmem_dealloc(ctl->tmem_base, kTmemCols);
 #undef SGBV_ISSUE
 #undef SGBV_FIRST_SWEEP_CELL
+#undef SGBV_C0
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -925,7 +931,9 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
     fp.ws = L.ws;
     fp.cluster = plan.cluster;
     fp.slice_cells = plan.slice_cells;
-    fp.nchains = L.s.B * L.s.K;
+    fp.nchains = L.s.B * L.s.cpr;
+    fp.carry_loga = L.carry_loga;
+    fp.carry_logb = L.carry_logb;
     fp.error_flag = error_flag;
     fp.poll_limit = g_opt_poll_us > 0 ? (long long)g_opt_poll_us * 2000ll : kWaitLimitCycles;
     fp.withhold = g_opt_withhold;
@@ -964,7 +972,7 @@ template <typename T, int KT>
 int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const Shape &s = L.s;
     const int cells = s.ntiles;
-    const long nchains = (long)s.B * s.K, units = nchains * s.gamma;
+    const long nchains = (long)s.B * s.cpr, units = nchains * s.gamma;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDevices) return SGBV_ERR_CUDA;
     if (prepare<T, false, KT>(dev) != cudaSuccess || prepare<T, true, KT>(dev) != cudaSuccess) {

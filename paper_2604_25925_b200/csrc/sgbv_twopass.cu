@@ -20,7 +20,7 @@ rowstats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
     const int sl = blockIdx.x % s.nsplit;
     const int i = r % s.gamma;
     const int bk = r / s.gamma;
-    const T *zq = zq_all + ((size_t)bk * (s.gamma + 1) + i) * s.V;
+    const T *zq = zq_all + ((size_t)bk * s.zq_rows + i) * s.V;
     const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
     const int x0 = sl * s.tiles_per_slice * kTile;
     const int x1 = min(s.V, x0 + s.tiles_per_slice * kTile);
@@ -43,7 +43,7 @@ rowstats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
         red[0][wid] = mq;
         red[1][wid] = mp;
     }
-    if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status + bk / s.K, SGBV_STATUS_NONFINITE_LOGIT);
+    if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status + bk / s.cpr, SGBV_STATUS_NONFINITE_LOGIT);
     if (threadIdx.x == 0) {
         float a = red[0][0], b = red[1][0];
         for (int w = 1; w < kThreads / 32; ++w) {
@@ -88,10 +88,12 @@ rowstats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
 template <typename T>
 __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all,
                              const int32_t *__restrict__ tok, Shape s, const float *__restrict__ part,
-                             RowInfo *__restrict__ rows, int32_t *__restrict__ status) {
+                             RowInfo *__restrict__ rows, int32_t *__restrict__ status,
+                             const double *__restrict__ carry_loga, const double *__restrict__ carry_logb) {
     const int bk = blockIdx.x * blockDim.x + threadIdx.x;
-    if (bk >= s.B * s.K) return;
-    double la = 0.0, lb = 0.0;
+    if (bk >= s.B * s.cpr) return;
+    // joint log-probabilities of the prefix: 0 at the start of a draft, or what Algorithm 2 carries in
+    double la = carry_loga ? carry_loga[bk] : 0.0, lb = carry_logb ? carry_logb[bk] : 0.0;
     for (int i = 0; i < s.gamma; ++i) {
         const int r = bk * s.gamma + i;
         const float *p = part + (size_t)r * s.nsplit * 4;
@@ -105,7 +107,7 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
             if (p[sl * 4 + 0] > -INFINITY) Zq += (double)p[sl * 4 + 1] * exp2((double)(p[sl * 4 + 0] - mq) * (double)s.scale);
             if (p[sl * 4 + 2] > -INFINITY) Zp += (double)p[sl * 4 + 3] * exp2((double)(p[sl * 4 + 2] - mp) * (double)s.scale);
         }
-        if (!(mq > -INFINITY) || !(mp > -INFINITY)) atomicOr(status + bk / s.K, SGBV_STATUS_NONFINITE_LOGIT);
+        if (!(mq > -INFINITY) || !(mp > -INFINITY)) atomicOr(status + bk / s.cpr, SGBV_STATUS_NONFINITE_LOGIT);
         RowInfo ri;
         ri.Zq = Zq;
         ri.Zp = Zp;
@@ -117,12 +119,13 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
         ri.pad_ = 0;
         ri.kappa = (float)(c * Zq / Zp);
         rows[r] = ri;
+        if (!tok) break;  // Algorithm 2: one position, nothing follows
         int t = tok[r];
         if (t < 0 || t >= s.V) {
-            atomicOr(status + bk / s.K, SGBV_STATUS_TOKEN_RANGE);
+            atomicOr(status + bk / s.cpr, SGBV_STATUS_TOKEN_RANGE);
             t = 0;
         }
-        const float zqt = ld_logit(zq_all, ((size_t)bk * (s.gamma + 1) + i) * s.V + t);
+        const float zqt = ld_logit(zq_all, ((size_t)bk * s.zq_rows + i) * s.V + t);
         const float zpt = ld_logit(zp_all, ((size_t)bk * s.gamma + i) * s.V + t);
         la += ((double)zqt - (double)mq) * s.inv_T - log(Zq);
         lb += ((double)zpt - (double)mp) * s.inv_T - log(Zp);
@@ -168,7 +171,7 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
     const int sl = blockIdx.x % s.nsplit;
     const int i = r % s.gamma;
     const int bk = r / s.gamma;
-    const T *zq = zq_all + ((size_t)bk * (s.gamma + 1) + i) * s.V;
+    const T *zq = zq_all + ((size_t)bk * s.zq_rows + i) * s.V;
     const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
     const RowInfo ri = rows[r];
     const int t0 = sl * s.tiles_per_slice, t1 = min(s.ntiles, t0 + s.tiles_per_slice);
@@ -182,13 +185,13 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
 template <typename T>
 int run(const Launch &L) {
     const Shape &s = L.s;
-    const int NR = s.B * s.K * s.gamma;
+    const int NR = s.B * s.cpr * s.gamma;
     const unsigned grid = (unsigned)NR * (unsigned)s.nsplit;
     const T *zq = (const T *)L.zq, *zp = (const T *)L.zp;
     rowstats_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.part, L.ws.status);
-    const int nbk = s.B * s.K;
+    const int nbk = s.B * s.cpr;
     chain_kernel<T><<<(nbk + 127) / 128, 128, 0, L.stream>>>(zq, zp, L.tok, s, L.ws.part, L.ws.rows,
-                                                            L.ws.status);
+                                                            L.ws.status, L.carry_loga, L.carry_logb);
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
     otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, L.ws.wpart, L.ws.dpart, L.ws.mpart);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
