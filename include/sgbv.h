@@ -141,6 +141,38 @@ int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, 
                 int32_t *out_status, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Comparison verifiers of the paper's Section 3 behind the same boundary (device pointers, layouts and
+ * error behaviour as sgbv_verify_ex; workspace >= sgbv_workspace_bytes(B,K,gamma,V,dtype) or NULL).  They
+ * serve the verification-cost comparison of the paper's Table 2 and are not tuned like the block verifier.
+ *
+ * sgbv_verify_kseq: SpecTr's position-wise K-SEQ (Section 3.2).  At every position the drafts that still match
+ * the accepted prefix (n of them, n = K at first) are tried in order; draft k's token x is accepted if
+ * eta < min{1, q(x)/(rho p(x))}, rho in [1,n] the root of 1 - (1 - beta(rho))^n = rho beta(rho) with
+ * beta(rho) = sum_x min{p(x), q(x)/rho}; the first accepted token extends the prefix.  If none is accepted the
+ * extra token comes from norm(max{q - rho p, 0}); after gamma accepted positions from the target row after
+ * the block.  uniforms[b, k*gamma + i] is eta of draft k at position i (0-based), the last entry draws the
+ * extra token.
+ *   out_rho         [B,gamma] float64 or NULL: rho of every position reached, NaN elsewhere
+ *   out_accept_prob [B,K,gamma] float64 or NULL: acceptance probability of every token tried, NaN elsewhere
+ * sgbv_verify_token: token-level speculative sampling (Section 3.1) = K-SEQ with one draft (rho = 1);
+ *   tensors without the K axis: target [B,gamma+1,V], draft [B,gamma,V], tokens [B,gamma], uniforms [B,gamma+1].
+ * sgbv_verify_gbv: single-draft greedy block verification (Section 3.3) = the block verifier with K = 1; same
+ *   tensors as sgbv_verify_token; out_accept_prob [B,gamma] or NULL holds the sub-block weights alpha(x^i).
+ */
+int sgbv_verify_kseq(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                     const float *uniforms, int B, int K, int gamma, int V, float temperature,
+                     int32_t *out_accept_len, int32_t *out_tokens, double *out_rho, double *out_accept_prob,
+                     int32_t *out_status, void *workspace, size_t workspace_bytes, void *stream);
+int sgbv_verify_token(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                      const float *uniforms, int B, int gamma, int V, float temperature, int32_t *out_accept_len,
+                      int32_t *out_tokens, double *out_accept_prob, int32_t *out_status, void *workspace,
+                      size_t workspace_bytes, void *stream);
+int sgbv_verify_gbv(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                    const float *uniforms, int B, int gamma, int V, float temperature, int32_t *out_accept_len,
+                    int32_t *out_tokens, double *out_accept_prob, int32_t *out_status, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
+/*
  * Allocation-free form of sgbv_verify_ex (the paper has no counterpart: this entry point exists
  * for deployment, not for the method).
  *

@@ -26,7 +26,8 @@ DTYPE_BF16 = 1
 EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_verify_ex",
            "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_last_main_kernel", "sgbv_status_string",
            "sgbv_profile_begin",
-           "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option", "sgbv_modify")
+           "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option", "sgbv_modify", "sgbv_verify_kseq",
+           "sgbv_verify_token", "sgbv_verify_gbv")
 
 _lib = None
 
@@ -67,6 +68,11 @@ def load() -> ctypes.CDLL:
         lib.sgbv_verify_host.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
         lib.sgbv_modify.restype = i32
         lib.sgbv_modify.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.sgbv_verify_kseq.restype = i32
+        lib.sgbv_verify_kseq.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp, vp, sz, vp]
+        for fn in (lib.sgbv_verify_token, lib.sgbv_verify_gbv):
+            fn.restype = i32
+            fn.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         lib.sgbv_last_launch_count.restype = i32
         lib.sgbv_last_launch_count.argtypes = []
         lib.sgbv_last_main_kernel.restype = ctypes.c_char_p
@@ -311,3 +317,63 @@ def sgbv_modify(target_logits, draft_logits, log_a, log_b, uniforms, K: int, tem
     if rc != OK:
         raise SgbvError(rc)
     return out
+
+
+@dataclass
+class PositionwiseOutput:
+    accept_len: torch.Tensor            # [B] int32
+    tokens: torch.Tensor                # [B, gamma+1] int32
+    rho: Optional[torch.Tensor]         # [B, gamma] float64 (K-SEQ only)
+    accept_prob: torch.Tensor           # [B, K, gamma] float64 (NaN where a token was not tried)
+    status: torch.Tensor                # [B] int32
+
+
+def sgbv_verify_kseq(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0) -> PositionwiseOutput:
+    """SpecTr's K-SEQ on the verify step's tensors ([B,K,gamma+1,V], [B,K,gamma,V], [B,K,gamma], [B,K*gamma+1])."""
+    B, K, gamma, V = _shapes(target_logits, draft_logits, draft_tokens, uniforms)
+    dev = target_logits.device
+    out = PositionwiseOutput(torch.empty(B, dtype=torch.int32, device=dev),
+                             torch.empty((B, gamma + 1), dtype=torch.int32, device=dev),
+                             torch.empty((B, gamma), dtype=torch.float64, device=dev),
+                             torch.empty((B, K, gamma), dtype=torch.float64, device=dev),
+                             torch.empty(B, dtype=torch.int32, device=dev))
+    with torch.cuda.device(dev):
+        rc = load().sgbv_verify_kseq(target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+                                     draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, V, float(temperature),
+                                     out.accept_len.data_ptr(), out.tokens.data_ptr(), out.rho.data_ptr(),
+                                     out.accept_prob.data_ptr(), out.status.data_ptr(), None, 0,
+                                     torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def _single_draft(name, target_logits, draft_logits, draft_tokens, uniforms, temperature):
+    B, g1, V = target_logits.shape
+    gamma = g1 - 1
+    if tuple(draft_logits.shape) != (B, gamma, V) or tuple(draft_tokens.shape) != (B, gamma) or \
+            tuple(uniforms.shape) != (B, gamma + 1):
+        raise ValueError("single-draft tensors: target [B,gamma+1,V], draft [B,gamma,V], tokens [B,gamma], uniforms [B,gamma+1]")
+    dev = target_logits.device
+    out = PositionwiseOutput(torch.empty(B, dtype=torch.int32, device=dev),
+                             torch.empty((B, gamma + 1), dtype=torch.int32, device=dev), None,
+                             torch.empty((B, 1, gamma), dtype=torch.float64, device=dev),
+                             torch.empty(B, dtype=torch.int32, device=dev))
+    with torch.cuda.device(dev):
+        rc = getattr(load(), name)(target_logits.data_ptr(), draft_logits.data_ptr(), _dtype_code(target_logits),
+                                   draft_tokens.data_ptr(), uniforms.data_ptr(), B, gamma, V, float(temperature),
+                                   out.accept_len.data_ptr(), out.tokens.data_ptr(), out.accept_prob.data_ptr(),
+                                   out.status.data_ptr(), None, 0, torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_verify_token(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0) -> PositionwiseOutput:
+    """Token-level speculative sampling, one draft per batch row."""
+    return _single_draft("sgbv_verify_token", target_logits, draft_logits, draft_tokens, uniforms, temperature)
+
+
+def sgbv_verify_gbv(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0) -> PositionwiseOutput:
+    """Single-draft greedy block verification (the block verifier with K = 1)."""
+    return _single_draft("sgbv_verify_gbv", target_logits, draft_logits, draft_tokens, uniforms, temperature)

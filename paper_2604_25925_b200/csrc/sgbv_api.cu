@@ -75,6 +75,8 @@ struct DeviceBuffers {
     size_t scratch_bytes = 0;
     void *stage = nullptr;
     size_t stage_bytes = 0;
+    void *idx = nullptr;        // accepted-draft indices that sgbv_verify_gbv has no output for
+    size_t idx_bytes = 0;
     // the ratio words at the head of the scratch may not hold the "not published yet" pattern (a call
     // failed between the kernel that consumes them and the one that puts them back)
     bool ratio_dirty = false;
@@ -382,6 +384,83 @@ int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, 
     t_last_launches = n1 + n2;
     t_last_kernel = fused ? "fused_chain_kernel" : "otreduce_kernel";
     return SGBV_OK;
+}
+
+int sgbv_verify_kseq(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                     const float *uniforms, int B, int K, int gamma, int V, float temperature, int32_t *out_accept_len,
+                     int32_t *out_tokens, double *out_rho, double *out_accept_prob, int32_t *out_status, void *workspace,
+                     size_t workspace_bytes, void *stream_) {
+    if (!target_logits || !draft_logits || !draft_tokens || !uniforms || !out_accept_len || !out_tokens) return SGBV_ERR_NULL;
+    int rc = check_shape(B, K, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return SGBV_ERR_TEMPERATURE;
+    const size_t esz = dtype == SGBV_DTYPE_BF16 ? 2 : 4;
+    if (((uintptr_t)target_logits % esz) || ((uintptr_t)draft_logits % esz) || ((uintptr_t)draft_tokens % 4) ||
+        ((uintptr_t)uniforms % 4) || ((uintptr_t)out_accept_len % 4) || ((uintptr_t)out_tokens % 4) ||
+        ((uintptr_t)out_rho % 8) || ((uintptr_t)out_accept_prob % 8) || ((uintptr_t)out_status % 4))
+        return SGBV_ERR_ALIGN;
+    Launch L;
+    L.s = make_shape(B, K, gamma, V, temperature);
+    const Carve c = carve(L.s);
+    unsigned char *base = nullptr;
+    if (workspace) {
+        if (workspace_bytes < c.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
+        base = (unsigned char *)workspace;
+    } else {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total, kRatioWords * sizeof(double));
+        if (rc != SGBV_OK) return rc;
+        base = (unsigned char *)g_buf[dev].scratch;
+    }
+    L.zq = target_logits;
+    L.zp = draft_logits;
+    L.dtype = dtype;
+    L.tok = draft_tokens;
+    L.u = uniforms;
+    L.out_tau = out_accept_len;
+    L.out_f = nullptr;
+    L.out_tokens = out_tokens;
+    L.stream = (cudaStream_t)stream_;
+    const int n = launch_kseq(L, (float *)(base + c.bonus), out_rho, out_accept_prob,
+                              out_status ? out_status : (int32_t *)(base + c.status));
+    if (n < 0) return n;
+    t_last_launches = n;
+    t_last_kernel = "kseq_kernel";
+    return SGBV_OK;
+}
+
+int sgbv_verify_token(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                      const float *uniforms, int B, int gamma, int V, float temperature, int32_t *out_accept_len,
+                      int32_t *out_tokens, double *out_accept_prob, int32_t *out_status, void *workspace,
+                      size_t workspace_bytes, void *stream) {
+    return sgbv_verify_kseq(target_logits, draft_logits, dtype, draft_tokens, uniforms, B, 1, gamma, V, temperature,
+                            out_accept_len, out_tokens, nullptr, out_accept_prob, out_status, workspace, workspace_bytes,
+                            stream);
+}
+
+int sgbv_verify_gbv(const void *target_logits, const void *draft_logits, int dtype, const int32_t *draft_tokens,
+                    const float *uniforms, int B, int gamma, int V, float temperature, int32_t *out_accept_len,
+                    int32_t *out_tokens, double *out_accept_prob, int32_t *out_status, void *workspace,
+                    size_t workspace_bytes, void *stream) {
+    if (!out_accept_len) return SGBV_ERR_NULL;
+    // single-draft greedy block verification is the K = 1 case of the block verifier; the accepted draft index
+    // (0 or -1) lands in scratch
+    int rc = check_shape(B, 1, gamma, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+    int32_t *f_scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].idx, &g_buf[dev].idx_bytes, (size_t)B * sizeof(int32_t));
+        if (rc != SGBV_OK) return rc;
+        f_scratch = (int32_t *)g_buf[dev].idx;
+    }
+    return verify_device(target_logits, draft_logits, dtype, draft_tokens, uniforms, B, 1, gamma, V, temperature,
+                         out_accept_len, f_scratch, out_tokens, workspace, workspace_bytes, out_accept_prob, nullptr,
+                         out_status, (cudaStream_t)stream);
 }
 
 int sgbv_last_launch_count(void) { return t_last_launches; }

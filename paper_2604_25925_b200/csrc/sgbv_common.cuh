@@ -183,6 +183,8 @@ int launch_finish(const Launch &L);   // weights, scan, extra token
 // Algorithm 2's draw per batch row from the cell sums of a gamma = 1 launch with carried logs
 int launch_modify_finish(const Launch &L, const float *u, int32_t *out_token, double *out_loga, double *out_logb,
                          double *out_resmass, int32_t *out_status);
+// K-SEQ / token-level verification, one CTA per batch row; tile_scratch: [B][2][ntiles] floats
+int launch_kseq(const Launch &L, float *tile_scratch, double *out_rho, double *out_acc, int32_t *out_status);
 bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0

@@ -83,3 +83,68 @@ def test_modify_over_several_positions_follows_the_oracle_chain():
         np.testing.assert_allclose(la.cpu().numpy()[ok], rla[ok], atol=5e-5)
         la = torch.from_numpy(rla).cuda()
         lb = torch.from_numpy(rlb).cuda()
+
+
+def _kseq_compare(inp, T):
+    out = binding.sgbv_verify_kseq(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, T)
+    torch.cuda.synchronize()
+    ref = oracle.kseq_verify(inp.target_logits.float().cpu().numpy(), inp.draft_logits.float().cpu().numpy(),
+                             inp.draft_tokens.cpu().numpy(), inp.uniforms.cpu().numpy(), T)
+    tau, tokens, st = out.accept_len.cpu().numpy(), out.tokens.cpu().numpy(), out.status.cpu().numpy()
+    rho, acc = out.rho.cpu().numpy(), out.accept_prob.cpu().numpy()
+    B = tau.shape[0]
+    near = (ref.margin_accept < 1e-6) | (ref.margin_sample < 1e-6)     # a uniform on a threshold: counted, excused
+    assert near.sum() <= max(2, B // 3)
+    ok = ~near
+    assert (st[ok] == ref.status[ok]).all()
+    assert (tau[ok] == ref.tau[ok]).all() and (tokens[ok] == ref.tokens[ok]).all()
+    # rho and the acceptance probabilities of what both sides tried
+    both = ok[:, None] & ~np.isnan(ref.rho) & ~np.isnan(rho)
+    np.testing.assert_allclose(rho[both], ref.rho[both], rtol=1e-5)
+    assert (np.isnan(rho[ok]) == np.isnan(ref.rho[ok])).all()
+    both = ok[:, None, None] & ~np.isnan(ref.acc) & ~np.isnan(acc)
+    np.testing.assert_allclose(acc[both], ref.acc[both], rtol=1e-5, atol=1e-9)
+    return out, ref
+
+
+@pytest.mark.parametrize("B,K,gamma,V,dtype,T,alpha", [(6, 3, 4, 4099, "fp32", 0.8, 0.8), (8, 4, 4, 32000, "fp32", 1.0, 0.85),
+                                                      (5, 1, 5, 9000, "fp32", 0.9, 0.9), (4, 8, 3, 32000, "bf16", 0.7, 0.7),
+                                                      (2, 2, 2, 151936, "fp32", 1.0, 0.9), (3, 5, 2, 17, "fp32", 1.0, 0.5)])
+def test_kseq_matches_the_oracle(B, K, gamma, V, dtype, T, alpha):
+    cfg = workloads.VerifyConfig("ks", B=B, K=K, gamma=gamma, V=V, dtype=dtype, temperature=T, alpha=alpha, seed=640 + K)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    _kseq_compare(inp, T)
+    assert binding.last_main_kernel() == "kseq_kernel"
+
+
+def test_kseq_flags():
+    cfg = workloads.VerifyConfig("ksf", B=4, K=2, gamma=2, V=300, alpha=0.8, seed=9)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    zq, tok = inp.target_logits.clone(), inp.draft_tokens.clone()
+    tok[1, 0, 1] = 300
+    zq[2, :, 0, 17] = float("nan")
+    mod = workloads.VerifyInputs(cfg, zq, inp.draft_logits, tok, inp.uniforms)
+    out, ref = _kseq_compare(mod, 1.0)
+    st = out.status.cpu().numpy()
+    assert st[1] & binding.STATUS_TOKEN_RANGE and st[2] & binding.STATUS_NONFINITE_LOGIT and st[0] == 0
+    assert (out.accept_len.cpu().numpy()[1:3] == -1).all()
+
+
+def test_single_draft_entry_points():
+    """Token-level speculative sampling = K-SEQ with one draft; single-draft greedy block verification = the block
+    verifier with K = 1 (whose parity with an independent GBV is covered by the verify-step tests)."""
+    cfg = workloads.VerifyConfig("sd", B=7, K=1, gamma=5, V=12000, temperature=0.8, alpha=0.85, seed=12)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    zq, zp, tok = inp.target_logits[:, 0].contiguous(), inp.draft_logits[:, 0].contiguous(), inp.draft_tokens[:, 0].contiguous()
+    sd = binding.sgbv_verify_token(zq, zp, tok, inp.uniforms, cfg.temperature)
+    ks = binding.sgbv_verify_kseq(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, cfg.temperature)
+    gb = binding.sgbv_verify_gbv(zq, zp, tok, inp.uniforms, cfg.temperature)
+    ex = binding.sgbv_verify_ex(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, cfg.temperature)
+    torch.cuda.synchronize()
+    assert torch.equal(sd.accept_len, ks.accept_len) and torch.equal(sd.tokens, ks.tokens)
+    assert torch.equal(gb.accept_len, ex.accept_len) and torch.equal(gb.tokens, ex.tokens)
+    assert torch.equal(gb.accept_prob[:, 0], ex.h[:, 0])
+    ref = oracle.kseq_verify(inp.target_logits.cpu().numpy(), inp.draft_logits.cpu().numpy(), inp.draft_tokens.cpu().numpy(),
+                             inp.uniforms.cpu().numpy(), cfg.temperature)
+    ok = (ref.margin_accept >= 1e-6) & (ref.margin_sample >= 1e-6)
+    assert (sd.accept_len.cpu().numpy()[ok] == ref.tau[ok]).all()
