@@ -173,6 +173,22 @@ int sgbv_verify_gbv(const void *target_logits, const void *draft_logits, int dty
                     size_t workspace_bytes, void *stream);
 
 /*
+ * Draft-token draw (Algorithm 3: "sample x_1^L, ..., x_K^L ~ p i.i.d."; the draft model produces one position's
+ * logits at a time, so the unit is one token per logit row): token r is drawn from softmax(logits[r]/temperature) by
+ * inverse CDF (ascending vocabulary index, first x whose cumulative mass exceeds u times the total), softmax and
+ * draw fused in one pass over the row.  Device pointers.
+ *   logits      [N,V] (dtype as in sgbv_verify_ex), one row per (batch row, draft) at the position being drafted
+ *   uniforms    [N] float32 in [0,1)
+ *   out_token   [N] int32, -1 for a row with NaN/+inf or without a finite logit
+ *   out_logprob [N] float64 or NULL: log softmax of the drawn token
+ *   out_status  [N] int32 or NULL: SGBV_STATUS_NONFINITE_LOGIT
+ *   workspace   >= sgbv_workspace_bytes(N, 1, 1, V, dtype) bytes, 256-byte aligned, or NULL (library buffer)
+ */
+int sgbv_draw_tokens(const void *logits, int dtype, const float *uniforms, int N, int V, float temperature,
+                     int32_t *out_token, double *out_logprob, int32_t *out_status, void *workspace,
+                     size_t workspace_bytes, void *stream);
+
+/*
  * Allocation-free form of sgbv_verify_ex (the paper has no counterpart: this entry point exists
  * for deployment, not for the method).
  *

@@ -67,6 +67,8 @@ def _load():
         lib.sgbv_oracle_modify.restype = ctypes.c_int
         lib.sgbv_oracle_modify.argtypes = [fp, fp, dp, dp, fp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                            ctypes.c_double, ip, dp, dp, dp, dp, ip, dp]
+        lib.sgbv_oracle_draw_tokens.restype = ctypes.c_int
+        lib.sgbv_oracle_draw_tokens.argtypes = [fp, fp, ctypes.c_int, ctypes.c_int, ctypes.c_double, ip, dp, dp]
         lib.sgbv_oracle_kseq_rho.restype = ctypes.c_double
         lib.sgbv_oracle_kseq_rho.argtypes = [dp, dp, ctypes.c_int, ctypes.c_int]
         lib.sgbv_oracle_kseq_verify.restype = ctypes.c_int
@@ -261,3 +263,17 @@ def kseq_verify(zq, zp, tok, uniforms, temperature: float = 1.0) -> KseqResult:
     if rc < 0:
         raise ValueError("oracle: bad argument")
     return KseqResult(tau, tokens, rho, acc, st, ma, ms)
+
+
+def draw_tokens(z, u, temperature: float = 1.0):
+    """Algorithm 3's draft draw for one position: token r ~ softmax(z[r]/T) by inverse CDF.
+    z [N,V], u [N] -> (tokens int32 [N], log-probabilities [N], margins [N])"""
+    z, u = _f32(z), _f32(u)
+    N, V = z.shape
+    tok = np.empty(N, np.int32)
+    lp, mg = np.empty(N, np.float64), np.empty(N, np.float64)
+    rc = _load().sgbv_oracle_draw_tokens(_p(z, ctypes.c_float), _p(u, ctypes.c_float), N, V, float(temperature),
+                                         _p(tok, ctypes.c_int32), _p(lp, ctypes.c_double), _p(mg, ctypes.c_double))
+    if rc < 0:
+        raise ValueError("oracle: bad argument")
+    return tok, lp, mg

@@ -582,3 +582,33 @@ int sgbv_oracle_kseq_verify(const float *zq, const float *zp, const int32_t *tok
     }
     return 1;
 }
+
+/* ============================================================================================== */
+/* Algorithm 3's draft draw, one position: token r ~ softmax(z[r]/T) by the inverse CDF of step 6.  */
+/*   z [N,V]; u [N]; out_token [N] (-1 for a row with NaN/+inf or no finite logit); out_logp [N]    */
+/*   (log softmax of the drawn token) and out_margin [N] may be NULL.                               */
+int sgbv_oracle_draw_tokens(const float *z, const float *u, int N, int V, double T, int32_t *out_token,
+                            double *out_logp, double *out_margin) {
+    if (N < 0 || V < 1 || !(T > 0.0) || !isfinite(T)) return -1;
+    double *prob = (double *)malloc((size_t)V * sizeof(double));
+    for (int r = 0; r < N; ++r) {
+        const float *row = z + (size_t)r * V;
+        int any = 0, bad = 0;
+        for (int x = 0; x < V; ++x) {
+            bad |= isnan(row[x]) || row[x] == INFINITY;
+            any |= isfinite(row[x]);
+        }
+        double margin = 0.0, lp = NAN;
+        int32_t y = -1;
+        if (!bad && any) {
+            double lse = sgbv_oracle_softmax(row, V, T, prob);
+            y = sgbv_oracle_sample(prob, V, (double)u[r], &margin);
+            lp = (double)row[y] / T - lse;
+        }
+        out_token[r] = y;
+        if (out_logp) out_logp[r] = lp;
+        if (out_margin) out_margin[r] = margin;
+    }
+    free(prob);
+    return 1;
+}

@@ -27,7 +27,7 @@ EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_veri
            "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_last_main_kernel", "sgbv_status_string",
            "sgbv_profile_begin",
            "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option", "sgbv_modify", "sgbv_verify_kseq",
-           "sgbv_verify_token", "sgbv_verify_gbv")
+           "sgbv_verify_token", "sgbv_verify_gbv", "sgbv_draw_tokens")
 
 _lib = None
 
@@ -73,6 +73,8 @@ def load() -> ctypes.CDLL:
         for fn in (lib.sgbv_verify_token, lib.sgbv_verify_gbv):
             fn.restype = i32
             fn.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]
+        lib.sgbv_draw_tokens.restype = i32
+        lib.sgbv_draw_tokens.argtypes = [vp, i32, vp, i32, i32, f32, vp, vp, vp, vp, sz, vp]
         lib.sgbv_last_launch_count.restype = i32
         lib.sgbv_last_launch_count.argtypes = []
         lib.sgbv_last_main_kernel.restype = ctypes.c_char_p
@@ -377,3 +379,24 @@ def sgbv_verify_token(target_logits, draft_logits, draft_tokens, uniforms, tempe
 def sgbv_verify_gbv(target_logits, draft_logits, draft_tokens, uniforms, temperature: float = 1.0) -> PositionwiseOutput:
     """Single-draft greedy block verification (the block verifier with K = 1)."""
     return _single_draft("sgbv_verify_gbv", target_logits, draft_logits, draft_tokens, uniforms, temperature)
+
+
+def sgbv_draw_tokens(logits, uniforms, temperature: float = 1.0):
+    """One token per row of logits [N,V] from softmax(logits/T) by inverse CDF. -> (tokens int32 [N], logprob float64 [N],
+    status int32 [N])"""
+    N, V = logits.shape
+    if tuple(uniforms.shape) != (N,) or uniforms.dtype != torch.float32 or not (logits.is_cuda and uniforms.is_cuda):
+        raise ValueError("uniforms must be float32 [N] on the device of the logits")
+    if not logits.is_contiguous():
+        raise ValueError("logits must be contiguous")
+    dev = logits.device
+    tok = torch.empty(N, dtype=torch.int32, device=dev)
+    lp = torch.empty(N, dtype=torch.float64, device=dev)
+    st = torch.empty(N, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = load().sgbv_draw_tokens(logits.data_ptr(), _dtype_code(logits), uniforms.data_ptr(), N, V, float(temperature),
+                                     tok.data_ptr(), lp.data_ptr(), st.data_ptr(), None, 0,
+                                     torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return tok, lp, st

@@ -463,6 +463,39 @@ int sgbv_verify_gbv(const void *target_logits, const void *draft_logits, int dty
                          out_status, (cudaStream_t)stream);
 }
 
+int sgbv_draw_tokens(const void *logits, int dtype, const float *uniforms, int N, int V, float temperature,
+                     int32_t *out_token, double *out_logprob, int32_t *out_status, void *workspace, size_t workspace_bytes,
+                     void *stream) {
+    if (!logits || !uniforms || !out_token) return SGBV_ERR_NULL;
+    int rc = check_shape(N, 1, 1, V, dtype);
+    if (rc != SGBV_OK) return rc;
+    if (!(temperature > 0.0f) || !isfinite(temperature)) return SGBV_ERR_TEMPERATURE;
+    const size_t esz = dtype == SGBV_DTYPE_BF16 ? 2 : 4;
+    if (((uintptr_t)logits % esz) || ((uintptr_t)uniforms % 4) || ((uintptr_t)out_token % 4) || ((uintptr_t)out_logprob % 8) ||
+        ((uintptr_t)out_status % 4))
+        return SGBV_ERR_ALIGN;
+    const Shape s = make_shape(N, 1, 1, V, temperature);
+    const Carve c = carve(s);
+    unsigned char *base = nullptr;
+    if (workspace) {
+        if (workspace_bytes < c.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
+        base = (unsigned char *)workspace;
+    } else {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SGBV_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_mu);
+        rc = grow(&g_buf[dev].scratch, &g_buf[dev].scratch_bytes, c.total, kRatioWords * sizeof(double));
+        if (rc != SGBV_OK) return rc;
+        base = (unsigned char *)g_buf[dev].scratch;
+    }
+    const int n = launch_draw_rows(logits, dtype, uniforms, s, (float *)(base + c.bonus), out_token, out_logprob, out_status,
+                                   (cudaStream_t)stream);
+    if (n < 0) return n;
+    t_last_launches = n;
+    t_last_kernel = "draw_rows_kernel";
+    return SGBV_OK;
+}
+
 int sgbv_last_launch_count(void) { return t_last_launches; }
 
 const char *sgbv_last_main_kernel(void) { return t_last_kernel; }

@@ -185,6 +185,9 @@ int launch_modify_finish(const Launch &L, const float *u, int32_t *out_token, do
                          double *out_resmass, int32_t *out_status);
 // K-SEQ / token-level verification, one CTA per batch row; tile_scratch: [B][2][ntiles] floats
 int launch_kseq(const Launch &L, float *tile_scratch, double *out_rho, double *out_acc, int32_t *out_status);
+// one token per row of z [s.B, s.V] from softmax(z/T) by inverse CDF; tile_scratch: [s.B][2][ntiles] floats
+int launch_draw_rows(const void *z, int dtype, const float *u, const Shape &s, float *tile_scratch, int32_t *out_token,
+                     double *out_logp, int32_t *out_status, cudaStream_t stream);
 bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0

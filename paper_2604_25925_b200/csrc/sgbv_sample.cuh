@@ -177,10 +177,12 @@ __device__ __forceinline__ void load_tile_pieces<uint16_t>(const uint16_t *zq, i
 // One token from softmax(zq/T) of a single row in one pass over memory: every tile's maximum and its sum of
 // exponentials relative to that maximum, then the row maximum, the factors that move the tile sums to it, the
 // tile search and the pick inside the tile.  tile_s, tile_m: ntiles floats each (shared or global scratch).
-// Returns the token, or -1 with `bad` set if the row holds NaN/+inf or no finite logit.  All threads must call.
+// Returns the token, or -1 with `bad` set if the row holds NaN/+inf or no finite logit; row_max_out (optional)
+// receives the row maximum.  On return tile_s[t] * tile_m[t] is tile t's sum of exponentials relative to the row
+// maximum.  All threads must call.
 template <typename T>
 __device__ int draw_from_row(const T *zq, const Shape &s, double us, float *tile_s, float *tile_m, SampleScratch *sc,
-                             bool &bad_out) {
+                             bool &bad_out, float *row_max_out = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads / 32;
     bool bad = false;
@@ -246,6 +248,7 @@ __device__ int draw_from_row(const T *zq, const Shape &s, double us, float *tile
         return -1;
     }
     bad_out = false;
+    if (row_max_out) *row_max_out = m;
     // tile_m becomes the factor exp((m_t - m)/T) of its tile
     for (int t = tid; t < s.ntiles; t += nthreads) tile_m[t] = (tile_m[t] > -INFINITY) ? expo(tile_m[t], m, s.scale) : 0.0f;
     __syncthreads();

@@ -148,3 +148,28 @@ def test_single_draft_entry_points():
                              inp.uniforms.cpu().numpy(), cfg.temperature)
     ok = (ref.margin_accept >= 1e-6) & (ref.margin_sample >= 1e-6)
     assert (sd.accept_len.cpu().numpy()[ok] == ref.tau[ok]).all()
+
+
+@pytest.mark.parametrize("N,V,dtype,T", [(9, 4099, "fp32", 0.8), (64, 32000, "fp32", 1.0), (33, 128256, "bf16", 0.7),
+                                        (3, 17, "fp32", 1.0), (300, 9000, "bf16", 0.4)])
+def test_draft_token_draw_matches_the_oracle(N, V, dtype, T):
+    cfg = workloads.VerifyConfig("dr", B=N, K=1, gamma=1, V=V, dtype=dtype, temperature=T, alpha=0.8, seed=40 + V % 89)
+    _, zp = _position_rows(cfg)
+    g = torch.Generator().manual_seed(N)
+    u = torch.rand(N, generator=g, dtype=torch.float32).cuda()
+    tok, lp, st = binding.sgbv_draw_tokens(zp, u, T)
+    torch.cuda.synchronize()
+    rtok, rlp, margin = oracle.draw_tokens(zp.float().cpu().numpy(), u.cpu().numpy(), T)
+    near = margin < 1e-6
+    assert near.sum() <= max(2, N // 3) and (st.cpu().numpy() == 0).all()
+    tok = tok.cpu().numpy()
+    assert (tok[~near] == rtok[~near]).all()
+    same = tok == rtok
+    np.testing.assert_allclose(lp.cpu().numpy()[same], rlp[same], atol=2e-5)
+    assert binding.last_main_kernel() == "draw_rows_kernel"
+    # the draws feed the verify step as draft tokens: in range, and a flagged row for a NaN logit
+    assert ((tok >= 0) & (tok < V)).all()
+    zbad = zp.clone()
+    zbad[0, 3] = float("nan")
+    tok2, _, st2 = binding.sgbv_draw_tokens(zbad, u, T)
+    assert tok2[0].item() == -1 and st2[0].item() & binding.STATUS_NONFINITE_LOGIT

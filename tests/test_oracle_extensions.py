@@ -157,3 +157,23 @@ def test_kseq_keeps_the_drafts_that_match_and_stops_at_the_first_position_withou
     tok[0, :, 1] = [1, 2, 4]
     res = oracle.kseq_verify(zq, zp, tok, u)
     assert res.tau[0] == 1 and res.tokens[0, 0] == 1 and res.tokens[0, 1] in (0, 3) and res.tokens[0, 2] == -1
+
+
+# ---- Algorithm 3's draft draw -------------------------------------------------------------------------------
+def test_draw_tokens_follow_the_softmax_law_on_a_grid_of_uniforms():
+    """Inverse CDF: of N equally spaced uniforms exactly the share p(x) (up to one grid point per cell edge) maps to
+    token x, tokens come out in non-decreasing order, and the reported log-probability is log softmax."""
+    rng = np.random.default_rng(11)
+    V, N, T = 13, 4000, 0.7
+    row = (2.0 * rng.standard_normal(V)).astype(np.float32)
+    row[4] = -np.inf
+    p = np_softmax(row, T)
+    u = ((np.arange(N) + 0.5) / N).astype(np.float32)
+    tok, lp, _ = oracle.draw_tokens(np.repeat(row[None], N, 0), u, T)
+    assert (np.diff(tok) >= 0).all() and (tok != 4).all()
+    counts = np.bincount(tok, minlength=V)
+    assert np.abs(counts - p * N).max() <= 1.0 + 1e-6
+    np.testing.assert_allclose(lp, np.log(p[tok]), atol=1e-12)
+    bad = row.copy()
+    bad[2] = np.nan
+    assert oracle.draw_tokens(bad[None], u[:1], T)[0][0] == -1
