@@ -318,6 +318,49 @@ def block_facts(wl):
     return n_bonus, be
 
 
+def compare_verifiers(dev):
+    """Verification cost of the four verifiers behind the boundary on the paper's operating points (K = 3 drafts of
+    L = 12 or 8 tokens, T = 0.4, 32k vocabulary): one prompt and a batch of 64, microseconds per verify call and
+    block efficiency.  The single-draft methods (token-level speculative sampling, GBV) see the first draft only."""
+    import torch
+    from paper_2604_25925_b200 import binding, workloads
+    rows = []
+    for name in ("paper_l12", "paper_l8"):
+        for B in (1, 64):
+            cfg = workloads.with_batch(workloads.CONFIGS[name], B)
+            nsets = 8 if B == 1 else 4
+            sets = [workloads.make_inputs(cfg, device=dev, set_index=500 + i) for i in range(nsets)]
+            single = [(i.target_logits[:, 0].contiguous(), i.draft_logits[:, 0].contiguous(),
+                       i.draft_tokens[:, 0].contiguous(), i.uniforms[:, :cfg.gamma + 1].contiguous()) for i in sets]
+            T = cfg.temperature
+            methods = {
+                "spectr_gbv": lambda j: binding.sgbv_verify(sets[j].target_logits, sets[j].draft_logits,
+                                                            sets[j].draft_tokens, sets[j].uniforms, T).accept_len,
+                "spectr_kseq": lambda j: binding.sgbv_verify_kseq(sets[j].target_logits, sets[j].draft_logits,
+                                                                  sets[j].draft_tokens, sets[j].uniforms, T).accept_len,
+                "gbv_single_draft": lambda j: binding.sgbv_verify_gbv(*single[j], T).accept_len,
+                "token_level_sd": lambda j: binding.sgbv_verify_token(*single[j], T).accept_len,
+            }
+            entry = {"workload": describe(cfg)}
+            for mname, fn in methods.items():
+                for j in range(nsets):
+                    fn(j)
+                torch.cuda.synchronize()
+                reps = 40
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for r in range(reps):
+                    fn(r % nsets)
+                e1.record()
+                torch.cuda.synchronize()
+                be = float(sum(float((fn(j).float() + 1).mean().item()) for j in range(nsets))) / nsets
+                entry[mname] = {"us_per_verify": 1e3 * e0.elapsed_time(e1) / reps, "block_efficiency": be}
+            rows.append(entry)
+            del sets, single
+            torch.cuda.empty_cache()
+    return rows
+
+
 PER_CONFIG = ("c2", "c3", "c5_K1_a0.8_T1.0", "c5_K8_a0.8_T1.0")
 
 
@@ -436,6 +479,7 @@ def main():
                 del w
                 torch.cuda.empty_cache()
             line["per_config"] = per
+            line["verifier_comparison"] = compare_verifiers(dev)
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

@@ -15,8 +15,8 @@
  *   draft_tokens  [B, K, gamma]        int32, token i of draft k, 0 <= token < V
  *   uniforms      [B, K*gamma + 1]     float32 in [0,1): entry k*gamma + (i-1) is the uniform eta of
  *                                      the Bernoulli trial on the length-i sub-block of draft k
- *                                      (Algorithm 1, lines "sample eta ~ U(0,1)"); the last entry
- *                                      draws the extra token by inverse CDF
+ *                                      in Algorithm 1; the last entry draws the extra token by
+ *                                      inverse CDF
  *   out_accept_len [B]                 int32 tau in 0..gamma, or -1 if the row was flagged invalid
  *   out_draft_idx  [B]                 int32 accepted draft f in 0..K-1, -1 when tau == 0
  *   out_tokens     [B, gamma+1]        int32: the tau accepted tokens, then the extra token y at
@@ -69,8 +69,10 @@ int sgbv_workspace_bytes(int B, int K, int gamma, int V, int dtype, size_t *out_
  * library grows with cudaMalloc when a larger shape is first seen (so the first call of a
  * shape is not stream-capturable; later ones allocate nothing).  Calls that use that buffer on
  * one device must be ordered with respect to one another (one stream, or events between streams):
- * they share it, and between two such calls of the same shape the library keeps part of it
- * prepared for the next call.  The kernels are launched with programmatic stream serialisation:
+ * they share it, and every call leaves part of it prepared for the next one (whatever their
+ * shapes, eager or replayed from a CUDA graph).  A CUDA graph captured on that buffer holds its
+ * address: a later call of a larger shape reallocates the buffer and invalidates such graphs, so
+ * call the largest shape first, or pass a workspace of your own to sgbv_verify_ex.  The kernels are launched with programmatic stream serialisation:
  * for batches of at most 16 rows the first kernel of a call may be scheduled while the kernel
  * ahead of it in the stream is still running; it touches no global memory until that kernel has
  * completed, so the caller sees ordinary stream order.
@@ -106,7 +108,9 @@ int sgbv_verify_ex(const void *target_logits, const void *draft_logits, int dtyp
  * Host-buffer form: every tensor pointer is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies the inputs to device staging buffers owned by the library, runs the
  * verify step on `stream`, copies the three outputs (and out_status if not NULL) back and
- * synchronises the stream before returning.
+ * synchronises the stream before returning.  All calls on one device share one staging buffer
+ * (grown with cudaMalloc when a larger shape is first seen): callers on the same device must be
+ * serialised with respect to one another.
  */
 int sgbv_verify_host(const void *target_logits, const void *draft_logits, int dtype,
                      const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma,
@@ -203,7 +207,11 @@ int sgbv_draw_tokens(const void *logits, int dtype, const float *uniforms, int N
  * and nothing is launched.
  *
  * First call on a device: resolves the array's device address (once per device, with that
- * device current).  Make that first call before starting any stream capture.
+ * device current); with CUDA's lazy module loading this is also when the driver loads the part of
+ * the library that holds the array and reserves its bytes, and the first launch of each kernel
+ * variant (shape, dtype, K) loads its code the same way.  So make one small call per variant that
+ * will be used at start-up: before the caller's pool takes the rest of the device memory, and
+ * before starting any stream capture.
  *
  * Sharing: all calls on a device use the same array, and it keeps the previous call's contents;
  * the call clears what has to start at zero itself.  Two calls that overlap on the GPU (different
@@ -238,11 +246,12 @@ int sgbv_profile_end(double *out_total_ms, int *out_records);
 /*
  * Tuning knobs for experiments (process-wide, not thread-safe; 0 restores the automatic choice):
  *   "path"         1 = always the generic two-sweep kernels, 2 = the fused single-read kernel or fail
- *   "cluster"      CTAs per cluster of the fused kernel (1, 2, 4, 8 or 16)
- *   "stages"       depth of its shared-memory ring (2..12)
+ *   "cluster"      CTAs per cluster of the fused kernel (1..8)
  *   "max_clusters" cap on the number of resident clusters it launches
  *   "walk"         1 = a cluster of the fused kernel walks whole draft chains, 2 = single rows
- *   "occupancy"    CTAs of the fused kernel per SM (2, 3 or 4; more CTAs hold fewer cells each)
+ * and two for the failure-detection test (a bounded device-side wait that runs out, see SGBV_STATUS_TIMEOUT):
+ *   "poll_us"      limit, in microseconds, of the row walk's wait for a ratio published by another cluster
+ *   "withhold"     1 = the first row of every chain does not publish its ratio
  * Returns SGBV_ERR_SHAPE for an unknown name or a value out of range.
  */
 int sgbv_set_option(const char *name, int value);
