@@ -41,9 +41,9 @@ constexpr int kMaxWarps = 32;              // warps per CTA: 32 (64 registers ea
 constexpr int kCell = kTile;               // 256 contiguous entries: the unit a warp works on
 constexpr int kCtasPerSm = 1;              // CTAs that share an SM (1 or 2): two are in different phases of their rows
                                            // most of the time, so that one's exponentials overlap the other's sums
-constexpr int kWarps = 32 / kCtasPerSm;    // warps per CTA
-constexpr int kCtaCells = 4 * kWarps;      // cells of a row per CTA (four per warp); 16 tensor-memory columns per cell in
-                                           // each of the 4 lane quarters: 128 cells = 32,768 entries per SM
+constexpr int kWarps = 32;                 // warps per CTA (16 warps of 128 registers measured a third slower)
+constexpr int kCtaCells = 128 / kCtasPerSm;  // cells of a row per CTA: 16 tensor-memory columns per cell in each of the 4
+                                           // lane quarters, 512 columns per SM: 128 cells = 32,768 entries per SM
 constexpr int kTmemCols = 512 / kCtasPerSm;  // this CTA's share of the SM's tensor memory
 constexpr int kMaxCluster = 8 * kCtasPerSm;  // CTAs per cluster (beyond 8 the size is not portable, which sm_100 allows)
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second of SM clock
@@ -874,7 +874,7 @@ std::mutex g_plan_mu;      // guards the options and the per-device caches below
 constexpr int kCtaSlots = 148 * kCtasPerSm;  // CTAs the device holds
 // ring slots per warp: half a row's cells for float32 (128 KB of copies under way per SM), all of them for bfloat16
 template <typename T>
-constexpr int slots_for() { return sizeof(T) == 4 ? 2 : 4; }
+constexpr int slots_for() { return (sizeof(T) == 4 ? 2 : 4) * 32 / kWarps / kCtasPerSm; }
 template <typename T>
 constexpr size_t smem_bytes() {
     return (size_t)kWarps * slots_for<T>() * (2 * kCell * sizeof(T) + 8) + (size_t)(kCtaCells / kWarps) * kWarps * 32 * 4 + sizeof(Control);
