@@ -38,7 +38,7 @@ Shape make_shape(int B, int K, int gamma, int V, float temperature) {
 }
 
 struct Carve {
-    size_t rows, part, wpart, dpart, mpart, ratio, bonus, h, resmass, status, error, total;
+    size_t rows, part, wpart, dpart, mpart, ratio, cut, bonus, h, resmass, status, error, total;
 };
 
 Carve carve(const Shape &s) {
@@ -53,6 +53,7 @@ Carve carve(const Shape &s) {
     c.wpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.dpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
     c.mpart = off;     off += align_up(NR * s.ntiles * sizeof(float));
+    c.cut = off;       off += align_up((size_t)s.B * s.cpr * sizeof(double));
     c.bonus = off;     off += align_up((size_t)s.B * 2 * s.ntiles * sizeof(float));
     c.h = off;         off += align_up(NR * sizeof(double));
     c.resmass = off;   off += align_up(NR * sizeof(double));
@@ -164,6 +165,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     L.ws.dpart = (float *)(base + c.dpart);
     L.ws.mpart = (float *)(base + c.mpart);
     L.ws.ratio = (double *)(base + c.ratio);
+    L.ws.cut = (double *)(base + c.cut);
     L.ws.bonus = (float *)(base + c.bonus);
     L.ws.h = out_h ? out_h : (double *)(base + c.h);
     L.ws.resmass = out_resmass ? out_resmass : (double *)(base + c.resmass);
@@ -347,6 +349,7 @@ int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, 
     L.ws.dpart = (float *)(base + c.dpart);
     L.ws.mpart = (float *)(base + c.mpart);
     L.ws.ratio = (double *)(base + c.ratio);
+    L.ws.cut = (double *)(base + c.cut);
     L.ws.ratio_used = 0;  // (a single position per chain never takes the row walk)
     L.ws.bonus = (float *)(base + c.bonus);
     L.ws.bonus_in_smem = 0;

@@ -44,6 +44,8 @@ struct Workspace {
     double *ratio;      // [kRatioWords]: p_i(tok_i)/q_i(tok_i) of each row (row walk of the fused kernel, which
                         // only runs when B*K*gamma <= kRatioWords); every word holds a NaN pattern ("not
                         // published yet") whenever no call is in flight
+    double *cut;        // [B*cpr]: c handed from the cluster that walks the head of a chain to the one that walks its tail
+                        // (chain walk of the fused kernel; preset to the NaN pattern when any range cuts a chain)
     int ratio_used;     // the streaming kernel walked rows: the finishing kernel puts the NaN pattern back
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory

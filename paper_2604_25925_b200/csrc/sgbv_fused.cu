@@ -495,18 +495,56 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     if (!kRow) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (blockIdx.x == 0 && tid == 0) *p.error_flag = 0;  // set again only by a wait that expires (about a second later)
     // The walk of this cluster: position n = 0, 1, ... is row (bk, i).
-    //   chain mode: chains cid, cid+G, ... each from i = 0 to gamma-1 (c_i is carried along the chain);
-    //   row mode:   rows u = cid, cid+G, ... of the list of all rows, u = bk*gamma + i.  Used when there
-    //               are few chains: all rows of a chain then run at the same time on different clusters,
-    //               and c_i comes from the ratios p_j(tok_j)/q_j(tok_j) that the clusters of rows j < i
-    //               publish in global memory.  A row only waits for rows earlier in the list, which are
-    //               walked no later by clusters that are all resident, so every wait ends.
-    // One step of the walk: bk += step_bk, i += step_i, and on i >= gamma: i -= gamma, bk += wrap_bk.
+    //   chain mode: the list of all rows, u = bk*gamma + i, is cut into G contiguous ranges of equal length (+-1), one
+    //               per cluster, so that the clusters finish together whatever the number of chains.  A range may
+    //               begin and end inside a chain.  The cluster walks first the HEAD of the chain its range ends in
+    //               (rows 0..off_hi-1 of chain_hi) and leaves the ratio c reached there in a word of global memory,
+    //               then its whole chains, and last the TAIL of the chain its range begins in (rows off_lo.. of
+    //               chain_lo), whose c it picks up from the word the cluster before it wrote at its very start.  The
+    //               words are preset to a NaN pattern; the one wait (bounded) is for something written long before.
+    //   row mode:   rows u = cid, cid+G, ... of the list.  Used when there are few rows: all rows of a chain then run
+    //               at the same time on different clusters, and c_i comes from the ratios p_j(tok_j)/q_j(tok_j) that
+    //               the clusters of rows j < i publish in global memory.  A row only waits for rows earlier in the
+    //               list, which are walked no later by clusters that are all resident, so every wait ends.
     constexpr bool row_mode = kRow;
-    const int step_bk = row_mode ? G / s.gamma : 0, step_i = row_mode ? G % s.gamma : 1, wrap_bk = row_mode ? 1 : G;
     const long total_rows = (long)p.nchains * s.gamma;
-    const int nrows = row_mode ? (int)((total_rows - cid + G - 1) / G)
-                               : ((p.nchains - cid + G - 1) / G) * s.gamma;  // rows this cluster walks
+    const long range_lo = row_mode ? 0 : total_rows * cid / G, range_hi = row_mode ? 0 : total_rows * (cid + 1) / G;
+    const int chain_lo = (int)(range_lo / s.gamma), off_lo = (int)(range_lo % s.gamma);
+    const int chain_hi = (int)(range_hi / s.gamma), off_hi = (int)(range_hi % s.gamma);
+    const int chain_mid = chain_lo + (off_lo > 0 ? 1 : 0);  // first whole chain of the range
+    const int nrows = row_mode ? (int)((total_rows - cid + G - 1) / G) : (int)(range_hi - range_lo);  // rows this cluster walks
+    // the row after (bk, i) in this cluster's walk
+    auto walk_next = [&](int &bk, int &i) {
+        if (row_mode) {
+            bk += G / s.gamma;
+            i += G % s.gamma;
+            if (i >= s.gamma) {
+                i -= s.gamma;
+                ++bk;
+            }
+            return;
+        }
+        ++i;
+        if (bk == chain_hi) {  // in the head
+            if (i >= off_hi) {
+                if (chain_mid < chain_hi) {
+                    bk = chain_mid;
+                    i = 0;
+                } else {
+                    bk = chain_lo;
+                    i = off_lo;
+                }
+            }
+        } else if (i >= s.gamma && !(bk == chain_lo && off_lo > 0)) {  // a whole chain is done (the tail is the last segment)
+            if (bk + 1 < chain_hi) {
+                ++bk;
+                i = 0;
+            } else {
+                bk = chain_lo;
+                i = off_lo;
+            }
+        }
+    };
     const uint32_t xbytes = (uint32_t)(C * sizeof(float4));  // one partial from every CTA of the cluster
     uint32_t timed_out = 0;
 
@@ -554,7 +592,7 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     // rows of the walk: A = the row whose second sweep runs, B = the one after it, whose first sweep runs in the
     // same loop, D = the one after B, whose cells are requested meanwhile
     int bk_a = 0, i_a = 0;  // (set when B becomes A)
-    int bk_b = row_mode ? cid / s.gamma : cid;
+    int bk_b = row_mode ? cid / s.gamma : (off_hi > 0 ? chain_hi : chain_mid);  // (a range of gamma rows or more has one of them)
     int i_b = row_mode ? cid % s.gamma : 0;
     const unsigned char *q_b = zq_warp + ((size_t)bk_b * s.zq_rows + i_b) * row_bytes;  // this warp's first cell of row B
     const unsigned char *p_b = zp_warp + ((size_t)bk_b * s.gamma + i_b) * row_bytes;
@@ -583,11 +621,8 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
     for (int n = -1; n < nrows; ++n) {
         const bool has_a = n >= 0, has_b = n + 1 < nrows;
         // row D, the one after B
-        int bk_d = bk_b + step_bk, i_d = i_b + step_i;
-        if (i_d >= s.gamma) {
-            i_d -= s.gamma;
-            bk_d += wrap_bk;
-        }
+        int bk_d = bk_b, i_d = i_b;
+        walk_next(bk_d, i_d);
         const bool has_d = n + 2 < nrows;
         const bool more = has_d && !timed_out;
         const unsigned char *q_d = zq_warp + ((size_t)bk_d * s.zq_rows + i_d) * row_bytes;
@@ -803,7 +838,31 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
             bar_arrive(2, kFThreads);
             // off the critical path: c of the next row of the chain walk (c_{i+1} = c_i ratio, and 1 at the start of
             // the next chain), and the row's record for the finishing kernel
-            if (!row_mode) c_carry = (i_b + 1 < s.gamma) ? cd * SGBV_RATIO() : (has_d ? SGBV_C0(bk_d) : 1.0);
+            if (!row_mode) {
+                const double c_next = cd * SGBV_RATIO();  // c after this row
+                // the head of a chain that another cluster continues: leave c where that cluster looks for it
+                if (bk_b == chain_hi && i_b == off_hi - 1 && lane == 0 && rank == 0)
+                    *reinterpret_cast<volatile double *>(p.ws.cut + bk_b) = (c_next != c_next) ? 0.0 : c_next;
+                if (has_d) {
+                    if (i_d == 0) {
+                        c_carry = SGBV_C0(bk_d);
+                    } else if (bk_d == bk_b) {
+                        c_carry = c_next;
+                    } else {  // the tail of a chain whose head another cluster walked at its very start
+                        const volatile double *word = reinterpret_cast<const volatile double *>(p.ws.cut + bk_d);
+                        double w = *word;
+                        if (w != w && !timed_out) {
+                            const long long t0 = clock64();
+                            while ((w = *word) != w)
+                                if (clock64() - t0 > kWaitLimitCycles) {
+                                    timed_out = 1;
+                                    break;
+                                }
+                        }
+                        c_carry = (w != w) ? 0.0 : w;
+                    }
+                }
+            }
             if (lane == 0 && rank == 0) {
                 // nonfinite logits: NaN poisons Z, +inf shows up as an infinite maximum, a row of
                 // -inf only has Z = 0
@@ -954,6 +1013,9 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
     cfg.attrs = attr;
     cfg.numAttrs = L.s.B <= kChainedLaunchMaxB ? 2 : 1;  // small batches only: see kChainedLaunchMaxB
     cfg.gridDim = dim3(clusters * plan.cluster);
+    if (!kRow && (fp.nchains % clusters) != 0 &&  // some ranges begin or end inside a chain: their hand-over words
+        cudaMemsetAsync(L.ws.cut, 0xff, (size_t)fp.nchains * sizeof(double), L.stream) != cudaSuccess)
+        return SGBV_ERR_CUDA;
     if (kRow && !L.ratio_preset &&
         cudaMemsetAsync(L.ws.ratio, 0xff, (size_t)fp.nchains * L.s.gamma * sizeof(double), L.stream) != cudaSuccess)
         return SGBV_ERR_CUDA;

@@ -151,6 +151,27 @@ def test_draft_counts_without_a_specialised_kernel(K, dtype):
     assert binding.last_main_kernel() == "fused_chain_kernel"
 
 
+@pytest.mark.parametrize("B,K,gamma,V,dtype", [(50, 3, 4, 2048, "fp32"), (75, 2, 7, 4096, "bf16"), (149, 1, 5, 1024, "fp32"),
+                                              (33, 4, 6, 40000, "fp32")])
+def test_chains_cut_between_clusters(B, K, gamma, V, dtype):
+    """The chain walk gives every cluster an equal share of the rows, so with a chain count that is no multiple of the
+    clusters most chains begin on one cluster and end on another (the ratio c is handed over through global memory).
+    Every batch row is compared."""
+    cfg = workloads.VerifyConfig(f"cut_{B}_{K}_{gamma}", B=B, K=K, gamma=gamma, V=V, dtype=dtype, temperature=0.9,
+                                 alpha=0.85, seed=700 + B)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    rep, _, _ = run_both(inp)
+    assert_parity(rep)
+    assert binding.last_main_kernel() == "fused_chain_kernel"
+    binding.set_option("walk", 1)            # and with the chain walk forced where the row walk would be chosen
+    try:
+        small = workloads.VerifyConfig("cut_small", B=7, K=3, gamma=5, V=3000, dtype=dtype, temperature=0.8, seed=701)
+        rep, _, _ = run_both(workloads.make_inputs(small, device="cuda"))
+        assert_parity(rep)
+    finally:
+        binding.set_option("walk", 0)
+
+
 EDGE_SHAPES = [
     # B, K, gamma, V
     (3, 1, 1, 1), (2, 2, 3, 7), (5, 3, 2, 1000), (2, 2, 2, 1025), (2, 4, 3, 32001), (1, 1, 1, 5000),
