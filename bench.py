@@ -374,6 +374,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--sweep-c5", action="store_true",
+                    help="instead of the default line: the 24 points of the B=256, gamma=4, V=32000 sweep, one JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 3
@@ -394,6 +396,30 @@ def main():
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.sweep_c5:
+        if world > 1:
+            raise RuntimeError("--sweep-c5 runs on one GPU")
+        points = []
+        for c in workloads.sweep_c5():
+            w = Workload(c, dev, rank)
+            c_steps = int(max(20, min(2000, 50.0 / max(0.02, c.logit_bytes() / 4.0e9))))
+            bl, _, _ = timed_blocks(w, c_steps, max(3, c_steps // 4), 1, min_seconds=0.3)
+            k_ms, k_n = kernel_pass(w, max(20, min(c_steps, 100)))
+            nb, c_be = block_facts(w)
+            c_ab = algorithmic_bytes(c, nb)
+            msb = sorted(bl)[len(bl) // 2]
+            r = roofline_of(w, c_ab, k_ms, k_n)
+            points.append({"workload": describe(c), "K": c.K, "alpha": c.alpha, "temperature": c.temperature,
+                           "value": c_steps / (msb * 1e-3), "ms_per_step": msb / c_steps, "block_efficiency": c_be,
+                           "hbm_gbs_step": c_ab["step"] / (msb / c_steps * 1e-3) / 1e9, "kernel_gbs": r["achieved"],
+                           "frac": r["frac"], "launches_timed": k_n})
+            del w
+            torch.cuda.empty_cache()
+        print(json.dumps({"metric": "verify_steps_per_s", "unit": "verify-steps/s", "n_gpus": 1, "data": "synthetic",
+                          "config": {"workload": "c5 sweep: B=256, gamma=4, V=32000, fp32, K x alpha x temperature"},
+                          "points": points}))
+        return
 
     cfg = workloads.get_config(args.workload)
     est_ms = max(0.02, cfg.logit_bytes() / 4.0e9)             # rough step time for choosing defaults
