@@ -361,6 +361,62 @@ def compare_verifiers(dev):
     return rows
 
 
+def vocab_sharded_leg(dev, n_ranks=8):
+    """The vocabulary-sharded form of the step on C4's shape split over `n_ranks` ranges: one rank's four local
+    phases timed on this device (every rank does the same amount of work; the three exchanges between the phases
+    move the byte counts listed and are not timed here, there being one GPU)."""
+    import torch
+    from paper_2604_25925_b200 import binding, sharded, workloads
+    cfg = workloads.get_config("c4")
+    inp = workloads.make_inputs(cfg, device=dev, set_index=700)
+    bounds = sharded.shard_bounds(cfg.V, n_ranks)
+    shards = [(inp.target_logits[..., lo:hi].contiguous(), inp.draft_logits[..., lo:hi].contiguous(), lo)
+              for lo, hi in bounds]
+    one = binding.sgbv_verify(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, cfg.temperature)
+    tok, u, T = inp.draft_tokens, inp.uniforms, cfg.temperature
+    del inp
+    torch.cuda.empty_cache()
+    outs = sharded.verify_all_ranks_on_one_device(shards, tok, u, T, cfg.V)
+    torch.cuda.synchronize()
+    agree = float((outs[0].accept_len == one.accept_len).float().mean().item())
+    same_tokens = float((outs[0].tokens == one.tokens).all(dim=1).float().mean().item())
+    stats_all = torch.stack([binding.sgbv_shard_stats(zq, zp, tok, vb, cfg.V, T) for zq, zp, vb in shards]).contiguous()
+    zq, zp, vb = shards[0]
+    ws = torch.empty(binding.sgbv_shard_workspace_bytes(cfg.B, cfg.K, cfg.gamma, zq.shape[-1]), dtype=torch.uint8, device=dev)
+    wss = [torch.empty_like(ws) for _ in shards]
+    sums_all = torch.stack([binding.sgbv_shard_sums(a, b, T, stats_all, wss[r]) for r, (a, b, _) in enumerate(shards)]).contiguous()
+    phases = {
+        "stats": lambda r: binding.sgbv_shard_stats(shards[r][0], shards[r][1], tok, shards[r][2], cfg.V, T),
+        "sums": lambda r: binding.sgbv_shard_sums(shards[r][0], shards[r][1], T, stats_all, wss[r]),
+        "decide": lambda r: binding.sgbv_shard_decide(tok, u, shards[r][0].shape[-1], T, stats_all, sums_all, wss[r]),
+        "draw": lambda r: binding.sgbv_shard_draw(shards[r][0], shards[r][1], shards[r][2], T, r, wss[r], outs[r].tokens),
+    }
+    shard_bytes = sum(t.numel() * t.element_size() for t in (zq, zp))
+    res = {}
+    for name, fn in phases.items():
+        for r in range(n_ranks):   # warm-up, and the rotation over the ranks' shards keeps the inputs out of L2
+            fn(r)
+        torch.cuda.synchronize()
+        reps = 3 * n_ranks
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i % n_ranks)
+        e1.record()
+        torch.cuda.synchronize()
+        res[name + "_us"] = 1e3 * e0.elapsed_time(e1) / reps
+    total_us = sum(res.values())
+    res.update({
+        "workload": describe(cfg) + f", vocabulary split over {n_ranks} ranks ({zq.shape[-1]} entries each)",
+        "per_rank_us": total_us, "per_rank_shard_bytes": shard_bytes,
+        "per_rank_gbs_over_both_sweeps": 2 * shard_bytes / (total_us * 1e-6) / 1e9,
+        "exchange_bytes": {"stats_all_gather": stats_all.numel() * 4, "sums_all_gather": sums_all.numel() * 8,
+                           "tokens_all_reduce": outs[0].tokens.numel() * 4},
+        "agreement_with_one_device": {"accept_len": agree, "whole_rows": same_tokens},
+        "note": "phases timed on one device over the ranks' shards in turn; exchanges not timed (one GPU)"})
+    return res
+
+
 PER_CONFIG = ("c2", "c3", "c5_K1_a0.8_T1.0", "c5_K8_a0.8_T1.0")
 
 
@@ -506,6 +562,7 @@ def main():
                 torch.cuda.empty_cache()
             line["per_config"] = per
             line["verifier_comparison"] = compare_verifiers(dev)
+            line["vocab_sharded"] = vocab_sharded_leg(dev)
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

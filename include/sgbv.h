@@ -193,6 +193,49 @@ int sgbv_draw_tokens(const void *logits, int dtype, const float *uniforms, int N
                      size_t workspace_bytes, void *stream);
 
 /*
+ * Vocabulary-sharded verify step (no counterpart in the paper, which verifies on one device; the results are those
+ * of Algorithm 1 on the whole vocabulary).  Rank r of n_ranks holds the logits of the vocabulary range
+ * [v_begin_r, v_begin_r + shard_V_r), the ranges ascending with the rank and covering [0,V) without gaps, as a
+ * tensor-parallel output layer leaves them:
+ *   target_shard [B,K,gamma+1,shard_V], draft_shard [B,K,gamma,shard_V] row-major, dtype as in sgbv_verify_ex;
+ * draft_tokens [B,K,gamma] (global ids) and uniforms [B,K*gamma+1] are the same on every rank.  All pointers are
+ * device pointers.  The step is four local calls with three exchanges between them, which the CALLER performs with
+ * its collective library (the Python binding uses torch.distributed); no call waits for another rank:
+ *   sgbv_shard_stats   -> out_stats [B,K,gamma+1,8] float32: per row the shard's (max, sum of exponentials relative
+ *                         to it) of the target and the draft row, the token's two logits if the shard holds it, flags
+ *     exchange 1: all-gather the records in rank order -> stats_all [n_ranks,B,K,gamma+1,8]
+ *   sgbv_shard_sums    -> normalisers and the ratios c_i of Eq. 2 from stats_all (identical on every rank), the
+ *                         vocabulary sums of Eq. 2 and Eq. 4 over the shard; out_sums [B,K,gamma,3] float64
+ *     exchange 2: all-gather -> sums_all [n_ranks,B,K,gamma,3]
+ *   sgbv_shard_decide  -> Eq. 2 / Eq. 3 and the scan of Algorithm 1 from the shards' sums added in rank order:
+ *                         identical out_accept_len, out_draft_idx, out_h, out_resmass, out_status on every rank;
+ *                         out_tokens holds the accepted prefix and -1 elsewhere.  The inverse CDF of the extra token
+ *                         (Eq. 4, or the target row) is split in rank order: which rank's range holds it, and where
+ *                         inside that rank's share of the mass (kept in the workspace)
+ *   sgbv_shard_draw    -> the owning rank finds the token inside its shard and writes its global id into
+ *                         tokens[b, accept_len]; the other ranks leave -1 there
+ *     exchange 3: max-all-reduce of tokens [B,gamma+1]
+ * workspace: >= sgbv_shard_workspace_bytes(B,K,gamma,shard_V,dtype) bytes, 256-byte aligned, the caller's, and the
+ * same buffer for the three calls of a step that take one (it carries the row records, the cell sums and the plan).
+ * The flat parts of stats_all and sums_all must be the ranks' outputs in rank order; n_ranks <= 64.
+ * Return codes as sgbv_verify_ex; per-row status bits as there (a token id outside [0,V), NaN/+inf in any shard).
+ */
+int sgbv_shard_workspace_bytes(int B, int K, int gamma, int shard_V, int dtype, size_t *out_bytes);
+int sgbv_shard_stats(const void *target_shard, const void *draft_shard, int dtype, const int32_t *draft_tokens, int B,
+                     int K, int gamma, int shard_V, int v_begin, int V, float temperature, float *out_stats,
+                     void *stream);
+int sgbv_shard_sums(const void *target_shard, const void *draft_shard, int dtype, int B, int K, int gamma, int shard_V,
+                    float temperature, const float *stats_all, int n_ranks, void *workspace, size_t workspace_bytes,
+                    double *out_sums, void *stream);
+int sgbv_shard_decide(const int32_t *draft_tokens, const float *uniforms, int B, int K, int gamma, int shard_V,
+                      float temperature, const float *stats_all, const double *sums_all, int n_ranks, void *workspace,
+                      size_t workspace_bytes, int32_t *out_accept_len, int32_t *out_draft_idx, int32_t *out_tokens,
+                      double *out_h, double *out_resmass, int32_t *out_status, void *stream);
+int sgbv_shard_draw(const void *target_shard, const void *draft_shard, int dtype, int B, int K, int gamma, int shard_V,
+                    int v_begin, float temperature, int rank, void *workspace, size_t workspace_bytes, int32_t *tokens,
+                    void *stream);
+
+/*
  * Allocation-free form of sgbv_verify_ex (the paper has no counterpart: this entry point exists
  * for deployment, not for the method).
  *

@@ -27,7 +27,8 @@ EXPORTS = ("sgbv_workspace_bytes", "sgbv_verify", "sgbv_verify_bf16", "sgbv_veri
            "sgbv_verify_host", "sgbv_last_launch_count", "sgbv_last_main_kernel", "sgbv_status_string",
            "sgbv_profile_begin",
            "sgbv_profile_end", "sgbv_verify_static", "sgbv_set_option", "sgbv_modify", "sgbv_verify_kseq",
-           "sgbv_verify_token", "sgbv_verify_gbv", "sgbv_draw_tokens")
+           "sgbv_verify_token", "sgbv_verify_gbv", "sgbv_draw_tokens", "sgbv_shard_workspace_bytes",
+           "sgbv_shard_stats", "sgbv_shard_sums", "sgbv_shard_decide", "sgbv_shard_draw")
 
 _lib = None
 
@@ -75,6 +76,16 @@ def load() -> ctypes.CDLL:
             fn.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, f32, vp, vp, vp, vp, vp, sz, vp]
         lib.sgbv_draw_tokens.restype = i32
         lib.sgbv_draw_tokens.argtypes = [vp, i32, vp, i32, i32, f32, vp, vp, vp, vp, sz, vp]
+        lib.sgbv_shard_workspace_bytes.restype = i32
+        lib.sgbv_shard_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(sz)]
+        lib.sgbv_shard_stats.restype = i32
+        lib.sgbv_shard_stats.argtypes = [vp, vp, i32, vp, i32, i32, i32, i32, i32, i32, f32, vp, vp]
+        lib.sgbv_shard_sums.restype = i32
+        lib.sgbv_shard_sums.argtypes = [vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, sz, vp, vp]
+        lib.sgbv_shard_decide.restype = i32
+        lib.sgbv_shard_decide.argtypes = [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, sz, vp, vp, vp, vp, vp, vp, vp]
+        lib.sgbv_shard_draw.restype = i32
+        lib.sgbv_shard_draw.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, f32, i32, vp, sz, vp, vp]
         lib.sgbv_last_launch_count.restype = i32
         lib.sgbv_last_launch_count.argtypes = []
         lib.sgbv_last_main_kernel.restype = ctypes.c_char_p
@@ -400,3 +411,92 @@ def sgbv_draw_tokens(logits, uniforms, temperature: float = 1.0):
     if rc != OK:
         raise SgbvError(rc)
     return tok, lp, st
+
+
+# ---- vocabulary-sharded verify step: the four local phases (the exchanges between them are the caller's) ----------
+
+def _shard_shapes(target_shard, draft_shard):
+    B, K, g1, Vs = target_shard.shape
+    gamma = g1 - 1
+    if tuple(draft_shard.shape) != (B, K, gamma, Vs) or draft_shard.dtype != target_shard.dtype:
+        raise ValueError(f"draft shard must be {(B, K, gamma, Vs)} of the target shard's dtype")
+    if not (target_shard.is_cuda and draft_shard.is_cuda and target_shard.is_contiguous() and draft_shard.is_contiguous()):
+        raise ValueError("shards must be contiguous CUDA tensors")
+    return B, K, gamma, Vs
+
+
+def sgbv_shard_workspace_bytes(B: int, K: int, gamma: int, shard_V: int, dtype: int = DTYPE_F32) -> int:
+    out = ctypes.c_size_t(0)
+    rc = load().sgbv_shard_workspace_bytes(B, K, gamma, shard_V, dtype, ctypes.byref(out))
+    if rc != OK:
+        raise SgbvError(rc)
+    return int(out.value)
+
+
+def sgbv_shard_stats(target_shard, draft_shard, draft_tokens, v_begin: int, V: int, temperature: float) -> torch.Tensor:
+    """-> this shard's statistics records, float32 [B,K,gamma+1,8]."""
+    B, K, gamma, Vs = _shard_shapes(target_shard, draft_shard)
+    dev = target_shard.device
+    out = torch.empty((B, K, gamma + 1, 8), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        rc = load().sgbv_shard_stats(target_shard.data_ptr(), draft_shard.data_ptr(), _dtype_code(target_shard),
+                                     draft_tokens.data_ptr(), B, K, gamma, Vs, int(v_begin), int(V), float(temperature),
+                                     out.data_ptr(), torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_shard_sums(target_shard, draft_shard, temperature: float, stats_all, workspace) -> torch.Tensor:
+    """stats_all: float32 [n_ranks,B,K,gamma+1,8] in rank order. -> this shard's row sums, float64 [B,K,gamma,3]."""
+    B, K, gamma, Vs = _shard_shapes(target_shard, draft_shard)
+    dev = target_shard.device
+    if tuple(stats_all.shape[1:]) != (B, K, gamma + 1, 8) or stats_all.dtype != torch.float32 or not stats_all.is_contiguous():
+        raise ValueError("stats_all must be contiguous float32 [n_ranks,B,K,gamma+1,8]")
+    out = torch.empty((B, K, gamma, 3), dtype=torch.float64, device=dev)
+    with torch.cuda.device(dev):
+        rc = load().sgbv_shard_sums(target_shard.data_ptr(), draft_shard.data_ptr(), _dtype_code(target_shard), B, K, gamma,
+                                    Vs, float(temperature), stats_all.data_ptr(), int(stats_all.shape[0]),
+                                    workspace.data_ptr(), workspace.numel(), out.data_ptr(),
+                                    torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_shard_decide(draft_tokens, uniforms, shard_V: int, temperature: float, stats_all, sums_all, workspace) -> VerifyOutput:
+    """Decisions from the gathered sums (identical on every rank); tokens hold the accepted prefix, -1 elsewhere."""
+    B, K, gamma = draft_tokens.shape
+    dev = draft_tokens.device
+    if tuple(sums_all.shape[1:]) != (B, K, gamma, 3) or sums_all.dtype != torch.float64 or not sums_all.is_contiguous() \
+            or sums_all.shape[0] != stats_all.shape[0]:
+        raise ValueError("sums_all must be contiguous float64 [n_ranks,B,K,gamma,3]")
+    if tuple(uniforms.shape) != (B, K * gamma + 1) or uniforms.dtype != torch.float32 or draft_tokens.dtype != torch.int32:
+        raise ValueError("draft_tokens int32 [B,K,gamma], uniforms float32 [B,K*gamma+1]")
+    out = VerifyOutput(torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev),
+                       torch.empty((B, gamma + 1), dtype=torch.int32, device=dev),
+                       torch.empty((B, K, gamma), dtype=torch.float64, device=dev),
+                       torch.empty((B, K, gamma), dtype=torch.float64, device=dev),
+                       torch.empty(B, dtype=torch.int32, device=dev))
+    with torch.cuda.device(dev):
+        rc = load().sgbv_shard_decide(draft_tokens.data_ptr(), uniforms.data_ptr(), B, K, gamma, int(shard_V),
+                                      float(temperature), stats_all.data_ptr(), sums_all.data_ptr(), int(stats_all.shape[0]),
+                                      workspace.data_ptr(), workspace.numel(), out.accept_len.data_ptr(),
+                                      out.draft_idx.data_ptr(), out.tokens.data_ptr(), out.h.data_ptr(),
+                                      out.resmass.data_ptr(), out.status.data_ptr(),
+                                      torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)
+    return out
+
+
+def sgbv_shard_draw(target_shard, draft_shard, v_begin: int, temperature: float, rank: int, workspace, tokens) -> None:
+    """The owning rank writes the extra token's global id into tokens[b, accept_len] (in place)."""
+    B, K, gamma, Vs = _shard_shapes(target_shard, draft_shard)
+    dev = target_shard.device
+    with torch.cuda.device(dev):
+        rc = load().sgbv_shard_draw(target_shard.data_ptr(), draft_shard.data_ptr(), _dtype_code(target_shard), B, K, gamma,
+                                    Vs, int(v_begin), float(temperature), int(rank), workspace.data_ptr(), workspace.numel(),
+                                    tokens.data_ptr(), torch.cuda.current_stream(dev).cuda_stream)
+    if rc != OK:
+        raise SgbvError(rc)

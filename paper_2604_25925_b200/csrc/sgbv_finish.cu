@@ -7,6 +7,7 @@
 //   3. the extra token: inverse CDF of Eq. 4's residual (located through the cached tile sums,
 //      only one tile is recomputed) or of the target row after a full accept.
 #include "sgbv_sample.cuh"
+#include "sgbv_weights.cuh"
 
 namespace sgbv {
 
@@ -17,57 +18,6 @@ constexpr int kMinThreads = 256;   // chain of memory latencies, so more warps p
 constexpr int kMaxWarps = kMaxThreads / 32;
 constexpr int kTilesInSmem = 4096;  // rows up to 2^20 entries keep the bonus row's tile sums in shared memory
 static_assert(kMinThreads >= kTile, "one thread per element of a tile");
-
-// 1 - (1-u)^K as the geometric sum u (1 + (1-u) + ... + (1-u)^(K-1)): all terms are positive, so
-// a tiny u keeps its full relative accuracy, and no transcendental function is needed.
-__device__ __forceinline__ double gfun(double u, int K) {
-    if (u >= 1.0) return 1.0;
-    if (!(u > 0.0)) return 0.0;
-    const double v = 1.0 - u;
-    double sum = 1.0;
-    for (int j = 1; j < K; ++j) sum = fma(sum, v, 1.0);
-    return u * sum;
-}
-
-__device__ __forceinline__ double clamp01(double x) {
-    if (!(x > 0.0)) return 0.0;
-    return x > 1.0 ? 1.0 : x;
-}
-
-// Eq. 2 from the three cached sums of the row that follows the sub-block (all divided by Zq):
-//   R = sum_x q (1 - min{c p/q,1})^K,  Dp = sum_x max(c p - q, 0),  M = sum_x q (c-t)^2 Q(t).
-// numerator/a   = R                                  (c >= 1)
-//               = M + K (1-c)^(K-1) Dp               (c <  1; equals R - (1-c)^K term by term)
-// denominator/a = numerator/a + g(b)/a - g(min(c,1))
-__device__ double weight_sub(double la, double lb, double R, double Dp, double M, int K, bool below_one) {
-    const double a = exp_short(la), b = exp_short(lb), c = exp_short(lb - la);
-    const double gb = gfun(b, K);
-    if (!(a > 0.0)) return gb > 0.0 ? 0.0 : 1.0;
-    double num, extra;
-    if (below_one) {  // decided on the float32 c the reduction pass used
-        double pw = 1.0;
-        for (int j = 1; j < K; ++j) pw *= (1.0 - c);
-        num = M + (double)K * pw * Dp;
-        extra = (K == 1) ? 0.0 : gb / a - gfun(c, K);
-    } else {
-        num = R;
-        extra = gb / a - 1.0;
-    }
-    if (extra < 0.0) extra = 0.0;
-    const double den = num + extra;
-    if (!(den > 1e-12 * (gb / a + 1.0))) return 1.0;  // 0/0: accept, as single-draft GBV does
-    return clamp01(num / den);
-}
-
-// Eq. 3.
-__device__ double weight_full(double la, double lb, int K) {
-    const double a = exp_short(la), b = exp_short(lb);
-    double c = exp_short(lb - la);
-    if (!(a > 0.0) || c > 1.0) c = 1.0;
-    const double den = gfun(b, K);
-    if (!(den > 0.0)) return 0.0;
-    return clamp01(a * gfun(c, K) / den);
-}
 
 template <typename T>
 __global__ void __launch_bounds__(kMaxThreads)
@@ -249,43 +199,8 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
 
     // ---- 2. scan (Algorithm 1), warp 0 ---------------------------------------------------------
     if (wid == 0) {
-        // The state is bit sets over the lengths 1..gamma (bit i-1 = length i): pass (shared memory, left by
-        // the weights above) = the lengths whose Bernoulli trial succeeds (eta < h); rej (registers, lane l
-        // owns drafts l and l + 32) = the lengths at which the draft entered H.  A draft's walk over i = tau+1..gamma does not
-        // depend on its own progress (the start is fixed when the draft is entered, H only holds earlier
-        // drafts), so it is evaluated for all lengths at once: the accepted length is the largest one in
-        // the range whose trial passes and whose sub-block is not in H.
-        auto low = [](int l) { return l >= 64 ? ~0ull : (1ull << l) - 1ull; };  // lengths 1..l
-        unsigned long long rej0 = 0, rej1 = 0;
-        int tau = 0, f = -1;
-        for (int k = 0; k < K; ++k) {
-            const unsigned long long passk = pass_s[k];
-            // common prefix of draft k with this lane's drafts; only earlier drafts can be in H
-            const int l0 = (lane < k) ? lcp_s[k * K + lane] : 0;
-            const int l1 = (lane + 32 < k) ? lcp_s[k * K + lane + 32] : 0;
-            // lengths at which an earlier draft with the same prefix of that length entered H
-            const unsigned long long mine = (rej0 & low(l0)) | (rej1 & low(l1));
-            // union over the lanes, through shared memory
-            if (lane == 0) sh_or[0] = sh_or[1] = 0u;
-            __syncwarp();
-            if ((unsigned)mine) atomicOr(&sh_or[0], (unsigned)mine);
-            if ((unsigned)(mine >> 32)) atomicOr(&sh_or[1], (unsigned)(mine >> 32));
-            __syncwarp();
-            const unsigned long long inH = ((unsigned long long)sh_or[1] << 32) | (unsigned long long)sh_or[0];
-            __syncwarp();
-            const unsigned long long range = low(g) & ~low(tau);  // lengths tau+1..gamma
-            const unsigned long long acc = passk & ~inH & range;
-            const unsigned long long rejk = range & ~acc;
-            if (acc != 0ull) {
-                tau = 64 - __clzll((long long)acc);
-                f = k;
-            }
-            if (lane == (k & 31)) {
-                if (k < 32) rej0 = rejk;
-                else rej1 = rejk;
-            }
-            if (tau == g) break;  // the whole block was accepted
-        }
+        int tau, f;
+        scan_block(pass_s, lcp_s, K, g, sh_or, tau, f);
         if (lane == 0) {
             sh_i[0] = tau;
             sh_i[1] = f;

@@ -198,7 +198,21 @@ int run(const Launch &L) {
     return cudaGetLastError() == cudaSuccess ? 3 : SGBV_ERR_CUDA;
 }
 
+template <typename T>
+int run_otreduce(const Launch &L) {
+    const Shape &s = L.s;
+    const unsigned grid = (unsigned)(s.B * s.cpr * s.gamma) * (unsigned)s.nsplit;
+    otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>((const T *)L.zq, (const T *)L.zp, s, L.ws.rows, L.ws.wpart,
+                                                       L.ws.dpart, L.ws.mpart);
+    return cudaGetLastError() == cudaSuccess ? 1 : SGBV_ERR_CUDA;
+}
+
 }  // namespace
+
+// the second sweep alone, over rows whose records are already in place
+int launch_otreduce(const Launch &L) {
+    return L.dtype == SGBV_DTYPE_BF16 ? run_otreduce<uint16_t>(L) : run_otreduce<float>(L);
+}
 
 int launch_twopass(const Launch &L) {
     return L.dtype == SGBV_DTYPE_BF16 ? run<uint16_t>(L) : run<float>(L);
