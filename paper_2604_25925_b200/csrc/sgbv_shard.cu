@@ -161,6 +161,101 @@ shard_stats_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, c
     }
 }
 
+// The same records in one pass over memory, for shards whose rows can be read in 16-byte pieces: every lane keeps a
+// running (max, sum relative to it) per tensor over the pieces it reads; the CTA merges them in a fixed order.
+struct Running {
+    float m, s;
+};
+
+__device__ __forceinline__ void running_add(Running &o, const float (&z)[kTile / 32], float scale, bool &bad) {
+    float cm = z[0];
+#pragma unroll
+    for (int e = 0; e < kTile / 32; ++e) {
+        bad |= (z[e] != z[e]) | (z[e] == INFINITY);
+        cm = fmaxf(cm, z[e]);
+    }
+    if (cm > o.m) {  // (an empty sum stays empty: 0 * 2^-inf = 0)
+        o.s *= exp2f((o.m - cm) * scale);
+        o.m = cm;
+    }
+    if (o.m > -INFINITY) {
+#pragma unroll
+        for (int e = 0; e < kTile / 32; ++e) o.s += exp2f((z[e] - o.m) * scale);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+shard_stats_pieces_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const int32_t *__restrict__ tok,
+                          Shape s, int v_begin, int V_total, float *__restrict__ out) {
+    const int row = blockIdx.x;
+    const int i = row % (s.gamma + 1), bk = row / (s.gamma + 1);
+    const bool has_p = i < s.gamma;
+    const T *zq = zq_all + (size_t)row * s.V;
+    const T *zp = zp_all + ((size_t)bk * s.gamma + (has_p ? i : 0)) * s.V;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    constexpr int kW = kThreads / 32;
+    __shared__ float red[4][kW];
+    Running q{-INFINITY, 0.0f}, p{-INFINITY, 0.0f};
+    bool bad = false;
+    for (int t = wid * 2; t < s.ntiles; t += 2 * kW) {  // two cells of both tensors in flight per warp
+        float a[2][kTile / 32], b[2][kTile / 32];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            load_tile_pieces<T>(zq, t + e, t + e < s.ntiles, s.V, lane, a[e]);
+            load_tile_pieces<T>(zp, t + e, has_p && t + e < s.ntiles, s.V, lane, b[e]);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            running_add(q, a[e], s.scale, bad);
+            running_add(p, b[e], s.scale, bad);
+        }
+    }
+    const float mq_w = warp_max(q.m), mp_w = warp_max(p.m);
+    if (lane == 0) {
+        red[0][wid] = mq_w;
+        red[1][wid] = mp_w;
+    }
+    bad = __syncthreads_or(bad);
+    const float mq = warp_max(lane < kW ? red[0][lane] : -INFINITY);
+    const float mp = warp_max(lane < kW ? red[1][lane] : -INFINITY);
+    float sq = q.m > -INFINITY ? q.s * exp2f((q.m - mq) * s.scale) : 0.0f;
+    float sp = p.m > -INFINITY ? p.s * exp2f((p.m - mp) * s.scale) : 0.0f;
+    sq = warp_sum(sq);
+    sp = warp_sum(sp);
+    if (lane == 0) {
+        red[2][wid] = sq;
+        red[3][wid] = sp;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float a = 0.0f, b = 0.0f;
+        for (int w = 0; w < kW; ++w) {  // fixed order
+            a += red[2][w];
+            b += red[3][w];
+        }
+        int flags = bad ? SGBV_STATUS_NONFINITE_LOGIT : 0;
+        float zqt = -INFINITY, zpt = -INFINITY;
+        if (has_p) {
+            const int t = tok[(size_t)bk * s.gamma + i];
+            if (t < 0 || t >= V_total) flags |= SGBV_STATUS_TOKEN_RANGE;
+            else if (t >= v_begin && t < v_begin + s.V) {
+                zqt = ld_logit(zq, t - v_begin);
+                zpt = ld_logit(zp, t - v_begin);
+            }
+        }
+        float *o = out + (size_t)row * kRec;
+        o[0] = mq;
+        o[1] = a;
+        o[2] = has_p ? mp : -INFINITY;
+        o[3] = has_p ? b : 0.0f;
+        o[4] = zqt;
+        o[5] = zpt;
+        o[6] = (float)flags;
+        o[7] = 0.0f;
+    }
+}
+
 // ---- phase 2 ----------------------------------------------------------------------------------------------------
 struct RowStats {
     double Zq, Zp;
@@ -191,35 +286,47 @@ __device__ RowStats combine_stats(const float *__restrict__ stats_all, int R, si
     return o;
 }
 
-// One thread per draft chain: normalisers, c_i and kappa_i of its gamma rows, as the one-device path computes them.
-__global__ void shard_chain_kernel(const float *__restrict__ stats_all, int R, Shape s, RowInfo *__restrict__ rows,
-                                   double *__restrict__ ltok) {
-    const int bk = blockIdx.x * blockDim.x + threadIdx.x;
-    if (bk >= s.B * s.K) return;
+// Normalisers, c_i and kappa_i of every row, as the one-device path computes them.  One thread per row (b,k,i)
+// combines the shards' records (the costly part: one float64 exponential per shard and tensor), a CTA holds whole
+// chains, and every thread then adds up the token log-probabilities before its row in the order of a running sum.
+constexpr int kChainThreads = 256;
+__global__ void __launch_bounds__(kChainThreads)
+shard_chain_kernel(const float *__restrict__ stats_all, int R, Shape s, int chains_per_cta,
+                   RowInfo *__restrict__ rows, double *__restrict__ ltok) {
+    __shared__ double lq_s[kChainThreads], lp_s[kChainThreads];
+    const int tid = threadIdx.x;
+    const int chain = tid / s.gamma, i = tid % s.gamma;
+    const int bk = blockIdx.x * chains_per_cta + chain;
+    const bool mine = chain < chains_per_cta && bk < s.B * s.K;
     const size_t nrows = (size_t)s.B * s.K * (s.gamma + 1);
-    double la = 0.0, lb = 0.0;
-    for (int i = 0; i < s.gamma; ++i) {
-        const RowStats st = combine_stats(stats_all, R, nrows, (size_t)bk * (s.gamma + 1) + i, s.scale);
-        RowInfo ri;
-        ri.Zq = st.Zq;
-        ri.Zp = st.Zp;
-        ri.mq = st.mq;
-        ri.mp = st.mp;
-        const double c = exp(lb - la);
-        ri.c = (float)c;
-        ri.kappa = (float)(c * st.Zq / st.Zp);
-        ri.flags = st.flags;
-        if (!(st.mq > -INFINITY) || !(st.mp > -INFINITY)) ri.flags |= SGBV_STATUS_NONFINITE_LOGIT;
-        ri.pad_ = 0;
-        const size_t r = (size_t)bk * s.gamma + i;
-        rows[r] = ri;
-        const double lq = ((double)st.zqt - (double)st.mq) * s.inv_T - log(st.Zq);
-        const double lp = ((double)st.zpt - (double)st.mp) * s.inv_T - log(st.Zp);
-        ltok[2 * r] = lq;
-        ltok[2 * r + 1] = lp;
-        la += lq;
-        lb += lp;
+    RowStats st{};
+    if (mine) {
+        st = combine_stats(stats_all, R, nrows, (size_t)bk * (s.gamma + 1) + i, s.scale);
+        lq_s[tid] = ((double)st.zqt - (double)st.mq) * s.inv_T - log(st.Zq);
+        lp_s[tid] = ((double)st.zpt - (double)st.mp) * s.inv_T - log(st.Zp);
     }
+    __syncthreads();
+    if (!mine) return;
+    double la = 0.0, lb = 0.0;
+    for (int j = 0; j < i; ++j) {
+        la += lq_s[chain * s.gamma + j];
+        lb += lp_s[chain * s.gamma + j];
+    }
+    RowInfo ri;
+    ri.Zq = st.Zq;
+    ri.Zp = st.Zp;
+    ri.mq = st.mq;
+    ri.mp = st.mp;
+    const double c = exp(lb - la);
+    ri.c = (float)c;
+    ri.kappa = (float)(c * st.Zq / st.Zp);
+    ri.flags = st.flags;
+    if (!(st.mq > -INFINITY) || !(st.mp > -INFINITY)) ri.flags |= SGBV_STATUS_NONFINITE_LOGIT;
+    ri.pad_ = 0;
+    const size_t r = (size_t)bk * s.gamma + i;
+    rows[r] = ri;
+    ltok[2 * r] = lq_s[tid];
+    ltok[2 * r + 1] = lp_s[tid];
 }
 
 // One warp per row: the totals of the shard's cell sums (float64, fixed order).
@@ -491,12 +598,19 @@ int sgbv_shard_stats(const void *target_shard, const void *draft_shard, int dtyp
         return SGBV_ERR_ALIGN;
     const Shape s = shard_shape(B, K, gamma, shard_V, temperature);
     const unsigned grid = (unsigned)((size_t)B * K * (gamma + 1));
-    if (dtype == SGBV_DTYPE_BF16)
-        shard_stats_kernel<uint16_t><<<grid, kThreads, 0, (cudaStream_t)stream>>>(
-            (const uint16_t *)target_shard, (const uint16_t *)draft_shard, draft_tokens, s, v_begin, V, out_stats);
-    else
-        shard_stats_kernel<float><<<grid, kThreads, 0, (cudaStream_t)stream>>>(
-            (const float *)target_shard, (const float *)draft_shard, draft_tokens, s, v_begin, V, out_stats);
+    cudaStream_t st = (cudaStream_t)stream;
+    // rows that start on 16-byte boundaries are read in 16-byte pieces, in one pass
+    const bool pieces = ((uintptr_t)target_shard % 16 == 0) && ((uintptr_t)draft_shard % 16 == 0) &&
+                        (shard_V % (16 / (int)esz) == 0);
+    if (dtype == SGBV_DTYPE_BF16) {
+        const uint16_t *zq = (const uint16_t *)target_shard, *zp = (const uint16_t *)draft_shard;
+        if (pieces) shard_stats_pieces_kernel<uint16_t><<<grid, kThreads, 0, st>>>(zq, zp, draft_tokens, s, v_begin, V, out_stats);
+        else shard_stats_kernel<uint16_t><<<grid, kThreads, 0, st>>>(zq, zp, draft_tokens, s, v_begin, V, out_stats);
+    } else {
+        const float *zq = (const float *)target_shard, *zp = (const float *)draft_shard;
+        if (pieces) shard_stats_pieces_kernel<float><<<grid, kThreads, 0, st>>>(zq, zp, draft_tokens, s, v_begin, V, out_stats);
+        else shard_stats_kernel<float><<<grid, kThreads, 0, st>>>(zq, zp, draft_tokens, s, v_begin, V, out_stats);
+    }
     return last_error();
 }
 
@@ -516,8 +630,9 @@ int sgbv_shard_sums(const void *target_shard, const void *draft_shard, int dtype
     const ShardSpace w = carve((unsigned char *)workspace, B, K, gamma, s.ntiles);
     if (workspace_bytes < w.total || ((uintptr_t)workspace % kAlign)) return SGBV_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)stream_;
-    const int nbk = B * K;
-    shard_chain_kernel<<<(nbk + 127) / 128, 128, 0, stream>>>(stats_all, n_ranks, s, w.rows, w.ltok);
+    const int nbk = B * K, chains_per_cta = kChainThreads / gamma;  // gamma <= 64: at least four chains per CTA
+    shard_chain_kernel<<<(nbk + chains_per_cta - 1) / chains_per_cta, kChainThreads, 0, stream>>>(
+        stats_all, n_ranks, s, chains_per_cta, w.rows, w.ltok);
     Launch L;
     L.zq = target_shard;
     L.zp = draft_shard;

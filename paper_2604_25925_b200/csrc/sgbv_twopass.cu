@@ -4,7 +4,7 @@
 //   sweep 2  (otreduce_kernel)  per-tile sums of the residual weights (and of the two
 //                               non-negative numerator terms when c_i < 1)
 // It reads each needed logit twice, so it is the fallback, not the fast path.
-#include "sgbv_common.cuh"
+#include "sgbv_sample.cuh"
 
 namespace sgbv {
 
@@ -134,7 +134,7 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
 
 // One warp per 256-element tile: lanes stride the tile, one shuffle reduction per sum.
 template <typename T, bool kNeedAux>
-__device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int t0,
+__device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int K, int t0,
                                              int t1, float *wpart, float *dpart, float *mpart) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (int t = t0 + wid; t < t1; t += kThreads / 32) {
@@ -144,7 +144,7 @@ __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Sha
             float eq = expo(ld_logit(zq, x), ri.mq, s.scale);
             float ep = expo(ld_logit(zp, x), ri.mp, s.scale);
             float w, dp = 0.0f, m2 = 0.0f;
-            element_terms<kNeedAux>(eq, ep, ri.kappa, ri.c, s.K, w, dp, m2);
+            element_terms<kNeedAux>(eq, ep, ri.kappa, ri.c, K, w, dp, m2);
             sw += w;
             sd += dp;
             sm += m2;
@@ -162,7 +162,50 @@ __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Sha
     }
 }
 
-template <typename T>
+// The same sums for rows that can be read in 16-byte pieces: a lane takes 8 entries of a cell of each tensor, two
+// cells per warp are in flight.
+template <typename T, bool kNeedAux>
+__device__ __forceinline__ void reduce_tiles_pieces(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int K,
+                                                    int t0, int t1, float *wpart, float *dpart, float *mpart) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int t = t0 + 2 * wid; t < t1; t += 2 * (kThreads / 32)) {
+        float a[2][kTile / 32], b[2][kTile / 32];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            load_tile_pieces<T>(zq, t + e, t + e < t1, s.V, lane, a[e]);
+            load_tile_pieces<T>(zp, t + e, t + e < t1, s.V, lane, b[e]);
+        }
+        float sw[2] = {0.0f, 0.0f}, sd[2] = {0.0f, 0.0f}, sm[2] = {0.0f, 0.0f};
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+            for (int j = 0; j < kTile / 32; ++j) {  // entries past the row hold -inf and add nothing
+                const float eq = expo(a[e][j], ri.mq, s.scale), ep = expo(b[e][j], ri.mp, s.scale);
+                float w, dp = 0.0f, m2 = 0.0f;
+                element_terms<kNeedAux>(eq, ep, ri.kappa, ri.c, K, w, dp, m2);
+                sw[e] += w;
+                sd[e] += dp;
+                sm[e] += m2;
+            }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            sw[e] = warp_sum(sw[e]);
+            if (kNeedAux) {
+                sd[e] = warp_sum(sd[e]);
+                sm[e] = warp_sum(sm[e]);
+            }
+            if (lane == 0 && t + e < t1) {
+                wpart[t + e] = sw[e];
+                dpart[t + e] = sd[e];
+                mpart[t + e] = sm[e];
+            }
+        }
+    }
+}
+
+// KT: the number of drafts as a compile-time constant (the power in Eq. 2 then unrolls, in the same order of
+// multiplications as the run-time loop), or 0 for the run-time value.
+template <typename T, int KT>
 __global__ void __launch_bounds__(kThreads)
 otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shape s,
                 const RowInfo *__restrict__ rows, float *__restrict__ wpart, float *__restrict__ dpart,
@@ -176,10 +219,33 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
     const RowInfo ri = rows[r];
     const int t0 = sl * s.tiles_per_slice, t1 = min(s.ntiles, t0 + s.tiles_per_slice);
     float *wp = wpart + (size_t)r * s.ntiles, *dp = dpart + (size_t)r * s.ntiles, *mp = mpart + (size_t)r * s.ntiles;
-    if (ri.c < 1.0f)
-        reduce_tiles<T, true>(zq, zp, s, ri, t0, t1, wp, dp, mp);
-    else
-        reduce_tiles<T, false>(zq, zp, s, ri, t0, t1, wp, dp, mp);
+    const int K = KT ? KT : s.K;
+    const bool pieces = (reinterpret_cast<uintptr_t>(zq) % 16 == 0) && (reinterpret_cast<uintptr_t>(zp) % 16 == 0) &&
+                        (s.V % (16 / (int)sizeof(T)) == 0);
+    if (ri.c < 1.0f) {
+        if (pieces) reduce_tiles_pieces<T, true>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
+        else reduce_tiles<T, true>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
+    } else {
+        if (pieces) reduce_tiles_pieces<T, false>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
+        else reduce_tiles<T, false>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
+    }
+}
+
+template <typename T>
+void launch_ot(const Launch &L, unsigned grid) {
+    const Shape &s = L.s;
+    const T *zq = (const T *)L.zq, *zp = (const T *)L.zp;
+#define SGBV_OT(KT) \
+    otreduce_kernel<T, KT><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, L.ws.wpart, L.ws.dpart, L.ws.mpart)
+    switch (s.K) {
+        case 1: SGBV_OT(1); break;
+        case 2: SGBV_OT(2); break;
+        case 3: SGBV_OT(3); break;
+        case 4: SGBV_OT(4); break;
+        case 8: SGBV_OT(8); break;
+        default: SGBV_OT(0); break;
+    }
+#undef SGBV_OT
 }
 
 template <typename T>
@@ -193,7 +259,7 @@ int run(const Launch &L) {
     chain_kernel<T><<<(nbk + 127) / 128, 128, 0, L.stream>>>(zq, zp, L.tok, s, L.ws.part, L.ws.rows,
                                                             L.ws.status, L.carry_loga, L.carry_logb);
     if (L.ev_begin) cudaEventRecord(L.ev_begin, L.stream);
-    otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, L.ws.wpart, L.ws.dpart, L.ws.mpart);
+    launch_ot<T>(L, grid);
     if (L.ev_end) cudaEventRecord(L.ev_end, L.stream);
     return cudaGetLastError() == cudaSuccess ? 3 : SGBV_ERR_CUDA;
 }
@@ -202,8 +268,7 @@ template <typename T>
 int run_otreduce(const Launch &L) {
     const Shape &s = L.s;
     const unsigned grid = (unsigned)(s.B * s.cpr * s.gamma) * (unsigned)s.nsplit;
-    otreduce_kernel<T><<<grid, kThreads, 0, L.stream>>>((const T *)L.zq, (const T *)L.zp, s, L.ws.rows, L.ws.wpart,
-                                                       L.ws.dpart, L.ws.mpart);
+    launch_ot<T>(L, grid);
     return cudaGetLastError() == cudaSuccess ? 1 : SGBV_ERR_CUDA;
 }
 
