@@ -432,6 +432,8 @@ def main():
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--sweep-c5", action="store_true",
                     help="instead of the default line: the 24 points of the B=256, gamma=4, V=32000 sweep, one JSON line")
+    ap.add_argument("--vocab-sharded", action="store_true",
+                    help="instead of the default line: one rank's phases of the vocabulary-sharded form, one JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = args.steps or 3
@@ -452,6 +454,13 @@ def main():
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.vocab_sharded:
+        if world > 1:
+            raise RuntimeError("--vocab-sharded times one rank's phases on one GPU")
+        print(json.dumps({"metric": "verify_steps_per_s", "n_gpus": 1, "data": "synthetic",
+                          "vocab_sharded": vocab_sharded_leg(dev)}))
+        return
 
     if args.sweep_c5:
         if world > 1:
