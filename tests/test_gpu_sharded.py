@@ -131,3 +131,30 @@ def test_argument_checks():
         binding.sgbv_shard_sums(zq, zp, 1.0, stats, small)
     assert "workspace" in str(e.value).lower()
     assert binding.sgbv_shard_workspace_bytes(2, 2, 2, 512) > 0
+
+
+def test_one_rank_over_nccl_runs_the_real_exchanges():
+    """The collectives of ``sharded.verify`` (two all-gathers, one max-all-reduce) on the device through NCCL, with a
+    process group of one rank that holds the whole vocabulary: the only multi-rank plumbing one GPU can exercise."""
+    import socket
+    import torch.distributed as dist
+    if dist.is_initialized():
+        pytest.skip("a process group is already up in this process")
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        cfg = workloads.VerifyConfig("nccl1", B=6, K=3, gamma=4, V=4096, temperature=0.7, alpha=0.85, seed=21)
+        inp = workloads.make_inputs(cfg, device="cuda")
+        out = sharded.verify(inp.target_logits, inp.draft_logits, inp.draft_tokens, inp.uniforms, cfg.temperature, 0,
+                             cfg.V, sharded.TorchExchange())
+        torch.cuda.synchronize()
+    finally:
+        dist.destroy_process_group()
+    ref = oracle.verify(_to_np32(inp.target_logits), _to_np32(inp.draft_logits), inp.draft_tokens.cpu().numpy(),
+                        inp.uniforms.cpu().numpy(), cfg.temperature)
+    rep = compare(ref, out.accept_len.cpu().numpy(), out.draft_idx.cpu().numpy(), out.tokens.cpu().numpy(),
+                  out.h.cpu().numpy(), out.resmass.cpu().numpy(), out.status.cpu().numpy())
+    assert_parity(rep)
