@@ -158,3 +158,16 @@ def test_one_rank_over_nccl_runs_the_real_exchanges():
     rep = compare(ref, out.accept_len.cpu().numpy(), out.draft_idx.cpu().numpy(), out.tokens.cpu().numpy(),
                   out.h.cpu().numpy(), out.resmass.cpu().numpy(), out.status.cpu().numpy())
     assert_parity(rep)
+
+
+@pytest.mark.parametrize("B,K,gamma,V,n_ranks", [(2, 64, 64, 768, 3), (1, 1, 1, 40, 2), (3, 5, 7, 1000, 64), (2, 2, 3, 70000, 2)])
+def test_edge_shapes_sharded(B, K, gamma, V, n_ranks):
+    """The largest draft count and length the interface takes, the smallest problem, as many ranks as it allows (most of
+    them with a handful of entries), and shards longer than the fused kernel's CTA slice."""
+    cfg = workloads.VerifyConfig(f"edge_sharded_{B}_{K}_{gamma}_{V}", B=B, K=K, gamma=gamma, V=V, temperature=0.9, alpha=0.8,
+                                 boost=4.0, seed=77 + V)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    bounds = sharded.shard_bounds(V, n_ranks)
+    bounds = [(lo, hi) for lo, hi in bounds if hi > lo]   # (ranks whose range would be empty hold nothing: left out)
+    rep, _, _ = run_sharded(inp, bounds)
+    assert_parity(rep)
