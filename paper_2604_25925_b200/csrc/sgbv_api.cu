@@ -203,6 +203,7 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         n1 = launch_twopass(L);
         if (n1 < 0) return n1;
     }
+    L.ws.have_aux = fused ? 0 : 1;  // the two-sweep path writes the extra sums of rows with c < 1, the fused kernel does not
     int n2 = launch_finish(L);
     if (own_dev >= 0 && L.ws.ratio_used) {
         // a walk that cleared the words itself is followed by a finishing kernel that puts them back: the

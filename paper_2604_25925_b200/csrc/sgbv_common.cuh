@@ -46,6 +46,8 @@ struct Workspace {
                         // published yet") whenever no call is in flight
     double *cut;        // [B*cpr]: c handed from the cluster that walks the head of a chain to the one that walks its tail
                         // (chain walk of the fused kernel; preset to the NaN pattern when any range cuts a chain)
+    int have_aux;       // dpart and mpart hold the two extra sums of the rows with c < 1 (the two-sweep path writes them);
+                        // 0: the finishing kernel works them out itself for the rows whose Eq. 2 needs them
     int ratio_used;     // the streaming kernel walked rows: the finishing kernel puts the NaN pattern back
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory

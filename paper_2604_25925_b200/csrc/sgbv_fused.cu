@@ -654,8 +654,10 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
         }
         float *wp = p.ws.wpart + r_a * s.ntiles + first_cell;
         // The common case by far has nothing to decide per cell: a warp with all its cells, rows before and after,
-        // no partial cell, the plain kind of row.  Its loop body is straight-line code.
-        const bool steady = ncw == kCellsPerWarp && has_a && more && tail_j < 0 && !(rs.c < 1.0f);
+        // no partial cell.  Its loop body is straight-line code.  (Rows with c < 1 get no special treatment here: the
+        // two extra sums that Eq. 2 may need for them are the finishing kernel's business, row by row and only where
+        // the plain form of the numerator would cancel.)
+        const bool steady = ncw == kCellsPerWarp && has_a && more && tail_j < 0;
         if (steady) {
 #pragma unroll
             for (int j = 0; j < kCellsPerWarp; ++j) {
@@ -677,28 +679,6 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
                                p_d + (size_t)slot * kStrideBytes, kHalfBytes, full_u32 + 8u * (uint32_t)slot, is_lane0,
                                kHalfBytes);
                 first_sweep_store(taddr + 16u * (uint32_t)j, s.scale, eq_, ep_, mq[j], mp[j], sq[j], sp[j]);
-            }
-        } else if (has_a && rs.c < 1.0f) {  // the rare kind of row: two more sums per cell
-            float *dp = p.ws.dpart + r_a * s.ntiles + first_cell, *mpp = p.ws.mpart + r_a * s.ntiles + first_cell;
-            float2 coef[KT > 2 ? KT - 2 : 1];
-            if (KT > 2) {
-                float vj = 1.0f;
-#pragma unroll
-                for (int t = 1; t <= KT - 2; ++t) {
-                    vj *= 1.0f - rs.c;
-                    coef[t - 1] = splat((float)(t + 1) * vj);
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < kCellsPerWarp; ++j) {
-                if (j < ncw) {  // warp-uniform
-                    float aux[2];
-                    second_sweep_cell<KT, true>(taddr + 16u * (uint32_t)j, fmq[j], rt[j], rs, s.K, coef,
-                                                fmp_stash + j * kFThreads, wsum[j], aux[0], aux[1]);
-                    warp_sum_multi<2>(aux, lane);  // the two extra sums of the cell leave right away
-                    if ((lane & 15) == 0) ((lane & 16) ? mpp : dp)[j * kFWarps] = aux[0];
-                    if (has_b) SGBV_FIRST_SWEEP_CELL(j, q_b, p_b, q_d, p_d, more);
-                }
             }
         } else {
 #pragma unroll

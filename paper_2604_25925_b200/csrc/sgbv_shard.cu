@@ -422,7 +422,7 @@ shard_decide_kernel(const int32_t *__restrict__ tok_all, const float *__restrict
         const double la = prefix(la_s + k * (g + 1), i), lb = prefix(lb_s + k * (g + 1), i);
         if (out_resmass) out_resmass[(size_t)b * KG + n] = invalid ? NAN : exp_short(la) * Rr;
         if (i >= 1) {
-            const double hv = weight_sub(la, lb, Rr, D_s[n] * inv_Zq, M_s[n] * inv_Zq, K, ri.c < 1.0f);
+            const double hv = weight_sub(la, lb, Rr, D_s[n] * inv_Zq, M_s[n] * inv_Zq, K, ri.c < 1.0f, true);
             if ((double)u_s[k * g + i - 1] < hv) atomicOr(&pass_s[k], 1ull << (i - 1));
             if (out_h) out_h[(size_t)b * KG + k * g + i - 1] = invalid ? NAN : hv;
         }

@@ -25,9 +25,10 @@ __device__ __forceinline__ double clamp01(double x) {
 // Eq. 2 from the three cached sums of the row that follows the sub-block (all divided by Zq):
 //   R = sum_x q (1 - min{c p/q,1})^K,  Dp = sum_x max(c p - q, 0),  M = sum_x q (c-t)^2 Q(t).
 // numerator/a   = R                                  (c >= 1)
-//               = M + K (1-c)^(K-1) Dp               (c <  1; equals R - (1-c)^K term by term)
+//               = M + K (1-c)^(K-1) Dp               (c <  1, `exact`; equals R - (1-c)^K term by term)
+//               = R - (1-c)^K                        (c <  1, not `exact`: only where plain_form_is_safe says so)
 // denominator/a = numerator/a + g(b)/a - g(min(c,1))
-static __device__ double weight_sub(double la, double lb, double R, double Dp, double M, int K, bool below_one) {
+static __device__ double weight_sub(double la, double lb, double R, double Dp, double M, int K, bool below_one, bool exact) {
     const double a = exp_short(la), b = exp_short(lb), c = exp_short(lb - la);
     const double gb = gfun(b, K);
     if (!(a > 0.0)) return gb > 0.0 ? 0.0 : 1.0;
@@ -35,7 +36,7 @@ static __device__ double weight_sub(double la, double lb, double R, double Dp, d
     if (below_one) {  // decided on the float32 c the reduction pass used
         double pw = 1.0;
         for (int j = 1; j < K; ++j) pw *= (1.0 - c);
-        num = M + (double)K * pw * Dp;
+        num = exact ? M + (double)K * pw * Dp : fmax(R - pw * (1.0 - c), 0.0);
         extra = (K == 1) ? 0.0 : gb / a - gfun(c, K);
     } else {
         num = R;
@@ -45,6 +46,16 @@ static __device__ double weight_sub(double la, double lb, double R, double Dp, d
     const double den = num + extra;
     if (!(den > 1e-12 * (gb / a + 1.0))) return 1.0;  // 0/0: accept, as single-draft GBV does
     return clamp01(num / den);
+}
+
+// For c < 1 the numerator of Eq. 2 over a is R - (1-c)^K, a difference of two numbers of which R carries the rounding
+// of a float32 vocabulary sum (a few 1e-7 relative).  As long as (1-c)^K is at most half of R the difference loses at
+// most one bit of that; beyond (p close to q on the part of the vocabulary that matters) the sums Dp and M, whose
+// terms are all non-negative, are needed.
+static __device__ bool plain_form_is_safe(double R, double c, int K) {
+    double pw = 1.0;
+    for (int j = 0; j < K; ++j) pw *= (1.0 - c);
+    return pw <= 0.5 * R;
 }
 
 // Eq. 3.
