@@ -112,7 +112,7 @@ int grow(void **ptr, size_t *have, size_t need, size_t preset_head = 0) {
 
 thread_local int t_last_launches = 0;
 thread_local const char *t_last_kernel = "none";
-int g_opt_path = 0, g_opt_cluster = 0, g_opt_max_clusters = 0, g_opt_walk = 0, g_opt_poll_us = 0, g_opt_withhold = 0;
+int g_opt_path = 0, g_opt_cluster = 0, g_opt_max_clusters = 0, g_opt_walk = 0, g_opt_poll_us = 0, g_opt_withhold = 0, g_opt_aux = 0;
 
 // Optional timing of the dominant kernel: event pairs recorded around it, summed on request.
 struct Profile {
@@ -191,7 +191,8 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
     bool fused = g_opt_path != 1 && fused_supported(L);
     L.ws.prestatus = nullptr;
     bool walked_rows = false;
-    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows) : 0;
+    bool aux_apart = false;
+    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows, &aux_apart) : 0;
     if (n1 < 0) return n1;
     L.ws.ratio_used = (n1 > 0 && walked_rows) ? 1 : 0;
     if (n1 == 0) {
@@ -203,7 +204,16 @@ int verify_device(const void *zq, const void *zp, int dtype, const int32_t *tok,
         n1 = launch_twopass(L);
         if (n1 < 0) return n1;
     }
-    L.ws.have_aux = fused ? 0 : 1;  // the two-sweep path writes the extra sums of rows with c < 1, the fused kernel does not
+    // the extra sums of Eq. 2 for rows with c < 1: written for all such rows by the two-sweep path and, for small and
+    // medium problems, by the fused kernel; for large ones it leaves them to kernels of their own, which do the few rows
+    // that need them
+    L.ws.have_aux = 1;
+    if (fused && aux_apart) {
+        const int na = launch_auxreduce(L);
+        if (na < 0) return na;
+        n1 += na;
+        L.ws.have_aux = 2;
+    }
     int n2 = launch_finish(L);
     if (own_dev >= 0 && L.ws.ratio_used) {
         // a walk that cleared the words itself is followed by a finishing kernel that puts them back: the
@@ -372,7 +382,8 @@ int sgbv_modify(const void *target_logits, const void *draft_logits, int dtype, 
     L.carry_logb = log_b;
     bool fused = g_opt_path != 1 && fused_supported(L);
     bool walked_rows = false;
-    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows) : 0;
+    bool aux_apart = false;  // (Algorithm 2 needs no extra sums: its draw only uses Eq. 4's weights)
+    int n1 = fused ? launch_fused(L, L.ws.error, &walked_rows, &aux_apart) : 0;
     if (n1 < 0) return n1;
     if (n1 == 0) {
         if (g_opt_path == 2) return SGBV_ERR_SHAPE;
@@ -524,10 +535,13 @@ int sgbv_set_option(const char *name, int value) {
     } else if (!strcmp(name, "withhold")) {
         if (value < 0 || value > 1) return SGBV_ERR_SHAPE;
         g_opt_withhold = value;
+    } else if (!strcmp(name, "aux")) {
+        if (value < 0 || value > 2) return SGBV_ERR_SHAPE;
+        g_opt_aux = value;
     } else {
         return SGBV_ERR_SHAPE;
     }
-    fused_set_options(g_opt_cluster, g_opt_max_clusters, g_opt_walk, g_opt_poll_us, g_opt_withhold);
+    fused_set_options(g_opt_cluster, g_opt_max_clusters, g_opt_walk, g_opt_poll_us, g_opt_withhold, g_opt_aux);
     return SGBV_OK;
 }
 

@@ -32,7 +32,7 @@ struct RowInfo {
     float c;        // c = p(x_k^i)/q(x_k^i), ratio of the joint prefix probabilities (c < 1 selects
                     // the cancellation-free numerator)
     int32_t flags;  // SGBV_STATUS_NONFINITE_LOGIT if the streaming pass found the row pair unusable
-    int32_t pad_;
+    int32_t pad_;   // 1: dpart/mpart hold this row's extra sums although only some rows have them (Workspace::have_aux = 2)
 };
 
 struct Workspace {
@@ -46,8 +46,9 @@ struct Workspace {
                         // published yet") whenever no call is in flight
     double *cut;        // [B*cpr]: c handed from the cluster that walks the head of a chain to the one that walks its tail
                         // (chain walk of the fused kernel; preset to the NaN pattern when any range cuts a chain)
-    int have_aux;       // dpart and mpart hold the two extra sums of the rows with c < 1 (the two-sweep path writes them);
-                        // 0: the finishing kernel works them out itself for the rows whose Eq. 2 needs them
+    int have_aux;       // which rows with c < 1 have their two extra sums in dpart and mpart: 1 = all of them (two-sweep
+                        // path, row walk of the fused kernel), 2 = those marked RowInfo::pad_ = 1 (chain walk of the fused
+                        // kernel followed by auxreduce_kernel); the others take the plain form of Eq. 2's numerator
     int ratio_used;     // the streaming kernel walked rows: the finishing kernel puts the NaN pattern back
     float *bonus;       // [B][2][ntiles]: per-tile sums and maxima of the row a bonus token is drawn from
     int bonus_in_smem;  // set by the finishing kernel's launcher: those tile sums fit its shared memory
@@ -183,6 +184,7 @@ struct Launch {
 };
 
 int launch_twopass(const Launch &L);  // statistics + chain + reduction, returns launches or <0
+int launch_auxreduce(const Launch &L); // the extra sums of Eq. 2 for the rows that need them (behind the fused chain walk)
 int launch_finish(const Launch &L);   // weights, scan, extra token
 // Algorithm 2's draw per batch row from the cell sums of a gamma = 1 launch with carried logs
 int launch_modify_finish(const Launch &L, const float *u, int32_t *out_token, double *out_loga, double *out_logb,
@@ -196,7 +198,8 @@ bool fused_supported(const Launch &L);
 // single-read cluster path for steps A1-A3: launches (> 0), 0 if it declined before launching
 // anything (the caller then takes the two-sweep path), or < 0
 // *walked_rows: the kernel used (and consumed the preset of) ws.ratio
-int launch_fused(const Launch &L, int *error_flag, bool *walked_rows);
-void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold);
+// *aux_apart: it left the two extra sums of the rows with c < 1 to launch_auxreduce
+int launch_fused(const Launch &L, int *error_flag, bool *walked_rows, bool *aux_apart);
+void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold, int aux);
 
 }  // namespace sgbv

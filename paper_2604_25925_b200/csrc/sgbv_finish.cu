@@ -83,7 +83,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
         const int k = n / g, i = n % g;
         const size_t r = ((size_t)b * K + k) * g + i;
         const RowInfo ri = ws.rows[r];
-        const bool aux = ws.have_aux && ri.c < 1.0f;
+        const bool aux = ri.c < 1.0f && (ws.have_aux == 1 || ri.pad_ == 1);
         const float *wp = ws.wpart + r * s.ntiles, *dp = ws.dpart + r * s.ntiles, *mp = ws.mpart + r * s.ntiles;
         double sw = 0.0, sd = 0.0, sm = 0.0;
         for (int t0 = 0; t0 < s.ntiles; t0 += 128) {  // four independent loads per array in flight
@@ -112,9 +112,7 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
             W_s[n] = sw;
             D_s[n] = sd;
             M_s[n] = sm;
-            // the streaming kernel leaves the two extra sums of a row with c < 1 to this kernel: they are worked out
-            // below, for the rows whose numerator of Eq. 2 would cancel in its plain form
-            exact_s[n] = aux || (!ws.have_aux && i >= 1 && ri.c < 1.0f && !plain_form_is_safe(sw / ri.Zq, (double)ri.c, K));
+            exact_s[n] = aux;
         }
     }
 
@@ -147,41 +145,6 @@ finish_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, const 
     __syncthreads();
     const int status_in = sh_flags & (SGBV_STATUS_TOKEN_RANGE | SGBV_STATUS_NONFINITE_LOGIT);
     const bool invalid = lost || status_in != 0;
-    // ---- the two extra sums of the rows marked above (rare: c < 1 and p close to q where it matters), one row after
-    //      the other, the whole CTA streaming the row pair once more: sum_x max(c p - q, 0) and sum_x q (c-t)^2 Q(t)
-    //      in row-max units, every term non-negative ----------------------------------------------------------------
-    if (!ws.have_aux && !invalid) {
-        for (int n = 0; n < KG; ++n) {
-            if (!exact_s[n]) continue;  // (the same decision in every thread)
-            const int k = n / g, i = n % g;
-            const size_t r = ((size_t)b * K + k) * g + i;
-            const RowInfo ri = ws.rows[r];
-            const T *zq_row = zq_all + (((size_t)b * K + k) * (g + 1) + i) * s.V, *zp_row = zp_all + r * s.V;
-            double sd = 0.0, sm = 0.0;
-            for (int x = tid; x < s.V; x += nthreads) {
-                const float eq = expo(ld_logit(zq_row, x), ri.mq, s.scale), ep = expo(ld_logit(zp_row, x), ri.mp, s.scale);
-                float w, dp, m2;
-                element_terms<true>(eq, ep, ri.kappa, ri.c, K, w, dp, m2);
-                sd += (double)dp;
-                sm += (double)m2;
-            }
-            sd = warp_sum(sd);
-            sm = warp_sum(sm);
-            if (lane == 0) sc.warp[wid] = sd;
-            __syncthreads();
-            const double td = warp_sum(lane < nwarps ? sc.warp[lane] : 0.0);
-            __syncthreads();
-            if (lane == 0) sc.warp[wid] = sm;
-            __syncthreads();
-            const double tm = warp_sum(lane < nwarps ? sc.warp[lane] : 0.0);
-            __syncthreads();
-            if (tid == 0) {
-                D_s[n] = td;
-                M_s[n] = tm;
-            }
-        }
-        __syncthreads();
-    }
     // la_s/lb_s[k][i+1] now hold log q_i(x_k^i), log p_i(x_k^i); every user below adds up the terms it needs
     // itself, in the order of a running sum (at most gamma additions, and no pass and barrier of its own)
     auto prefix = [&](const double *row, int len) {

@@ -63,6 +63,7 @@ struct FusedParams {
     int *error_flag;  // set to 1 if a bounded wait expired
     long long poll_limit;  // cycles a poll of a published ratio may take (row walk)
     int withhold;     // failure-detection test: the first row of every chain does not publish its ratio
+    int aux_here;     // rows with c < 1 get their two extra sums in this kernel (else: the kernels that follow it)
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -654,10 +655,13 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
         }
         float *wp = p.ws.wpart + r_a * s.ntiles + first_cell;
         // The common case by far has nothing to decide per cell: a warp with all its cells, rows before and after,
-        // no partial cell.  Its loop body is straight-line code.  (Rows with c < 1 get no special treatment here: the
-        // two extra sums that Eq. 2 may need for them are the finishing kernel's business, row by row and only where
-        // the plain form of the numerator would cancel.)
-        const bool steady = ncw == kCellsPerWarp && has_a && more && tail_j < 0;
+        // no partial cell.  Its loop body is straight-line code.
+        // Rows with c < 1 may need two more sums for Eq. 2.  Small and medium problems work them out here, for all
+        // such rows (p.aux_here).  Large ones leave them to two kernels that follow this one and only touch the rows
+        // whose plain numerator would cancel, a few per cent: here they slow every row with c < 1, and with it the
+        // whole cluster, by more than half, which is worth two more launches only when the step is long.
+        const bool aux_row = p.aux_here && rs.c < 1.0f;
+        const bool steady = ncw == kCellsPerWarp && has_a && more && tail_j < 0 && !aux_row;
         if (steady) {
 #pragma unroll
             for (int j = 0; j < kCellsPerWarp; ++j) {
@@ -679,6 +683,28 @@ __global__ void __launch_bounds__(W * 32, kCtasPerSm) fused_chain_kernel(const F
                                p_d + (size_t)slot * kStrideBytes, kHalfBytes, full_u32 + 8u * (uint32_t)slot, is_lane0,
                                kHalfBytes);
                 first_sweep_store(taddr + 16u * (uint32_t)j, s.scale, eq_, ep_, mq[j], mp[j], sq[j], sp[j]);
+            }
+        } else if (has_a && aux_row) {  // the rare kind of row: two more sums per cell
+            float *dp = p.ws.dpart + r_a * s.ntiles + first_cell, *mpp = p.ws.mpart + r_a * s.ntiles + first_cell;
+            float2 coef[KT > 2 ? KT - 2 : 1];
+            if (KT > 2) {
+                float vj = 1.0f;
+#pragma unroll
+                for (int t = 1; t <= KT - 2; ++t) {
+                    vj *= 1.0f - rs.c;
+                    coef[t - 1] = splat((float)(t + 1) * vj);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kCellsPerWarp; ++j) {
+                if (j < ncw) {  // warp-uniform
+                    float aux[2];
+                    second_sweep_cell<KT, true>(taddr + 16u * (uint32_t)j, fmq[j], rt[j], rs, s.K, coef,
+                                                fmp_stash + j * kFThreads, wsum[j], aux[0], aux[1]);
+                    warp_sum_multi<2>(aux, lane);  // the two extra sums of the cell leave right away
+                    if ((lane & 15) == 0) ((lane & 16) ? mpp : dp)[j * kFWarps] = aux[0];
+                    if (has_b) SGBV_FIRST_SWEEP_CELL(j, q_b, p_b, q_d, p_d, more);
+                }
             }
         } else {
 #pragma unroll
@@ -905,6 +931,8 @@ int g_opt_max_clusters = 0;
 int g_opt_walk = 0;        // 0 = automatic, 1 = chains, 2 = rows
 int g_opt_poll_us = 0;     // 0 = about a second
 int g_opt_withhold = 0;
+int g_opt_aux = 0;         // 0 = automatic, 1 = the extra sums of rows with c < 1 in the streaming kernel, 2 = in kernels of their own
+constexpr double kAuxApartMinBytes = 1024.0 * 1024 * 1024;
 
 constexpr int kSmemPerCta = (228 * 1024) / kCtasPerSm - 1024;  // largest dynamic shared memory of one CTA
 constexpr int kDevices = 64;
@@ -961,7 +989,7 @@ int resident_clusters(int dev, int C) {
 }
 
 template <typename T, bool kRow, int KT>
-int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) {
+int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters, bool aux_here) {
     FusedParams fp;
     fp.zq = L.zq;
     fp.zp = L.zp;
@@ -976,6 +1004,7 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
     fp.error_flag = error_flag;
     fp.poll_limit = g_opt_poll_us > 0 ? (long long)g_opt_poll_us * 2000ll : kWaitLimitCycles;
     fp.withhold = g_opt_withhold;
+    fp.aux_here = aux_here ? 1 : 0;
 
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kWarps * 32);
@@ -1011,7 +1040,7 @@ int launch_as(const Launch &L, const Plan &plan, int *error_flag, int clusters) 
 
 // Chooses the cluster size and the walk, then launches.  Returns launches, 0 if declined, or < 0.
 template <typename T, int KT>
-int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
+int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows, bool *aux_apart) {
     const Shape &s = L.s;
     const int cells = s.ntiles;
     const long nchains = (long)s.B * s.cpr, units = nchains * s.gamma;
@@ -1055,14 +1084,20 @@ int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows) {
     const long share = plan.row_mode ? units : nchains;  // what the clusters share out
     if (clusters > share) clusters = (int)share;
     *walked_rows = plan.row_mode != 0;
-    return plan.row_mode ? launch_as<T, true, KT>(L, plan, error_flag, clusters)
-                         : launch_as<T, false, KT>(L, plan, error_flag, clusters);
+    // the extra sums of rows with c < 1: in this kernel, or for long steps (chain walk, 1 GB of logits or more) in the
+    // kernels that the caller queues behind it
+    const double bytes = 2.0 * (double)units * (double)s.V * (double)sizeof(T);
+    const bool aux_here = plan.row_mode || g_opt_aux == 1 || (g_opt_aux == 0 && bytes < kAuxApartMinBytes);
+    *aux_apart = !aux_here;
+    return plan.row_mode ? launch_as<T, true, KT>(L, plan, error_flag, clusters, true)
+                         : launch_as<T, false, KT>(L, plan, error_flag, clusters, aux_here);
 }
 
 }  // namespace
 
-void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold) {
+void fused_set_options(int cluster, int max_clusters, int walk, int poll_us, int withhold, int aux) {
     std::lock_guard<std::mutex> lock(g_plan_mu);
+    g_opt_aux = aux;
     g_opt_withhold = withhold;
     g_opt_walk = walk;
     g_opt_cluster = cluster;
@@ -1079,22 +1114,23 @@ bool fused_supported(const Launch &L) {
 }
 
 template <typename T>
-int dispatch_k(const Launch &L, int *error_flag, bool *walked_rows) {
+int dispatch_k(const Launch &L, int *error_flag, bool *walked_rows, bool *aux_apart) {
     switch (L.s.K) {
-        case 1: return plan_and_launch<T, 1>(L, error_flag, walked_rows);
-        case 2: return plan_and_launch<T, 2>(L, error_flag, walked_rows);
-        case 3: return plan_and_launch<T, 3>(L, error_flag, walked_rows);
-        case 4: return plan_and_launch<T, 4>(L, error_flag, walked_rows);
-        case 8: return plan_and_launch<T, 8>(L, error_flag, walked_rows);
-        default: return plan_and_launch<T, 0>(L, error_flag, walked_rows);
+        case 1: return plan_and_launch<T, 1>(L, error_flag, walked_rows, aux_apart);
+        case 2: return plan_and_launch<T, 2>(L, error_flag, walked_rows, aux_apart);
+        case 3: return plan_and_launch<T, 3>(L, error_flag, walked_rows, aux_apart);
+        case 4: return plan_and_launch<T, 4>(L, error_flag, walked_rows, aux_apart);
+        case 8: return plan_and_launch<T, 8>(L, error_flag, walked_rows, aux_apart);
+        default: return plan_and_launch<T, 0>(L, error_flag, walked_rows, aux_apart);
     }
 }
 
-int launch_fused(const Launch &L, int *error_flag, bool *walked_rows) {
+int launch_fused(const Launch &L, int *error_flag, bool *walked_rows, bool *aux_apart) {
     *walked_rows = false;
+    *aux_apart = false;
     std::lock_guard<std::mutex> lock(g_plan_mu);
-    return L.dtype == SGBV_DTYPE_BF16 ? dispatch_k<uint16_t>(L, error_flag, walked_rows)
-                                      : dispatch_k<float>(L, error_flag, walked_rows);
+    return L.dtype == SGBV_DTYPE_BF16 ? dispatch_k<uint16_t>(L, error_flag, walked_rows, aux_apart)
+                                      : dispatch_k<float>(L, error_flag, walked_rows, aux_apart);
 }
 
 }  // namespace sgbv

@@ -5,6 +5,7 @@
 //                               non-negative numerator terms when c_i < 1)
 // It reads each needed logit twice, so it is the fallback, not the fast path.
 #include "sgbv_sample.cuh"
+#include "sgbv_weights.cuh"
 
 namespace sgbv {
 
@@ -133,7 +134,7 @@ __global__ void chain_kernel(const T *__restrict__ zq_all, const T *__restrict__
 }
 
 // One warp per 256-element tile: lanes stride the tile, one shuffle reduction per sum.
-template <typename T, bool kNeedAux>
+template <typename T, bool kNeedAux, bool kStoreW = true>
 __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int K, int t0,
                                              int t1, float *wpart, float *dpart, float *mpart) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -155,7 +156,7 @@ __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Sha
             sm = warp_sum(sm);
         }
         if (lane == 0) {
-            wpart[t] = sw;
+            if (kStoreW) wpart[t] = sw;
             dpart[t] = sd;
             mpart[t] = sm;
         }
@@ -164,7 +165,7 @@ __device__ __forceinline__ void reduce_tiles(const T *zq, const T *zp, const Sha
 
 // The same sums for rows that can be read in 16-byte pieces: a lane takes 8 entries of a cell of each tensor, two
 // cells per warp are in flight.
-template <typename T, bool kNeedAux>
+template <typename T, bool kNeedAux, bool kStoreW = true>
 __device__ __forceinline__ void reduce_tiles_pieces(const T *zq, const T *zp, const Shape &s, const RowInfo &ri, int K,
                                                     int t0, int t1, float *wpart, float *dpart, float *mpart) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -195,7 +196,7 @@ __device__ __forceinline__ void reduce_tiles_pieces(const T *zq, const T *zp, co
                 sm[e] = warp_sum(sm[e]);
             }
             if (lane == 0 && t + e < t1) {
-                wpart[t + e] = sw[e];
+                if (kStoreW) wpart[t + e] = sw[e];
                 dpart[t + e] = sd[e];
                 mpart[t + e] = sm[e];
             }
@@ -228,6 +229,54 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
     } else {
         if (pieces) reduce_tiles_pieces<T, false>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
         else reduce_tiles<T, false>(zq, zp, s, ri, K, t0, t1, wp, dp, mp);
+    }
+}
+
+// Behind a fused kernel that left the two extra sums of Eq. 2 aside (large problems), two small kernels:
+//   auxflag_kernel  one warp per row: for a row with c < 1 whose numerator R - (1-c)^K would cancel in that plain form
+//                   (plain_form_is_safe; R from the cell sums the fused kernel wrote), the row is put on a list and
+//                   marked in its record (RowInfo::pad_ = 1) for the finishing kernel;
+//   auxwork_kernel  a fixed grid shares out the listed rows in slices of kAuxSliceTiles cells and writes, per cell, the
+//                   sums over max(c p - q, 0) and q (c-t)^2 Q(t) from a second read of the row pair.
+// A few per cent of the rows are listed; the order of the list varies from run to run, the sums do not.
+constexpr int kAuxSliceTiles = 32;
+
+__global__ void __launch_bounds__(kThreads)
+auxflag_kernel(Shape s, RowInfo *__restrict__ rows, const float *__restrict__ wpart, int *__restrict__ list) {
+    const int lane = threadIdx.x & 31;
+    const size_t r = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (r >= (size_t)s.B * s.cpr * s.gamma || r % s.gamma == 0) return;  // Eq. 2 is about sub-blocks of length i >= 1
+    const RowInfo ri = rows[r];
+    if (!(ri.c < 1.0f) || ri.flags) return;
+    double sw = 0.0;
+    for (int t = lane; t < s.ntiles; t += 32) sw += (double)wpart[r * s.ntiles + t];
+    sw = warp_sum(sw);
+    if (plain_form_is_safe(sw / ri.Zq, (double)ri.c, s.K)) return;
+    if (lane == 0) {
+        list[1 + atomicAdd(list, 1)] = (int)r;  // list[0] counts
+        rows[r].pad_ = 1;
+    }
+}
+
+template <typename T, int KT>
+__global__ void __launch_bounds__(kThreads)
+auxwork_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shape s, const RowInfo *__restrict__ rows,
+               const int *__restrict__ list, float *__restrict__ dpart, float *__restrict__ mpart) {
+    const int K = KT ? KT : s.K;
+    const int per_row = (s.ntiles + kAuxSliceTiles - 1) / kAuxSliceTiles;
+    const long items = (long)list[0] * per_row;
+    for (long w = blockIdx.x; w < items; w += gridDim.x) {
+        const int r = list[1 + w / per_row], sl = (int)(w % per_row);
+        const RowInfo ri = rows[r];
+        const int bk = r / s.gamma, i = r % s.gamma;
+        const T *zq = zq_all + ((size_t)bk * s.zq_rows + i) * s.V;
+        const T *zp = zp_all + ((size_t)bk * s.gamma + i) * s.V;
+        const int t0 = sl * kAuxSliceTiles, t1 = min(s.ntiles, t0 + kAuxSliceTiles);
+        float *dp = dpart + (size_t)r * s.ntiles, *mp = mpart + (size_t)r * s.ntiles;
+        const bool pieces = (reinterpret_cast<uintptr_t>(zq) % 16 == 0) && (reinterpret_cast<uintptr_t>(zp) % 16 == 0) &&
+                            (s.V % (16 / (int)sizeof(T)) == 0);
+        if (pieces) reduce_tiles_pieces<T, true, false>(zq, zp, s, ri, K, t0, t1, nullptr, dp, mp);
+        else reduce_tiles<T, true, false>(zq, zp, s, ri, K, t0, t1, nullptr, dp, mp);
     }
 }
 
@@ -272,7 +321,37 @@ int run_otreduce(const Launch &L) {
     return cudaGetLastError() == cudaSuccess ? 1 : SGBV_ERR_CUDA;
 }
 
+template <typename T>
+int run_auxreduce(const Launch &L) {
+    const Shape &s = L.s;
+    const size_t NR = (size_t)s.B * s.cpr * s.gamma;
+    // the list lives where the two-sweep path keeps its slice partials (at least 16 bytes per row), unused here
+    int *list = reinterpret_cast<int *>(L.ws.part);
+    if (cudaMemsetAsync(list, 0, sizeof(int), L.stream) != cudaSuccess) return SGBV_ERR_CUDA;
+    auxflag_kernel<<<(unsigned)((NR + kThreads / 32 - 1) / (kThreads / 32)), kThreads, 0, L.stream>>>(s, L.ws.rows, L.ws.wpart,
+                                                                                                     list);
+    const T *zq = (const T *)L.zq, *zp = (const T *)L.zp;
+    const unsigned grid = 4 * 148;
+#define SGBV_AUX(KT) \
+    auxwork_kernel<T, KT><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, list, L.ws.dpart, L.ws.mpart)
+    switch (s.K) {
+        case 1: SGBV_AUX(1); break;
+        case 2: SGBV_AUX(2); break;
+        case 3: SGBV_AUX(3); break;
+        case 4: SGBV_AUX(4); break;
+        case 8: SGBV_AUX(8); break;
+        default: SGBV_AUX(0); break;
+    }
+#undef SGBV_AUX
+    return cudaGetLastError() == cudaSuccess ? 2 : SGBV_ERR_CUDA;
+}
+
 }  // namespace
+
+// the two extra sums of Eq. 2 for the rows that need them, behind the fused kernel's chain walk
+int launch_auxreduce(const Launch &L) {
+    return L.dtype == SGBV_DTYPE_BF16 ? run_auxreduce<uint16_t>(L) : run_auxreduce<float>(L);
+}
 
 // the second sweep alone, over rows whose records are already in place
 int launch_otreduce(const Launch &L) {

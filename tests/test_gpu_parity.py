@@ -245,7 +245,7 @@ def _slice_fits(V, cluster):
 
 @pytest.mark.parametrize("option", [("path", 1), ("path", 2), ("cluster", 1), ("cluster", 2), ("cluster", 3),
                                     ("cluster", 4), ("cluster", 5), ("cluster", 7), ("cluster", 8),
-                                    ("max_clusters", 3), ("walk", 1), ("walk", 2)])
+                                    ("max_clusters", 3), ("walk", 1), ("walk", 2), ("aux", 1), ("aux", 2)])
 def test_every_kernel_path_and_launch_shape_matches(option):
     """The generic two-sweep kernels and the fused kernel at every cluster size / walk /
     persistent-grid size must all agree with the oracle (automatic choice is covered elsewhere)."""
@@ -266,6 +266,31 @@ def test_every_kernel_path_and_launch_shape_matches(option):
             assert_parity(rep)
     finally:
         binding.set_option(option[0], 0)
+
+
+@pytest.mark.parametrize("K,dtype,alpha,T", [(1, "fp32", 0.8, 1.0), (2, "bf16", 0.9, 0.7), (8, "fp32", 0.9, 1.0),
+                                             (3, "fp32", 0.9995, 1.0), (5, "fp32", 0.99, 0.4), (8, "bf16", 0.9999, 1.0)])
+def test_extra_sums_in_kernels_of_their_own(K, dtype, alpha, T):
+    """Chain walk with the two extra sums of Eq. 2 (rows with c < 1) left to the kernels behind the fused kernel, which
+    only do the rows whose plain numerator would cancel: ordinary drafts (few such rows), drafts nearly equal to the
+    target (nearly all rows with c < 1 qualify), and a draft count without a specialised kernel; and the same inputs
+    with the sums worked out in the fused kernel must give the same weights."""
+    cfg = workloads.VerifyConfig(f"aux_{K}_{dtype}_{alpha}", B=24, K=K, gamma=5, V=40192, dtype=dtype, temperature=T,
+                                 alpha=alpha, seed=300 + K)
+    inp = workloads.make_inputs(cfg, device="cuda")
+    res = {}
+    for aux in (2, 1):
+        binding.set_option("walk", 1)
+        binding.set_option("aux", aux)
+        try:
+            rep, out, _ = run_both(inp)
+            assert_parity(rep)
+            res[aux] = out.h.cpu().numpy()
+            assert binding.last_launch_count() == (4 if aux == 2 else 2)
+        finally:
+            binding.set_option("walk", 0)
+            binding.set_option("aux", 0)
+    np.testing.assert_allclose(res[2], res[1], rtol=2e-5, atol=1e-9)
 
 
 def test_unaligned_views_and_repeated_calls_are_deterministic():
