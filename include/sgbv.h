@@ -295,7 +295,7 @@ int sgbv_profile_end(double *out_total_ms, int *out_records);
  *   "aux"          where the two extra vocabulary sums that Eq. 2 may need for a row with p(x^i) < q(x^i) are worked out:
  *                  1 = in the fused kernel, for every such row; 2 = in two small kernels behind it, for the rows that
  *                  need them (one more read of a few per cent of the rows); 0 = the second for steps of 1 GB of logits
- *                  or more, else the first
+ *                  or more, else the first.  The row walk always works them out itself.
  * and two for the failure-detection test (a bounded device-side wait that runs out, see SGBV_STATUS_TIMEOUT):
  *   "poll_us"      limit, in microseconds, of the row walk's wait for a ratio published by another cluster
  *   "withhold"     1 = the first row of every chain does not publish its ratio
