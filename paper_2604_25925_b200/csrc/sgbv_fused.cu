@@ -397,8 +397,11 @@ __device__ __forceinline__ void second_sweep_cell(uint32_t taddr_cell, float fmq
         const float2 q = eq[e];
         const float2 diff = __ffma2_rn(nkt, ep[e], q);  // q - c p, thread units
         const float2 pos = make_float2(fmaxf(diff.x, 0.0f), fmaxf(diff.y, 0.0f));
-        if (KT == 1) sw = __fadd2_rn(sw, pos);
-        if (KT == 1 && !kAux) continue;
+        if (KT == 1) {  // one draft: Q = 0, the second extra sum vanishes and nothing needs the ratio
+            sw = __fadd2_rn(sw, pos);
+            if (kAux) sd = __fadd2_rn(sd, make_float2(fmaxf(-diff.x, 0.0f), fmaxf(-diff.y, 0.0f)));
+            continue;
+        }
         // r = 1 - min{c p/q, 1}; q = 0 gives -inf or NaN before the clamp, 0 after it
         const float2 t = __fmul2_rn(diff, make_float2(rcp(q.x), rcp(q.y)));
         const float2 r = make_float2(fmaxf(t.x, 0.0f), fmaxf(t.y, 0.0f));
@@ -1087,7 +1090,8 @@ int plan_and_launch(const Launch &L, int *error_flag, bool *walked_rows, bool *a
     // the extra sums of rows with c < 1: in this kernel, or for long steps (chain walk, 1 GB of logits or more) in the
     // kernels that the caller queues behind it
     const double bytes = 2.0 * (double)units * (double)s.V * (double)sizeof(T);
-    const bool aux_here = plan.row_mode || g_opt_aux == 1 || (g_opt_aux == 0 && bytes < kAuxApartMinBytes);
+    // (with one draft the extra sum costs the kernel next to nothing, and most rows with c < 1 would be listed)
+    const bool aux_here = plan.row_mode || g_opt_aux == 1 || (g_opt_aux == 0 && (bytes < kAuxApartMinBytes || s.K == 1));
     *aux_apart = !aux_here;
     return plan.row_mode ? launch_as<T, true, KT>(L, plan, error_flag, clusters, true)
                          : launch_as<T, false, KT>(L, plan, error_flag, clusters, aux_here);
