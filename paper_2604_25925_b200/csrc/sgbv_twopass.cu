@@ -239,7 +239,7 @@ otreduce_kernel(const T *__restrict__ zq_all, const T *__restrict__ zp_all, Shap
 //   auxwork_kernel  a fixed grid shares out the listed rows in slices of kAuxSliceTiles cells and writes, per cell, the
 //                   sums over max(c p - q, 0) and q (c-t)^2 Q(t) from a second read of the row pair.
 // A few per cent of the rows are listed; the order of the list varies from run to run, the sums do not.
-constexpr int kAuxSliceTiles = 32;
+constexpr int kAuxSliceTiles = 16;
 
 __global__ void __launch_bounds__(kThreads)
 auxflag_kernel(Shape s, RowInfo *__restrict__ rows, const float *__restrict__ wpart, int *__restrict__ list) {
@@ -331,7 +331,7 @@ int run_auxreduce(const Launch &L) {
     auxflag_kernel<<<(unsigned)((NR + kThreads / 32 - 1) / (kThreads / 32)), kThreads, 0, L.stream>>>(s, L.ws.rows, L.ws.wpart,
                                                                                                      list);
     const T *zq = (const T *)L.zq, *zp = (const T *)L.zp;
-    const unsigned grid = 4 * 148;
+    const unsigned grid = 8 * 148;
 #define SGBV_AUX(KT) \
     auxwork_kernel<T, KT><<<grid, kThreads, 0, L.stream>>>(zq, zp, s, L.ws.rows, list, L.ws.dpart, L.ws.mpart)
     switch (s.K) {
